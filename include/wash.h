@@ -1,0 +1,211 @@
+/*
+ * wash.h -- C ABI of the B200 WASH population library (libwash.so).
+ *
+ * A population is N copies of one model, held on one GPU as a "stack": every model's
+ * learnable tensors laid end to end in a row of padded_P elements (each tensor starts
+ * on a multiple of 8 elements), the N rows stored either model-major, [N][padded_P],
+ * or coordinate-major, [padded_P][N].  The library runs, in hand-written sm_100a
+ * kernels, the population operators of the WASH paper (Fournier et al., "WASH: Train
+ * your Ensemble with Communication-Efficient Weight Shuffling, then Average"):
+ *
+ *   wash_shuffle / _opt_state / _both   the shuffling step, Eq. 3 and Algorithm 1
+ *   papa_ema                            PAPA's pull toward the consensus, Eq. 1
+ *   population_average                  the averaged model, output of Algorithm 1
+ *   papa_all                            PAPA-all / DART: every model := the average
+ *   wash_consensus_sq                   squared distances to the consensus (Fig. 2)
+ *
+ * Conventions common to all calls
+ *   - Every function returns a wash_status (0 = success, negative = error) and never
+ *     throws, aborts or traps.  wash_last_error() gives a message for the last failure
+ *     of the calling thread.
+ *   - Pointers are HOST pointers unless the comment says DEVICE.  Stacks are DEVICE
+ *     memory BORROWED from the caller: the library never frees, moves or resizes
+ *     them.  The context owns only its small tables.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the default stream).  Kernel
+ *     launches are asynchronous on it; argument errors are reported before any launch.
+ *     Calls on one context must be issued on one stream at a time (the context's
+ *     tables are rewritten in stream order when the probabilities change).
+ *   - Randomness is a pure function of (seed, step, tensor index, coordinate index)
+ *     through Philox4x32-10, so a result does not depend on layout, dtype, grid size,
+ *     kernel variant, or on which of the shuffle entry points produced it.
+ *   - Padding elements of a row are not coordinates: no call reads them into a result
+ *     or writes them.
+ */
+#ifndef WASH_H_
+#define WASH_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct wash_ctx wash_ctx; /* opaque; made by wash_create*, released by wash_destroy */
+
+enum wash_status {
+    WASH_OK = 0,
+    WASH_ERR_ARG = -1,         /* invalid argument (range, NULL, NaN, size mismatch)      */
+    WASH_ERR_STATE = -2,       /* call not valid now (e.g. stack not bound)               */
+    WASH_ERR_ALLOC = -3,       /* host or device allocation failed                        */
+    WASH_ERR_CUDA = -4,        /* a CUDA runtime call or a launch failed                  */
+    WASH_ERR_UNSUPPORTED = -5, /* valid request this build has no kernel for              */
+    WASH_ERR_DEVICE_CHECK = -6 /* a device-side consistency check tripped (wash_check)    */
+};
+enum wash_layout { WASH_LAYOUT_NP = 0 /* [N][padded_P] */, WASH_LAYOUT_PN = 1 /* [padded_P][N] */ };
+enum wash_dtype { WASH_F32 = 0, WASH_BF16 = 1 };
+enum wash_stack { WASH_STACK_PARAMS = 0, WASH_STACK_OPT = 1 };
+enum wash_schedule { WASH_SCHEDULE_DECREASING = 0, WASH_SCHEDULE_CONSTANT = 1, WASH_SCHEDULE_INCREASING = 2 };
+enum wash_mode {
+    WASH_MODE_STREAM = 0, /* one pass that reads the whole stack; writes selected coordinates */
+    WASH_MODE_SPARSE = 1  /* draws the mask first; touches only selected coordinates          */
+};
+
+#define WASH_MAX_N 64            /* largest population                                     */
+#define WASH_ALIGN_ELEMS 8       /* tensors start on a multiple of this many elements      */
+
+/* Counters a shuffle ADDS to (Table 1's "communication volume", measured):
+ *   selected_coords  coordinates that drew "shuffle" (each stands for N values routed
+ *                    through a permutation);
+ *   moved_values     among those, values whose model index changed, i.e. the sum over
+ *                    selected i of #{n : pi_i(n) != n}.
+ * Counted once per coordinate, whether one stack or two were shuffled. */
+typedef struct {
+    uint64_t selected_coords;
+    uint64_t moved_values;
+} wash_stats;
+
+/* ---- context ------------------------------------------------------------------- */
+
+/* Describe a population of N models (2 <= N <= WASH_MAX_N) made of n_tensors tensors,
+ * tensor t holding numel[t] coordinates (0 < numel[t] < 2^32); the tensor's index t
+ * is what the paper's Algorithm 1 calls the layer l when per-layer probabilities are
+ * given.  `device` is the CUDA device ordinal that owns the stacks.  On success *out
+ * is a new context.  Errors: WASH_ERR_ARG, WASH_ERR_ALLOC, WASH_ERR_CUDA. */
+int wash_create(wash_ctx **out, int32_t N, int32_t n_tensors, const int64_t *numel,
+                int32_t layout, int32_t device);
+
+/* As wash_create, for a SHARD of a larger population: segment s holds numel[s]
+ * coordinates that are coordinates coord_begin[s] .. coord_begin[s]+numel[s]-1 of the
+ * global tensor tensor_id[s].  Because the random draws are keyed by the global
+ * (tensor, coordinate), shards processed on different GPUs reproduce the unsharded
+ * result exactly and need no communication.  coord_begin[s] must be a multiple of 4
+ * and coord_begin[s] + numel[s] <= 2^32.  tensor_id / coord_begin may be NULL
+ * (meaning s and 0). */
+int wash_create_segments(wash_ctx **out, int32_t N, int32_t n_segments, const int64_t *numel,
+                         const uint32_t *tensor_id, const int64_t *coord_begin,
+                         int32_t layout, int32_t device);
+
+/* Release the context's tables.  Bound stacks are the caller's and are left alone. */
+int wash_destroy(wash_ctx *ctx);
+
+/* Row geometry: *padded_P = elements per model row; offsets[t] (array of n_tensors,
+ * may be NULL) = element offset of tensor t inside a row.  A stack is N * padded_P
+ * elements; element (n, e) lives at n*padded_P + e (WASH_LAYOUT_NP) or e*N + n
+ * (WASH_LAYOUT_PN). */
+int wash_stack_elems(const wash_ctx *ctx, int64_t *padded_P, int64_t *offsets);
+
+/* Lend a DEVICE buffer of n_elems == N * padded_P elements of `dtype` to the context
+ * as its parameter stack or optimizer-state stack.  The pointer must be 16-byte
+ * aligned.  Passing dev_ptr == NULL unbinds. */
+int wash_bind(wash_ctx *ctx, int32_t stack, int32_t dtype, void *dev_ptr, int64_t n_elems);
+
+/* Which kernel family the shuffle entry points launch (default WASH_MODE_STREAM).
+ * Results are bit-identical across modes. */
+int wash_set_mode(wash_ctx *ctx, int32_t mode);
+
+/* Launch shape override for tuning: threads per block (multiple of 32 in 64..256;
+ * 0 = default) and blocks per SM for the persistent grids (0 = as many as fit;
+ * negative = no persistence, one group per thread). */
+int wash_set_launch(wash_ctx *ctx, int32_t threads, int32_t blocks_per_sm);
+
+/* ---- the shuffling step ----------------------------------------------------------- */
+
+/* Layer-wise probabilities (section "Layer-wise adaptation via WASH"): writes out[l],
+ * l = 0..L-1, as p*(1 - l/(L-1)) (DECREASING, the paper's schedule: first layer p,
+ * last layer never shuffled), p (CONSTANT) or p*l/(L-1) (INCREASING; the two variants
+ * of Table 4).  L == 1 gives out[0] = p.  Host-only helper. */
+int wash_layer_probs(int32_t L, double p, int32_t schedule, double *out);
+
+/* One shuffling step on the parameter stack (Eq. 3; Algorithm 1, "Shuffling step").
+ * Every coordinate i of tensor t is selected with probability p_layer[t] (or p when
+ * p_layer is NULL; probabilities in [0,1]; realised as word < floor(p*2^32) on a
+ * 32-bit Philox word), one draw per coordinate shared by all models; for a selected
+ * coordinate a permutation pi_i, uniform over the N! permutations, is drawn and the N
+ * values are rearranged in place as new[n] = old[pi_i(n)], as raw bits.  Unselected
+ * coordinates are not written.
+ *   step   < 2^56, the training step; seed: any 64-bit value.
+ *   stats  DEVICE-accessible pointer (device memory or mapped pinned host memory) to a
+ *          wash_stats the kernel atomically adds to; may be NULL.
+ * Errors: WASH_ERR_ARG (p out of range / NaN, step too large), WASH_ERR_STATE (stack
+ * not bound), WASH_ERR_UNSUPPORTED, WASH_ERR_CUDA. */
+int wash_shuffle(wash_ctx *ctx, uint64_t step, double p, const double *p_layer,
+                 uint64_t seed, void *stream, wash_stats *stats);
+
+/* The same step applied to the optimizer-state stack (WASH+Opt, section "Training
+ * methods"): with equal (seed, step, p) it selects the same coordinates and applies
+ * the same permutations as wash_shuffle, so the momentum follows its parameter. */
+int wash_shuffle_opt_state(wash_ctx *ctx, uint64_t step, double p, const double *p_layer,
+                           uint64_t seed, void *stream, wash_stats *stats);
+
+/* Both stacks in one launch; equal to wash_shuffle followed by wash_shuffle_opt_state
+ * with the same arguments, with the draws made once. */
+int wash_shuffle_both(wash_ctx *ctx, uint64_t step, double p, const double *p_layer,
+                      uint64_t seed, void *stream, wash_stats *stats);
+
+/* ---- comparison operators --------------------------------------------------------- */
+
+/* PAPA's EMA (Eq. 1), in place on the chosen stack, 0 < alpha < 1:
+ *     m = (((x_0 + x_1) + x_2) + ... + x_{N-1}) / N ;  x_n <- alpha*x_n + (1-alpha)*m
+ * evaluated in binary32 with every operation rounded to nearest even once (no fused
+ * multiply-add), terms added in the order n = 0..N-1.  bf16 stacks are widened,
+ * computed in binary32 and rounded back to nearest even. */
+int papa_ema(wash_ctx *ctx, int32_t stack, float alpha, void *stream);
+
+/* The averaged model (output of Algorithm 1): dev_out[e] = m as defined above for
+ * every coordinate; dev_out is a DEVICE row of padded_P elements of out_dtype
+ * (16-byte aligned), laid out like one model's row; its padding is not written. */
+int population_average(wash_ctx *ctx, int32_t stack, void *dev_out, int32_t out_dtype, void *stream);
+
+/* PAPA-all / DART step (section "Reducing distance to consensus"): every model's
+ * coordinates are overwritten by m. */
+int papa_all(wash_ctx *ctx, int32_t stack, void *stream);
+
+/* Squared distance of every model to the consensus (the quantity of Eq. 2 and Eq. 5,
+ * whose square root averaged over models is plotted in Fig. 2), over tensors
+ * [tensor_lo, tensor_hi):  dev_sq_out[n] += sum_i (x_n^i - mean^i)^2, accumulated in
+ * binary64.  dev_sq_out is a DEVICE array of N doubles the caller has zeroed. */
+int wash_consensus_sq(wash_ctx *ctx, int32_t stack, int32_t tensor_lo, int32_t tensor_hi,
+                      double *dev_sq_out, void *stream);
+
+/* ---- whole step over HOST buffers ------------------------------------------------- */
+
+enum wash_step_ops { WASH_OP_SHUFFLE = 1, WASH_OP_EMA = 2, WASH_OP_AVERAGE = 4 };
+
+/* One pass of the selected operators over stacks that live in HOST memory (pinned
+ * memory makes the copies asynchronous): copies host_params (and host_opt, if not
+ * NULL) into the bound device stacks, runs, in this order, the shuffle (both stacks
+ * when host_opt is given), papa_ema on the parameters and population_average, copies
+ * the stacks back to the same host buffers and the average (row of padded_P elements
+ * of the parameter dtype) to host_avg (may be NULL unless WASH_OP_AVERAGE), and waits
+ * for the stream.  host_stats (may be NULL) receives this call's counters.  The
+ * device stacks must be bound; they serve as staging and hold the results too. */
+int wash_step_host(wash_ctx *ctx, int32_t ops, void *host_params, void *host_opt, void *host_avg,
+                   uint64_t step, double p, const double *p_layer, uint64_t seed, float alpha,
+                   void *stream, wash_stats *host_stats);
+
+/* ---- diagnostics ------------------------------------------------------------------ */
+
+/* Waits for `stream` and returns WASH_ERR_DEVICE_CHECK if a kernel recorded an
+ * inconsistency (an index outside its table) since the last check, else WASH_OK. */
+int wash_check(wash_ctx *ctx, void *stream);
+
+/* Message for the calling thread's most recent error (never NULL). */
+const char *wash_last_error(void);
+
+/* Number of kernels this library has launched in this process. */
+uint64_t wash_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* WASH_H_ */

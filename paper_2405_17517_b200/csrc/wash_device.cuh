@@ -1,0 +1,154 @@
+// Device-side building blocks: Philox4x32-10, element types, segment lookup.
+#pragma once
+#include <cstdint>
+#include <cuda_runtime.h>
+#include "wash_internal.h"
+
+namespace wash {
+
+// ---- Philox4x32-10 (Salmon et al., SC'11) ------------------------------------------
+// Ten rounds of two 32x32->64 multiplies; the key advances by the two Weyl constants
+// after every round.
+struct Philox4 {
+    uint32_t x, y, z, w;
+};
+
+__device__ __forceinline__ Philox4 philox4x32_10(uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3,
+                                                 uint32_t k0, uint32_t k1)
+{
+    constexpr uint32_t kMul0 = 0xD2511F53u, kMul1 = 0xCD9E8D57u;
+    constexpr uint32_t kWeyl0 = 0x9E3779B9u, kWeyl1 = 0xBB67AE85u;
+#pragma unroll
+    for (int r = 0; r < 10; ++r) {
+        const uint32_t hi0 = __umulhi(kMul0, c0), lo0 = kMul0 * c0;
+        const uint32_t hi1 = __umulhi(kMul1, c2), lo1 = kMul1 * c2;
+        c0 = hi1 ^ c1 ^ k0;
+        c2 = hi0 ^ c3 ^ k1;
+        c1 = lo1;
+        c3 = lo0;
+        k0 += kWeyl0;
+        k1 += kWeyl1;
+    }
+    return Philox4{c0, c1, c2, c3};
+}
+
+// ---- element types -------------------------------------------------------------------
+// A "group" is 4 consecutive elements: 16 bytes of fp32, 8 bytes of bf16.  Values are
+// carried as raw bits (uint32 per element, bf16 in the low half).
+struct F32 {
+    using vec = uint4;
+    static constexpr int kBytes = 4;
+    static constexpr int kCode = kDtypeF32;
+    static __device__ __forceinline__ vec load_group(const void *p)
+    {
+        vec v;
+        asm volatile("ld.global.v4.u32 {%0,%1,%2,%3}, [%4];"
+                     : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
+        return v;
+    }
+    static __device__ __forceinline__ void store_group(void *p, vec v) { *reinterpret_cast<vec *>(p) = v; }
+    static __device__ __forceinline__ uint32_t get(const vec &v, int c)
+    {
+        return c == 0 ? v.x : c == 1 ? v.y : c == 2 ? v.z : v.w;
+    }
+    static __device__ __forceinline__ vec pack(uint32_t a, uint32_t b, uint32_t c, uint32_t d) { return make_uint4(a, b, c, d); }
+    static __device__ __forceinline__ uint32_t load_elem(const void *base, long long idx) { return reinterpret_cast<const uint32_t *>(base)[idx]; }
+    static __device__ __forceinline__ void store_elem(void *base, long long idx, uint32_t bits) { reinterpret_cast<uint32_t *>(base)[idx] = bits; }
+    static __device__ __forceinline__ float to_float(uint32_t bits) { return __uint_as_float(bits); }
+    static __device__ __forceinline__ uint32_t from_float(float f) { return __float_as_uint(f); }
+};
+
+struct BF16 {
+    using vec = uint2;
+    static constexpr int kBytes = 2;
+    static constexpr int kCode = kDtypeBF16;
+    static __device__ __forceinline__ vec load_group(const void *p)
+    {
+        vec v;
+        asm volatile("ld.global.v2.u32 {%0,%1}, [%2];" : "=r"(v.x), "=r"(v.y) : "l"(p));
+        return v;
+    }
+    static __device__ __forceinline__ void store_group(void *p, vec v) { *reinterpret_cast<vec *>(p) = v; }
+    static __device__ __forceinline__ uint32_t get(const vec &v, int c)
+    {
+        return c == 0 ? (v.x & 0xFFFFu) : c == 1 ? (v.x >> 16) : c == 2 ? (v.y & 0xFFFFu) : (v.y >> 16);
+    }
+    static __device__ __forceinline__ vec pack(uint32_t a, uint32_t b, uint32_t c, uint32_t d) { return make_uint2(a | (b << 16), c | (d << 16)); }
+    static __device__ __forceinline__ uint32_t load_elem(const void *base, long long idx) { return reinterpret_cast<const uint16_t *>(base)[idx]; }
+    static __device__ __forceinline__ void store_elem(void *base, long long idx, uint32_t bits) { reinterpret_cast<uint16_t *>(base)[idx] = static_cast<uint16_t>(bits); }
+    static __device__ __forceinline__ float to_float(uint32_t bits) { return __uint_as_float(bits << 16); }
+    // round to nearest, ties to even; a NaN stays a quiet NaN
+    static __device__ __forceinline__ uint32_t from_float(float f)
+    {
+        uint32_t u = __float_as_uint(f);
+        if ((u & 0x7FFFFFFFu) > 0x7F800000u) return (u >> 16) | 0x0040u;
+        u += 0x7FFFu + ((u >> 16) & 1u);
+        return u >> 16;
+    }
+};
+
+struct NoStack {   // placeholder for "no second stack"
+    using vec = uint32_t;
+    static constexpr int kBytes = 0;
+    static constexpr int kCode = kDtypeNone;
+};
+
+// ---- addressing ----------------------------------------------------------------------
+// element index of (model n, row element e)
+template <int LAYOUT>
+__device__ __forceinline__ long long elem_index(const PopView &pop, int n, long long e)
+{
+    return LAYOUT == kLayoutNP ? static_cast<long long>(n) * pop.padded_P + e
+                               : e * static_cast<long long>(pop.N) + n;
+}
+
+// Byte address of the j-th vector of group g.  [N][P]: vector j is model j's group.
+// [P][N]: the group's 4N elements are contiguous and vector j is elements 4j..4j+3.
+template <class T, int LAYOUT>
+__device__ __forceinline__ char *group_vec_ptr(void *base, const PopView &pop, uint64_t g, int j)
+{
+    const long long e = LAYOUT == kLayoutNP ? static_cast<long long>(j) * pop.padded_P + 4ll * static_cast<long long>(g)
+                                            : 4ll * static_cast<long long>(g) * pop.N + 4ll * j;
+    return static_cast<char *>(base) + e * T::kBytes;
+}
+
+// raw bits of (model n, coordinate c of the group) out of the group's N vectors
+template <class T, int LAYOUT, int CAP>
+__device__ __forceinline__ uint32_t group_value(const typename T::vec (&v)[CAP], int n_models, int n, int c)
+{
+    if (LAYOUT == kLayoutNP) return T::get(v[n], c);
+    const int f = c * n_models + n;
+    return T::get(v[f >> 2], f & 3);
+}
+
+// ---- which segment does group g belong to ---------------------------------------------
+struct GroupInfo {
+    uint32_t tensor_id;
+    uint32_t cgroup;      // index of the group within its tensor (coordinate / 4)
+    int valid;            // coordinates of this group that exist (0..4)
+    uint64_t thr;
+};
+
+__device__ __forceinline__ GroupInfo find_group(const PopView &pop, uint32_t g, uint32_t *status)
+{
+    uint32_t s = __ldg(pop.tile_first + (g >> kTileShift));
+    const uint32_t last = static_cast<uint32_t>(pop.n_seg) - 1u;
+    while (s < last && g >= __ldg(&pop.seg[s].group_end)) ++s;
+    const uint4 lo = __ldg(reinterpret_cast<const uint4 *>(pop.seg + s));       // begin, end, tensor, cgroup_begin
+    const uint4 hi = __ldg(reinterpret_cast<const uint4 *>(pop.seg + s) + 1);   // numel, -, thr
+    GroupInfo gi;
+    if (g < lo.x || g >= lo.y) {   // table inconsistent with the row: report, touch nothing
+        if (status) atomicOr(status, 1u);
+        gi.tensor_id = 0; gi.cgroup = 0; gi.valid = 0; gi.thr = 0;
+        return gi;
+    }
+    const uint32_t local = g - lo.x;
+    const long long left = static_cast<long long>(hi.x) - 4ll * local;
+    gi.tensor_id = lo.z;
+    gi.cgroup = lo.w + local;
+    gi.valid = left >= 4 ? 4 : (left > 0 ? static_cast<int>(left) : 0);
+    gi.thr = static_cast<uint64_t>(hi.z) | (static_cast<uint64_t>(hi.w) << 32);
+    return gi;
+}
+
+}  // namespace wash

@@ -1,0 +1,59 @@
+// Chooses the kernel instantiation for a population size.
+#include <atomic>
+#include "wash_internal.h"
+#include "wash_nlist.h"
+
+namespace wash {
+
+#define WASH_DECL(n)                                                                                     \
+    cudaError_t launch_shuffle_stream_n##n(const ShuffleArgs &, int, int, const LaunchShape &, cudaStream_t, bool *); \
+    cudaError_t launch_reduce_n##n(const ReduceArgs &, int, int, int, const LaunchShape &, cudaStream_t, bool *);
+WASH_N_LIST(WASH_DECL)
+#undef WASH_DECL
+cudaError_t launch_shuffle_sparse(const ShuffleArgs &, int, int, const LaunchShape &, cudaStream_t, bool *);
+cudaError_t launch_reduce_n0(const ReduceArgs &, int, int, int, const LaunchShape &, cudaStream_t, bool *);
+
+static std::atomic<uint64_t> g_launches{0};
+void count_launch() { g_launches.fetch_add(1, std::memory_order_relaxed); }
+uint64_t launch_count() { return g_launches.load(std::memory_order_relaxed); }
+
+bool has_unrolled_kernels(int N)
+{
+    switch (N) {
+#define WASH_CASE(n) case n:
+        WASH_N_LIST(WASH_CASE)
+#undef WASH_CASE
+        return true;
+    default:
+        return false;
+    }
+}
+
+cudaError_t launch_shuffle(const ShuffleArgs &args, int a_dtype, int b_dtype, int mode,
+                           const LaunchShape &shape, cudaStream_t stream, bool *supported)
+{
+    if (mode == kModeStream) {
+        switch (args.pop.N) {
+#define WASH_CASE(n) case n: return launch_shuffle_stream_n##n(args, a_dtype, b_dtype, shape, stream, supported);
+            WASH_N_LIST(WASH_CASE)
+#undef WASH_CASE
+        default:
+            break;   // no unrolled kernel for this N: the sparse kernel gives the same bits
+        }
+    }
+    return launch_shuffle_sparse(args, a_dtype, b_dtype, shape, stream, supported);
+}
+
+cudaError_t launch_reduce(const ReduceArgs &args, int op, int dtype, int out_dtype,
+                          const LaunchShape &shape, cudaStream_t stream, bool *supported)
+{
+    switch (args.pop.N) {
+#define WASH_CASE(n) case n: return launch_reduce_n##n(args, op, dtype, out_dtype, shape, stream, supported);
+        WASH_N_LIST(WASH_CASE)
+#undef WASH_CASE
+    default:
+        return launch_reduce_n0(args, op, dtype, out_dtype, shape, stream, supported);
+    }
+}
+
+}  // namespace wash

@@ -1,0 +1,77 @@
+// Internal interface between the C ABI (wash_api.cu) and the kernel launchers.
+#pragma once
+#include <cstdint>
+#include <cuda_runtime.h>
+
+namespace wash {
+
+constexpr int kMaxN = 64;          // largest population (WASH_MAX_N)
+constexpr int kTileShift = 8;      // lookup tile = 256 groups = 1024 coordinates
+constexpr int kDtypeF32 = 0, kDtypeBF16 = 1, kDtypeNone = -1;
+constexpr int kLayoutNP = 0, kLayoutPN = 1;
+constexpr int kModeStream = 0, kModeSparse = 1;
+
+// One row of a stack is cut into groups of 4 consecutive elements; a group never
+// straddles two tensors because tensors start on multiples of 8 elements.
+struct SegEntry {
+    uint32_t group_begin;   // first group of the segment within a row
+    uint32_t group_end;     // one past its last group (padding groups included)
+    uint32_t tensor_id;     // RNG tensor index
+    uint32_t cgroup_begin;  // (first coordinate's index within its tensor) / 4
+    uint32_t numel;         // coordinates in the segment
+    uint32_t reserved;
+    uint64_t thr;           // floor(p * 2^32): coordinate selected iff word < thr
+};
+static_assert(sizeof(SegEntry) == 32, "SegEntry must stay 32 bytes");
+
+struct PopView {
+    int N;
+    int layout;
+    long long padded_P;           // elements per model row
+    uint32_t n_groups;            // padded_P / 4
+    int n_seg;
+    const SegEntry *seg;          // device, n_seg entries
+    const uint32_t *tile_first;   // device, segment of the first group of every tile
+};
+
+struct ShuffleArgs {
+    PopView pop;
+    void *a;                      // first stack (device)
+    void *b;                      // second stack or nullptr
+    uint32_t key0, key1;          // seed
+    uint32_t step_lo, step_hi8;   // step & 0xFFFFFFFF, (step >> 32) << 8
+    unsigned long long *stats;    // device-accessible {selected, moved} or nullptr
+    uint32_t *status;             // device status word
+};
+
+struct ReduceArgs {
+    PopView pop;
+    void *stack;                  // device stack (read; written by EMA / papa_all)
+    void *out;                    // average row (device) or nullptr
+    float alpha, one_minus_alpha;
+    uint32_t group_lo, group_hi;  // range of groups to process
+    double *sq_out;               // consensus: N doubles (device) or nullptr
+    uint32_t *status;
+};
+
+enum ReduceOp { kOpEma = 0, kOpAverage = 1, kOpPapaAll = 2, kOpConsensus = 3 };
+
+struct LaunchShape {
+    int threads;         // 0 = default
+    int blocks_per_sm;   // 0 = as many as fit, < 0 = one group per thread
+    int sm_count;
+};
+
+// Each returns cudaSuccess or the launch error; *supported = false (and no launch) if
+// this build has no kernel for the combination.
+cudaError_t launch_shuffle(const ShuffleArgs &args, int a_dtype, int b_dtype, int mode,
+                           const LaunchShape &shape, cudaStream_t stream, bool *supported);
+cudaError_t launch_reduce(const ReduceArgs &args, int op, int dtype, int out_dtype,
+                          const LaunchShape &shape, cudaStream_t stream, bool *supported);
+
+// true if a streaming shuffle kernel was compiled for this population size
+bool has_unrolled_kernels(int N);
+
+void count_launch();
+
+}  // namespace wash
