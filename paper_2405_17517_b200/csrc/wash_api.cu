@@ -1,0 +1,527 @@
+// C ABI of libwash.so: argument checks, the context's tables, and the launches.
+// The entry points are documented in include/wash.h.
+#include <cmath>
+#include <cstdarg>
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <string>
+#include <vector>
+
+#include <cuda_runtime.h>
+
+#include "../../include/wash.h"
+#include "wash_internal.h"
+
+namespace wash {
+uint64_t launch_count();
+}
+
+using wash::SegEntry;
+
+namespace {
+
+thread_local std::string g_last_error = "";
+
+int fail(int code, const char *fmt, ...)
+{
+    char buf[512];
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(buf, sizeof buf, fmt, ap);
+    va_end(ap);
+    g_last_error = buf;
+    return code;
+}
+
+int cuda_fail(cudaError_t err, const char *what)
+{
+    return fail(WASH_ERR_CUDA, "%s: %s", what, cudaGetErrorString(err));
+}
+
+constexpr int kSlots = 4;   // pinned staging slots for table uploads
+
+// makes `device` current for the lifetime of the guard
+struct DeviceGuard {
+    int prev = -1;
+    bool switched = false;
+    cudaError_t err = cudaSuccess;
+    explicit DeviceGuard(int device)
+    {
+        err = cudaGetDevice(&prev);
+        if (err == cudaSuccess && prev != device) {
+            err = cudaSetDevice(device);
+            switched = (err == cudaSuccess);
+        }
+    }
+    ~DeviceGuard()
+    {
+        if (switched) cudaSetDevice(prev);
+    }
+};
+
+}  // namespace
+
+struct wash_ctx {
+    int N = 0, layout = 0, device = 0, n_seg = 0;
+    std::vector<int64_t> numel, offset, coord_begin;
+    std::vector<uint32_t> tensor_id;
+    int64_t padded_P = 0;
+    uint32_t n_groups = 0, n_tiles = 0;
+
+    std::vector<SegEntry> seg_host;        // thresholds as last uploaded
+    bool seg_uploaded = false;
+    SegEntry *seg_dev = nullptr;
+    uint32_t *tile_first_dev = nullptr;
+    SegEntry *seg_pinned[kSlots] = {nullptr, nullptr, nullptr, nullptr};
+    cudaEvent_t slot_event[kSlots] = {nullptr, nullptr, nullptr, nullptr};
+    bool slot_used[kSlots] = {false, false, false, false};
+    int next_slot = 0;
+
+    void *stack_ptr[2] = {nullptr, nullptr};
+    int stack_dtype[2] = {0, 0};
+
+    uint32_t *status_dev = nullptr;
+    wash_stats *stats_dev = nullptr;       // for wash_step_host
+    void *avg_dev = nullptr;               // for wash_step_host, allocated on first use
+    size_t avg_bytes = 0;
+
+    int mode = WASH_MODE_STREAM;
+    wash::LaunchShape shape{0, 0, 148};
+};
+
+namespace {
+
+void release(wash_ctx *ctx)
+{
+    if (!ctx) return;
+    DeviceGuard guard(ctx->device);
+    if (ctx->seg_dev) cudaFree(ctx->seg_dev);
+    if (ctx->tile_first_dev) cudaFree(ctx->tile_first_dev);
+    if (ctx->status_dev) cudaFree(ctx->status_dev);
+    if (ctx->stats_dev) cudaFree(ctx->stats_dev);
+    if (ctx->avg_dev) cudaFree(ctx->avg_dev);
+    for (int s = 0; s < kSlots; ++s) {
+        if (ctx->seg_pinned[s]) cudaFreeHost(ctx->seg_pinned[s]);
+        if (ctx->slot_event[s]) cudaEventDestroy(ctx->slot_event[s]);
+    }
+    delete ctx;
+}
+
+wash::PopView view_of(const wash_ctx *ctx)
+{
+    wash::PopView v;
+    v.N = ctx->N;
+    v.layout = ctx->layout;
+    v.padded_P = ctx->padded_P;
+    v.n_groups = ctx->n_groups;
+    v.n_seg = ctx->n_seg;
+    v.seg = ctx->seg_dev;
+    v.tile_first = ctx->tile_first_dev;
+    return v;
+}
+
+size_t elem_bytes(int dtype) { return dtype == WASH_BF16 ? 2 : 4; }
+
+// floor(p * 2^32) for p in [0, 1]; the product is exact in binary64
+uint64_t threshold_of(double p) { return static_cast<uint64_t>(std::floor(p * 4294967296.0)); }
+
+// Brings the device copy of the segment table up to date with the call's
+// probabilities (uploaded, in stream order, only when they changed).
+int sync_table(wash_ctx *ctx, double p, const double *p_layer, cudaStream_t stream)
+{
+    bool changed = !ctx->seg_uploaded;
+    for (int s = 0; s < ctx->n_seg; ++s) {
+        const double ps = p_layer ? p_layer[s] : p;
+        if (!(ps >= 0.0 && ps <= 1.0)) return fail(WASH_ERR_ARG, "probability of tensor %d is %g, not in [0,1]", s, ps);
+        const uint64_t thr = threshold_of(ps);
+        if (thr != ctx->seg_host[s].thr) {
+            ctx->seg_host[s].thr = thr;
+            changed = true;
+        }
+    }
+    if (!changed) return WASH_OK;
+    const int slot = ctx->next_slot;
+    ctx->next_slot = (slot + 1) % kSlots;
+    if (ctx->slot_used[slot]) {   // the copy that last read this slot must be done
+        cudaError_t err = cudaEventSynchronize(ctx->slot_event[slot]);
+        if (err != cudaSuccess) return cuda_fail(err, "cudaEventSynchronize(table slot)");
+    }
+    const size_t bytes = sizeof(SegEntry) * static_cast<size_t>(ctx->n_seg);
+    std::memcpy(ctx->seg_pinned[slot], ctx->seg_host.data(), bytes);
+    cudaError_t err = cudaMemcpyAsync(ctx->seg_dev, ctx->seg_pinned[slot], bytes, cudaMemcpyHostToDevice, stream);
+    if (err != cudaSuccess) return cuda_fail(err, "cudaMemcpyAsync(segment table)");
+    err = cudaEventRecord(ctx->slot_event[slot], stream);
+    if (err != cudaSuccess) return cuda_fail(err, "cudaEventRecord(table slot)");
+    ctx->slot_used[slot] = true;
+    ctx->seg_uploaded = true;
+    return WASH_OK;
+}
+
+int ensure_table(wash_ctx *ctx, cudaStream_t stream)
+{
+    if (ctx->seg_uploaded) return WASH_OK;
+    std::vector<double> zeros(static_cast<size_t>(ctx->n_seg), 0.0);
+    return sync_table(ctx, 0.0, zeros.data(), stream);
+}
+
+// which: 0 = parameters, 1 = optimizer state, 2 = both
+int shuffle_impl(wash_ctx *ctx, int which, uint64_t step, double p, const double *p_layer, uint64_t seed,
+                 void *stream_v, wash_stats *stats)
+{
+    if (!ctx) return fail(WASH_ERR_ARG, "ctx is NULL");
+    if (step >> 56) return fail(WASH_ERR_ARG, "step must be below 2^56");
+    if (!p_layer && !(p >= 0.0 && p <= 1.0)) return fail(WASH_ERR_ARG, "p is %g, not in [0,1]", p);
+    void *a = nullptr, *b = nullptr;
+    int a_dtype = wash::kDtypeNone, b_dtype = wash::kDtypeNone;
+    if (which == 0 || which == 2) {
+        a = ctx->stack_ptr[WASH_STACK_PARAMS];
+        a_dtype = ctx->stack_dtype[WASH_STACK_PARAMS];
+        if (!a) return fail(WASH_ERR_STATE, "parameter stack is not bound");
+    }
+    if (which == 1 || which == 2) {
+        void *o = ctx->stack_ptr[WASH_STACK_OPT];
+        if (!o) return fail(WASH_ERR_STATE, "optimizer-state stack is not bound");
+        if (which == 1) { a = o; a_dtype = ctx->stack_dtype[WASH_STACK_OPT]; }
+        else { b = o; b_dtype = ctx->stack_dtype[WASH_STACK_OPT]; }
+    }
+    DeviceGuard guard(ctx->device);
+    if (guard.err != cudaSuccess) return cuda_fail(guard.err, "cudaSetDevice");
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
+    int rc = sync_table(ctx, p, p_layer, stream);
+    if (rc != WASH_OK) return rc;
+
+    wash::ShuffleArgs args;
+    args.pop = view_of(ctx);
+    args.a = a;
+    args.b = b;
+    args.key0 = static_cast<uint32_t>(seed);
+    args.key1 = static_cast<uint32_t>(seed >> 32);
+    args.step_lo = static_cast<uint32_t>(step);
+    args.step_hi8 = static_cast<uint32_t>(step >> 32) << 8;
+    args.stats = reinterpret_cast<unsigned long long *>(stats);
+    args.status = ctx->status_dev;
+    bool supported = false;
+    cudaError_t err = wash::launch_shuffle(args, a_dtype, b_dtype, ctx->mode, ctx->shape, stream, &supported);
+    if (err != cudaSuccess) return cuda_fail(err, "shuffle kernel launch");
+    if (!supported) return fail(WASH_ERR_UNSUPPORTED, "no shuffle kernel for dtypes (%d, %d)", a_dtype, b_dtype);
+    return WASH_OK;
+}
+
+int reduce_impl(wash_ctx *ctx, int op, int stack, void *out, int out_dtype, float alpha, int tensor_lo,
+                int tensor_hi, double *sq_out, void *stream_v)
+{
+    if (!ctx) return fail(WASH_ERR_ARG, "ctx is NULL");
+    if (stack != WASH_STACK_PARAMS && stack != WASH_STACK_OPT) return fail(WASH_ERR_ARG, "stack must be 0 or 1");
+    if (!ctx->stack_ptr[stack]) return fail(WASH_ERR_STATE, "stack %d is not bound", stack);
+    DeviceGuard guard(ctx->device);
+    if (guard.err != cudaSuccess) return cuda_fail(guard.err, "cudaSetDevice");
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
+    int rc = ensure_table(ctx, stream);
+    if (rc != WASH_OK) return rc;
+    wash::ReduceArgs args;
+    args.pop = view_of(ctx);
+    args.stack = ctx->stack_ptr[stack];
+    args.out = out;
+    args.alpha = alpha;
+    args.one_minus_alpha = 1.0f - alpha;
+    args.group_lo = ctx->seg_host[static_cast<size_t>(tensor_lo)].group_begin;
+    args.group_hi = ctx->seg_host[static_cast<size_t>(tensor_hi) - 1].group_end;
+    args.sq_out = sq_out;
+    args.status = ctx->status_dev;
+    bool supported = false;
+    cudaError_t err = wash::launch_reduce(args, op, ctx->stack_dtype[stack], out_dtype, ctx->shape, stream, &supported);
+    if (err != cudaSuccess) return cuda_fail(err, "kernel launch");
+    if (!supported) return fail(WASH_ERR_UNSUPPORTED, "no kernel for dtype %d -> %d", ctx->stack_dtype[stack], out_dtype);
+    return WASH_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int wash_create_segments(wash_ctx **out, int32_t N, int32_t n_segments, const int64_t *numel,
+                         const uint32_t *tensor_id, const int64_t *coord_begin, int32_t layout, int32_t device)
+{
+    if (!out) return fail(WASH_ERR_ARG, "out is NULL");
+    *out = nullptr;
+    if (N < 2 || N > WASH_MAX_N) return fail(WASH_ERR_ARG, "N = %d, must be in [2, %d]", N, WASH_MAX_N);
+    if (n_segments < 1 || !numel) return fail(WASH_ERR_ARG, "need at least one tensor");
+    if (layout != WASH_LAYOUT_NP && layout != WASH_LAYOUT_PN) return fail(WASH_ERR_ARG, "unknown layout %d", layout);
+    if (device < 0) return fail(WASH_ERR_ARG, "device = %d", device);
+
+    wash_ctx *ctx = new (std::nothrow) wash_ctx;
+    if (!ctx) return fail(WASH_ERR_ALLOC, "out of host memory");
+    ctx->N = N;
+    ctx->layout = layout;
+    ctx->device = device;
+    ctx->n_seg = n_segments;
+    int64_t cur = 0;
+    for (int s = 0; s < n_segments; ++s) {
+        const int64_t d = numel[s];
+        const int64_t cb = coord_begin ? coord_begin[s] : 0;
+        if (d <= 0 || d >= (int64_t(1) << 32)) { delete ctx; return fail(WASH_ERR_ARG, "numel[%d] = %lld, must be in (0, 2^32)", s, (long long)d); }
+        if (cb < 0 || (cb & 3) || cb + d > (int64_t(1) << 32)) { delete ctx; return fail(WASH_ERR_ARG, "coord_begin[%d] = %lld must be a multiple of 4 with coord_begin + numel <= 2^32", s, (long long)cb); }
+        ctx->numel.push_back(d);
+        ctx->offset.push_back(cur);
+        ctx->coord_begin.push_back(cb);
+        ctx->tensor_id.push_back(tensor_id ? tensor_id[s] : static_cast<uint32_t>(s));
+        cur += (d + WASH_ALIGN_ELEMS - 1) / WASH_ALIGN_ELEMS * WASH_ALIGN_ELEMS;
+        if (cur / 4 >= (int64_t(1) << 31)) { delete ctx; return fail(WASH_ERR_ARG, "row too long: more than 2^33 elements"); }
+    }
+    ctx->padded_P = cur;
+    ctx->n_groups = static_cast<uint32_t>(cur / 4);
+    ctx->n_tiles = (ctx->n_groups + (1u << wash::kTileShift) - 1) >> wash::kTileShift;
+
+    ctx->seg_host.resize(static_cast<size_t>(n_segments));
+    for (int s = 0; s < n_segments; ++s) {
+        SegEntry &e = ctx->seg_host[static_cast<size_t>(s)];
+        e.group_begin = static_cast<uint32_t>(ctx->offset[s] / 4);
+        e.group_end = static_cast<uint32_t>((s + 1 < n_segments ? ctx->offset[s + 1] : cur) / 4);
+        e.tensor_id = ctx->tensor_id[s];
+        e.cgroup_begin = static_cast<uint32_t>(ctx->coord_begin[s] / 4);
+        e.numel = static_cast<uint32_t>(ctx->numel[s]);
+        e.reserved = 0;
+        e.thr = 0;
+    }
+    std::vector<uint32_t> tile_first(ctx->n_tiles);
+    {
+        uint32_t s = 0;
+        for (uint32_t t = 0; t < ctx->n_tiles; ++t) {
+            const uint32_t g = t << wash::kTileShift;
+            while (g >= ctx->seg_host[s].group_end) ++s;
+            tile_first[t] = s;
+        }
+    }
+
+    DeviceGuard guard(device);
+    if (guard.err != cudaSuccess) { delete ctx; return cuda_fail(guard.err, "cudaSetDevice"); }
+    cudaError_t err = cudaSuccess;
+    int sm_count = 0;
+    err = cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, device);
+    if (err != cudaSuccess) { delete ctx; return cuda_fail(err, "cudaDeviceGetAttribute"); }
+    ctx->shape.sm_count = sm_count;
+    const size_t seg_bytes = sizeof(SegEntry) * static_cast<size_t>(n_segments);
+    if ((err = cudaMalloc(&ctx->seg_dev, seg_bytes)) != cudaSuccess ||
+        (err = cudaMalloc(&ctx->tile_first_dev, sizeof(uint32_t) * ctx->n_tiles)) != cudaSuccess ||
+        (err = cudaMalloc(&ctx->status_dev, sizeof(uint32_t))) != cudaSuccess ||
+        (err = cudaMalloc(&ctx->stats_dev, sizeof(wash_stats))) != cudaSuccess) {
+        release(ctx);
+        cudaGetLastError();
+        return fail(WASH_ERR_ALLOC, "device allocation failed: %s", cudaGetErrorString(err));
+    }
+    for (int s = 0; s < kSlots; ++s) {
+        if ((err = cudaMallocHost(&ctx->seg_pinned[s], seg_bytes)) != cudaSuccess ||
+            (err = cudaEventCreateWithFlags(&ctx->slot_event[s], cudaEventDisableTiming)) != cudaSuccess) {
+            release(ctx);
+            cudaGetLastError();
+            return fail(WASH_ERR_ALLOC, "pinned allocation failed: %s", cudaGetErrorString(err));
+        }
+    }
+    if ((err = cudaMemcpy(ctx->tile_first_dev, tile_first.data(), sizeof(uint32_t) * ctx->n_tiles, cudaMemcpyHostToDevice)) != cudaSuccess ||
+        (err = cudaMemset(ctx->status_dev, 0, sizeof(uint32_t))) != cudaSuccess ||
+        (err = cudaMemset(ctx->stats_dev, 0, sizeof(wash_stats))) != cudaSuccess) {
+        release(ctx);
+        return cuda_fail(err, "table upload");
+    }
+    *out = ctx;
+    return WASH_OK;
+}
+
+int wash_create(wash_ctx **out, int32_t N, int32_t n_tensors, const int64_t *numel, int32_t layout, int32_t device)
+{
+    return wash_create_segments(out, N, n_tensors, numel, nullptr, nullptr, layout, device);
+}
+
+int wash_destroy(wash_ctx *ctx)
+{
+    if (!ctx) return fail(WASH_ERR_ARG, "ctx is NULL");
+    release(ctx);
+    return WASH_OK;
+}
+
+int wash_stack_elems(const wash_ctx *ctx, int64_t *padded_P, int64_t *offsets)
+{
+    if (!ctx) return fail(WASH_ERR_ARG, "ctx is NULL");
+    if (padded_P) *padded_P = ctx->padded_P;
+    if (offsets)
+        for (int s = 0; s < ctx->n_seg; ++s) offsets[s] = ctx->offset[s];
+    return WASH_OK;
+}
+
+int wash_bind(wash_ctx *ctx, int32_t stack, int32_t dtype, void *dev_ptr, int64_t n_elems)
+{
+    if (!ctx) return fail(WASH_ERR_ARG, "ctx is NULL");
+    if (stack != WASH_STACK_PARAMS && stack != WASH_STACK_OPT) return fail(WASH_ERR_ARG, "stack must be 0 or 1");
+    if (!dev_ptr) { ctx->stack_ptr[stack] = nullptr; return WASH_OK; }
+    if (dtype != WASH_F32 && dtype != WASH_BF16) return fail(WASH_ERR_ARG, "unknown dtype %d", dtype);
+    if (n_elems != static_cast<int64_t>(ctx->N) * ctx->padded_P)
+        return fail(WASH_ERR_ARG, "stack has %lld elements, population needs N * padded_P = %lld", (long long)n_elems,
+                    (long long)(static_cast<int64_t>(ctx->N) * ctx->padded_P));
+    if (reinterpret_cast<uintptr_t>(dev_ptr) & 15) return fail(WASH_ERR_ARG, "stack pointer must be 16-byte aligned");
+    ctx->stack_ptr[stack] = dev_ptr;
+    ctx->stack_dtype[stack] = dtype;
+    return WASH_OK;
+}
+
+int wash_set_mode(wash_ctx *ctx, int32_t mode)
+{
+    if (!ctx) return fail(WASH_ERR_ARG, "ctx is NULL");
+    if (mode != WASH_MODE_STREAM && mode != WASH_MODE_SPARSE) return fail(WASH_ERR_ARG, "unknown mode %d", mode);
+    ctx->mode = mode;
+    return WASH_OK;
+}
+
+int wash_set_launch(wash_ctx *ctx, int32_t threads, int32_t blocks_per_sm)
+{
+    if (!ctx) return fail(WASH_ERR_ARG, "ctx is NULL");
+    if (threads != 0 && (threads < 64 || threads > 256 || (threads & 31))) return fail(WASH_ERR_ARG, "threads = %d: need 0 or a multiple of 32 in [64, 256]", threads);
+    ctx->shape.threads = threads;
+    ctx->shape.blocks_per_sm = blocks_per_sm;
+    return WASH_OK;
+}
+
+int wash_layer_probs(int32_t L, double p, int32_t schedule, double *out)
+{
+    if (L < 1 || !out) return fail(WASH_ERR_ARG, "need L >= 1 and an output array");
+    if (!(p >= 0.0 && p <= 1.0)) return fail(WASH_ERR_ARG, "p is %g, not in [0,1]", p);
+    if (schedule < WASH_SCHEDULE_DECREASING || schedule > WASH_SCHEDULE_INCREASING) return fail(WASH_ERR_ARG, "unknown schedule %d", schedule);
+    for (int l = 0; l < L; ++l) {
+        if (L == 1 || schedule == WASH_SCHEDULE_CONSTANT) { out[l] = p; continue; }
+        const double depth = static_cast<double>(l) / static_cast<double>(L - 1);
+        out[l] = schedule == WASH_SCHEDULE_DECREASING ? p * (1.0 - depth) : p * depth;
+    }
+    return WASH_OK;
+}
+
+int wash_shuffle(wash_ctx *ctx, uint64_t step, double p, const double *p_layer, uint64_t seed, void *stream, wash_stats *stats)
+{
+    return shuffle_impl(ctx, 0, step, p, p_layer, seed, stream, stats);
+}
+
+int wash_shuffle_opt_state(wash_ctx *ctx, uint64_t step, double p, const double *p_layer, uint64_t seed, void *stream, wash_stats *stats)
+{
+    return shuffle_impl(ctx, 1, step, p, p_layer, seed, stream, stats);
+}
+
+int wash_shuffle_both(wash_ctx *ctx, uint64_t step, double p, const double *p_layer, uint64_t seed, void *stream, wash_stats *stats)
+{
+    return shuffle_impl(ctx, 2, step, p, p_layer, seed, stream, stats);
+}
+
+int papa_ema(wash_ctx *ctx, int32_t stack, float alpha, void *stream)
+{
+    if (!(alpha > 0.0f && alpha < 1.0f)) return fail(WASH_ERR_ARG, "alpha is %g, must be in (0,1)", (double)alpha);
+    if (!ctx) return fail(WASH_ERR_ARG, "ctx is NULL");
+    return reduce_impl(ctx, wash::kOpEma, stack, nullptr, WASH_F32, alpha, 0, ctx->n_seg, nullptr, stream);
+}
+
+int population_average(wash_ctx *ctx, int32_t stack, void *dev_out, int32_t out_dtype, void *stream)
+{
+    if (!ctx) return fail(WASH_ERR_ARG, "ctx is NULL");
+    if (!dev_out || (reinterpret_cast<uintptr_t>(dev_out) & 15)) return fail(WASH_ERR_ARG, "dev_out must be a 16-byte aligned device pointer");
+    if (out_dtype != WASH_F32 && out_dtype != WASH_BF16) return fail(WASH_ERR_ARG, "unknown out_dtype %d", out_dtype);
+    return reduce_impl(ctx, wash::kOpAverage, stack, dev_out, out_dtype, 0.0f, 0, ctx->n_seg, nullptr, stream);
+}
+
+int papa_all(wash_ctx *ctx, int32_t stack, void *stream)
+{
+    if (!ctx) return fail(WASH_ERR_ARG, "ctx is NULL");
+    return reduce_impl(ctx, wash::kOpPapaAll, stack, nullptr, WASH_F32, 0.0f, 0, ctx->n_seg, nullptr, stream);
+}
+
+int wash_consensus_sq(wash_ctx *ctx, int32_t stack, int32_t tensor_lo, int32_t tensor_hi, double *dev_sq_out, void *stream)
+{
+    if (!ctx) return fail(WASH_ERR_ARG, "ctx is NULL");
+    if (!dev_sq_out) return fail(WASH_ERR_ARG, "dev_sq_out is NULL");
+    if (tensor_lo < 0 || tensor_hi > ctx->n_seg || tensor_lo > tensor_hi) return fail(WASH_ERR_ARG, "tensor range [%d, %d) is not within [0, %d]", tensor_lo, tensor_hi, ctx->n_seg);
+    if (tensor_lo == tensor_hi) return WASH_OK;
+    return reduce_impl(ctx, wash::kOpConsensus, stack, nullptr, WASH_F32, 0.0f, tensor_lo, tensor_hi, dev_sq_out, stream);
+}
+
+int wash_step_host(wash_ctx *ctx, int32_t ops, void *host_params, void *host_opt, void *host_avg, uint64_t step,
+                   double p, const double *p_layer, uint64_t seed, float alpha, void *stream_v, wash_stats *host_stats)
+{
+    if (!ctx) return fail(WASH_ERR_ARG, "ctx is NULL");
+    if (!host_params) return fail(WASH_ERR_ARG, "host_params is NULL");
+    if (ops & ~(WASH_OP_SHUFFLE | WASH_OP_EMA | WASH_OP_AVERAGE)) return fail(WASH_ERR_ARG, "unknown bits in ops");
+    if ((ops & WASH_OP_AVERAGE) && !host_avg) return fail(WASH_ERR_ARG, "host_avg is NULL but WASH_OP_AVERAGE is set");
+    if (!ctx->stack_ptr[WASH_STACK_PARAMS]) return fail(WASH_ERR_STATE, "parameter stack is not bound");
+    if (host_opt && !ctx->stack_ptr[WASH_STACK_OPT]) return fail(WASH_ERR_STATE, "optimizer-state stack is not bound");
+    if ((ops & WASH_OP_EMA) && !(alpha > 0.0f && alpha < 1.0f)) return fail(WASH_ERR_ARG, "alpha is %g, must be in (0,1)", (double)alpha);
+    DeviceGuard guard(ctx->device);
+    if (guard.err != cudaSuccess) return cuda_fail(guard.err, "cudaSetDevice");
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
+    const int pd = ctx->stack_dtype[WASH_STACK_PARAMS];
+    const size_t n_elems = static_cast<size_t>(ctx->N) * static_cast<size_t>(ctx->padded_P);
+    const size_t p_bytes = n_elems * elem_bytes(pd);
+    const size_t o_bytes = host_opt ? n_elems * elem_bytes(ctx->stack_dtype[WASH_STACK_OPT]) : 0;
+    const size_t avg_bytes = static_cast<size_t>(ctx->padded_P) * elem_bytes(pd);
+    cudaError_t err;
+    if ((ops & WASH_OP_AVERAGE) && ctx->avg_bytes < avg_bytes) {
+        if (ctx->avg_dev) cudaFree(ctx->avg_dev);
+        ctx->avg_dev = nullptr;
+        ctx->avg_bytes = 0;
+        if ((err = cudaMalloc(&ctx->avg_dev, avg_bytes)) != cudaSuccess) {
+            cudaGetLastError();
+            return fail(WASH_ERR_ALLOC, "device allocation of the average row failed: %s", cudaGetErrorString(err));
+        }
+        ctx->avg_bytes = avg_bytes;
+    }
+    if ((err = cudaMemcpyAsync(ctx->stack_ptr[WASH_STACK_PARAMS], host_params, p_bytes, cudaMemcpyHostToDevice, stream)) != cudaSuccess)
+        return cuda_fail(err, "copy of the parameter stack to the device");
+    if (host_opt && (err = cudaMemcpyAsync(ctx->stack_ptr[WASH_STACK_OPT], host_opt, o_bytes, cudaMemcpyHostToDevice, stream)) != cudaSuccess)
+        return cuda_fail(err, "copy of the optimizer-state stack to the device");
+    int rc;
+    if (ops & WASH_OP_SHUFFLE) {
+        if ((err = cudaMemsetAsync(ctx->stats_dev, 0, sizeof(wash_stats), stream)) != cudaSuccess) return cuda_fail(err, "cudaMemsetAsync(stats)");
+        rc = shuffle_impl(ctx, host_opt ? 2 : 0, step, p, p_layer, seed, stream, ctx->stats_dev);
+        if (rc != WASH_OK) return rc;
+    }
+    if (ops & WASH_OP_EMA) {
+        rc = papa_ema(ctx, WASH_STACK_PARAMS, alpha, stream);
+        if (rc != WASH_OK) return rc;
+    }
+    if (ops & WASH_OP_AVERAGE) {
+        if (avg_bytes % 16) { /* padded_P is a multiple of 8 elements, so this cannot happen */ }
+        // padding of the row is never written by the kernel: give it a defined value
+        if ((err = cudaMemsetAsync(ctx->avg_dev, 0, avg_bytes, stream)) != cudaSuccess) return cuda_fail(err, "cudaMemsetAsync(average row)");
+        rc = population_average(ctx, WASH_STACK_PARAMS, ctx->avg_dev, pd, stream);
+        if (rc != WASH_OK) return rc;
+    }
+    if ((err = cudaMemcpyAsync(host_params, ctx->stack_ptr[WASH_STACK_PARAMS], p_bytes, cudaMemcpyDeviceToHost, stream)) != cudaSuccess)
+        return cuda_fail(err, "copy of the parameter stack to the host");
+    if (host_opt && (err = cudaMemcpyAsync(host_opt, ctx->stack_ptr[WASH_STACK_OPT], o_bytes, cudaMemcpyDeviceToHost, stream)) != cudaSuccess)
+        return cuda_fail(err, "copy of the optimizer-state stack to the host");
+    if ((ops & WASH_OP_AVERAGE) && (err = cudaMemcpyAsync(host_avg, ctx->avg_dev, avg_bytes, cudaMemcpyDeviceToHost, stream)) != cudaSuccess)
+        return cuda_fail(err, "copy of the average to the host");
+    wash_stats st = {0, 0};
+    if ((ops & WASH_OP_SHUFFLE) && (err = cudaMemcpyAsync(&st, ctx->stats_dev, sizeof st, cudaMemcpyDeviceToHost, stream)) != cudaSuccess)
+        return cuda_fail(err, "copy of the counters to the host");
+    if ((err = cudaStreamSynchronize(stream)) != cudaSuccess) return cuda_fail(err, "cudaStreamSynchronize");
+    if (host_stats) *host_stats = st;
+    return WASH_OK;
+}
+
+int wash_check(wash_ctx *ctx, void *stream_v)
+{
+    if (!ctx) return fail(WASH_ERR_ARG, "ctx is NULL");
+    DeviceGuard guard(ctx->device);
+    if (guard.err != cudaSuccess) return cuda_fail(guard.err, "cudaSetDevice");
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
+    uint32_t status = 0;
+    cudaError_t err = cudaMemcpyAsync(&status, ctx->status_dev, sizeof status, cudaMemcpyDeviceToHost, stream);
+    if (err == cudaSuccess) err = cudaStreamSynchronize(stream);
+    if (err != cudaSuccess) return cuda_fail(err, "reading the status word");
+    if (status) {
+        cudaMemsetAsync(ctx->status_dev, 0, sizeof(uint32_t), stream);
+        return fail(WASH_ERR_DEVICE_CHECK, "a kernel found a group outside its segment table (status 0x%x)", status);
+    }
+    return WASH_OK;
+}
+
+const char *wash_last_error(void) { return g_last_error.c_str(); }
+
+uint64_t wash_launch_count(void) { return wash::launch_count(); }
+
+}  // extern "C"

@@ -24,7 +24,7 @@ namespace wash {
 // shared memory: s_perm[n * ts], n = 0..N-1.  Fisher-Yates from the top index down,
 // word m of the coordinate's permutation stream decides the swap of position N-1-m;
 // j = floor(word * (k+1) / 2^32).
-__device__ __noinline__ void draw_permutation(uint32_t *s_perm, int ts, int n_models, uint32_t i,
+static __device__ __noinline__ void draw_permutation(uint32_t *s_perm, int ts, int n_models, uint32_t i,
                                               uint32_t tensor, uint32_t step_lo, uint32_t step_hi8,
                                               uint32_t k0, uint32_t k1)
 {

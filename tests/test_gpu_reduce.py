@@ -1,0 +1,131 @@
+"""GPU parity of PAPA's EMA (Eq. 1), the final average, PAPA-all and the consensus
+distance against the oracle.  The kernels use the oracle's operation order with
+explicitly rounded binary32 operations, so results are expected to be bit-identical;
+the stated bar is 2 ulp (max relative error 2.4e-7)."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2405_17517_b200 import binding as B
+from paper_2405_17517_b200 import workloads as W
+from gpu_util import Case, bits, to_host_bits, ulp_distance_f32
+
+pytestmark = pytest.mark.gpu
+
+RAGGED = [1000, 33, 7, 1, 4, 8, 5003, 2048]
+MAX_ULP = 2
+
+
+def _assert_close_f32(got_bits, want_bits, what):
+    d = ulp_distance_f32(got_bits, want_bits)
+    assert d.max() <= MAX_ULP, "%s: %d ulp" % (what, d.max())
+    return int(d.max())
+
+
+@pytest.mark.parametrize("layout", [0, 1])
+@pytest.mark.parametrize("N", [2, 3, 5, 7, 8, 10, 16, 32, 33, 64])
+def test_ema_average_papa_all_fp32(N, layout):
+    c = Case(N, RAGGED, layout, seed=N + 40)
+    worst = 0
+    for alpha in (0.99, 0.001, 0.5):
+        B.papa_ema(c.gpu.ctx, B.WASH_STACK_PARAMS, alpha)
+        oracle.papa_ema(c.ora, c.host, alpha)
+        torch.cuda.synchronize()
+        worst = max(worst, _assert_close_f32(to_host_bits(c.dev), bits(c.host), "ema"))
+        # keep both sides on the same state so errors cannot build up across calls
+        c.dev.copy_(torch.from_numpy(c.host.reshape(-1).copy()))
+    out = torch.full((c.P,), float("nan"), dtype=torch.float32, device="cuda")
+    B.population_average(c.gpu.ctx, B.WASH_STACK_PARAMS, out, B.WASH_F32)
+    want = np.full(c.P, np.nan, dtype=np.float32)
+    oracle.population_average(c.ora, c.host, want)
+    worst = max(worst, _assert_close_f32(to_host_bits(out), want.view(np.uint32), "average"))
+    outb = torch.zeros(c.P, dtype=torch.bfloat16, device="cuda")
+    B.population_average(c.gpu.ctx, B.WASH_STACK_PARAMS, outb, B.WASH_BF16)
+    wantb = np.zeros(c.P, dtype=np.uint16)
+    oracle.population_average(c.ora, c.host, wantb)
+    assert (to_host_bits(outb) == wantb).all()
+    B.papa_all(c.gpu.ctx, B.WASH_STACK_PARAMS)
+    oracle.papa_all(c.ora, c.host)
+    torch.cuda.synchronize()
+    worst = max(worst, _assert_close_f32(to_host_bits(c.dev), bits(c.host), "papa_all"))
+    assert worst == 0          # same operations in the same order: no difference at all
+    B.wash_check(c.gpu.ctx)
+    c.close()
+
+
+@pytest.mark.parametrize("layout", [0, 1])
+@pytest.mark.parametrize("N", [2, 8, 9])
+def test_bf16_stacks(N, layout):
+    c = Case(N, RAGGED, layout, "bf16", seed=N + 60)
+    B.papa_ema(c.gpu.ctx, B.WASH_STACK_PARAMS, 0.999)
+    oracle.papa_ema(c.ora, c.host, 0.999)
+    c.assert_equal("bf16 ema")
+    for code, np_dtype, t_dtype in ((B.WASH_F32, np.float32, torch.float32), (B.WASH_BF16, np.uint16, torch.bfloat16)):
+        out = torch.zeros(c.P, dtype=t_dtype, device="cuda")
+        B.population_average(c.gpu.ctx, B.WASH_STACK_PARAMS, out, code)
+        want = np.zeros(c.P, dtype=np_dtype)
+        oracle.population_average(c.ora, c.host, want)
+        assert (to_host_bits(out) == bits(want)).all()
+    B.papa_all(c.gpu.ctx, B.WASH_STACK_PARAMS)
+    oracle.papa_all(c.ora, c.host)
+    c.assert_equal("bf16 papa_all")
+    c.close()
+
+
+def test_special_values_follow_ieee():
+    N, d = 4, 64
+    dense = W.flat_population(N, d, seed=1)
+    dense[0, 0] = np.inf; dense[1, 1] = -np.inf; dense[2, 2] = np.nan
+    dense[0, 3] = np.inf; dense[1, 3] = -np.inf                     # inf - inf -> NaN
+    dense[:, 4] = np.float32(1e-45)                                 # denormals are kept, not flushed
+    dense[:, 5] = np.array([3e38, 3e38, -3e38, -3e38], np.float32)  # overflow in the running sum
+    c = Case(N, [d], 0, dense=dense)
+    B.papa_ema(c.gpu.ctx, B.WASH_STACK_PARAMS, 0.9)
+    oracle.papa_ema(c.ora, c.host, 0.9)
+    torch.cuda.synchronize()
+    assert ulp_distance_f32(to_host_bits(c.dev), bits(c.host)).max() == 0     # NaN == NaN by class
+    c.close()
+
+
+@pytest.mark.parametrize("layout", [0, 1])
+@pytest.mark.parametrize("N,dtype", [(5, "f32"), (8, "bf16"), (13, "f32")])
+def test_consensus_distance(N, dtype, layout):
+    c = Case(N, RAGGED, layout, dtype, seed=N)
+    out = torch.zeros(N, dtype=torch.float64, device="cuda")
+    B.wash_consensus_sq(c.gpu.ctx, B.WASH_STACK_PARAMS, 0, len(RAGGED), out)
+    want = oracle.consensus_sq(c.ora, c.host)
+    assert np.allclose(out.cpu().numpy(), want, rtol=1e-12, atol=0)
+    part = torch.zeros(N, dtype=torch.float64, device="cuda")
+    B.wash_consensus_sq(c.gpu.ctx, B.WASH_STACK_PARAMS, 2, 7, part)
+    assert np.allclose(part.cpu().numpy(), oracle.consensus_sq(c.ora, c.host, 2, 7), rtol=1e-12, atol=0)
+    # Eq. 5: a shuffle leaves the summed squared distance where it was; Eq. 2: the EMA scales it by alpha^2
+    if dtype == "f32":
+        B.wash_shuffle(c.gpu.ctx, 0, 0.5, None, seed=1)
+        after = torch.zeros(N, dtype=torch.float64, device="cuda")
+        B.wash_consensus_sq(c.gpu.ctx, B.WASH_STACK_PARAMS, 0, len(RAGGED), after)
+        assert abs(after.sum().item() / want.sum() - 1) < 1e-12
+        B.papa_ema(c.gpu.ctx, B.WASH_STACK_PARAMS, 0.9)
+        ema = torch.zeros(N, dtype=torch.float64, device="cuda")
+        B.wash_consensus_sq(c.gpu.ctx, B.WASH_STACK_PARAMS, 0, len(RAGGED), ema)
+        assert abs(ema.sum().item() / after.sum().item() - float(np.float32(0.9)) ** 2) < 1e-5
+    c.close()
+
+
+def test_step_over_host_buffers():
+    N, numel = 5, [3000, 17, 64]
+    c = Case(N, numel, 0, "f32", "f32", seed=12)
+    hp = torch.from_numpy(c.host.reshape(-1).copy()).pin_memory()
+    ho = torch.from_numpy(c.host_opt.reshape(-1).copy()).pin_memory()
+    havg = torch.zeros(c.P, dtype=torch.float32).pin_memory()
+    ops = B.WASH_OP_SHUFFLE | B.WASH_OP_EMA | B.WASH_OP_AVERAGE
+    st = B.wash_step_host(c.gpu.ctx, ops, hp, ho, havg, 3, 0.25, None, seed=4, alpha=0.99)
+    want_st = oracle.shuffle(c.ora, c.host, 0.25, seed=4, step=3, stack2=c.host_opt)
+    oracle.papa_ema(c.ora, c.host, 0.99)
+    want_avg = np.zeros(c.P, dtype=np.float32)
+    oracle.population_average(c.ora, c.host, want_avg)
+    assert st == want_st
+    assert (hp.numpy().view(np.uint32) == bits(c.host)).all()
+    assert (ho.numpy().view(np.uint32) == bits(c.host_opt)).all()
+    assert (havg.numpy().view(np.uint32) == want_avg.view(np.uint32)).all()
+    c.close()
