@@ -1,0 +1,435 @@
+#!/usr/bin/env python
+"""Benchmark of the WASH hot path on B200: one JSON line on stdout.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+                    [--workload cfg2_resnet18_n5|cfg3_resnet50_n10|cfg4_resnet50_bf16_n8|cfg1_flat_n3]
+
+A step is one pass of the whole hot path over one synthetic population: the shuffle of
+the parameter and momentum stacks (WASH+Opt, one launch), PAPA's EMA on the parameters
+and the final average -- three kernel launches.  `value` is the bytes those kernels
+must stream (see algorithmic_bytes) divided by the step time, in GB/s, with the stacks
+resident in HBM; `e2e` is the same through wash_step_host with the stacks in pinned
+host memory (copies inside the timed region).  For N > 1 (torchrun) every rank holds
+its own shard of an N-times deeper population (tensor indices offset by rank), no
+communication: weak scaling.
+
+--impl reference times the CPU oracle (oracle/) on the host cores instead.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2405_17517_b200 import workloads as W  # noqa: E402
+
+METRIC = "shuffle GB/s and parameter-swaps/s at 1 B200; % of HBM roofline"
+FALLBACK_HBM_GBS = 6650.0
+ALPHA = 0.99
+SEED = 0
+
+
+def measured_peak():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured (MEASURED_PEAKS.json hbm_gbs)"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback (no MEASURED_PEAKS.json)"
+
+
+class Workload:
+    def __init__(self, name: str, rank: int = 0):
+        cfg = W.CONFIGS[name]
+        self.name, self.cfg = name, cfg
+        self.N = cfg["N"]
+        self.table = W.table_from_spec(cfg["table"])
+        self.numel = W.numels(self.table)
+        self.T = len(self.table)
+        self.P = int(self.numel.sum())
+        self.p = cfg["p"]
+        self.bf16 = cfg["dtype"] == "bf16"
+        self.opt = cfg["opt"]
+        self.E = 2 if self.bf16 else 4
+        self.E_opt = 4 if self.opt else 0
+        # rank r holds tensors r*T .. r*T+T-1 of a world_size-times deeper population
+        self.tensor_id = np.arange(self.T, dtype=np.uint32) + np.uint32(rank * self.T)
+        self.schedule = cfg["schedule"]     # None = uniform p; each arm derives p_layer with its own routine
+        self.p_layer = None
+        self.rank = rank
+
+    def algorithmic_bytes(self, selected: float) -> dict:
+        """Bytes each kernel must move per launch (logical coordinates only)."""
+        N, P = self.N, self.P
+        shuffle = N * P * (self.E + self.E_opt) + selected * N * (self.E + self.E_opt)   # read all, write selected
+        ema = 2 * N * P * self.E
+        avg = N * P * self.E + P * self.E
+        return {"shuffle": shuffle, "ema": ema, "average": avg, "step": shuffle + ema + avg}
+
+    def host_stacks(self, offsets, padded_P):
+        dense = W.init_population(self.table, self.N, seed=SEED + 17 * self.rank) if self.T > 1 else \
+            W.flat_population(self.N, self.P, seed=SEED + 17 * self.rank, std=0.05)
+        if self.bf16:
+            dense = W.to_bf16_bits(dense)
+        params = W.to_stack(dense, self.numel, offsets, padded_P)
+        opt = None
+        if self.opt:
+            opt = W.to_stack(W.init_momentum(self.table, self.N, seed=SEED + 1 + 17 * self.rank), self.numel, offsets, padded_P)
+        return params, opt
+
+
+class ClockSampler(threading.Thread):
+    """Samples SM clock and throttle reasons (read-only NVML queries) while running."""
+
+    def __init__(self, index: int, period: float = 0.02):
+        super().__init__(daemon=True)
+        self.index, self.period = index, period
+        self.samples, self.reasons = [], set()
+        self.max_mhz = None
+        self._halt = threading.Event()
+        self.ok = False
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = int(pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM))
+            self.ok = True
+        except Exception:
+            self.nv = None
+
+    def run(self):
+        if not self.ok:
+            return
+        nv = self.nv
+        names = {
+            getattr(nv, "nvmlClocksThrottleReasonHwSlowdown", 0x8): "hw_slowdown",
+            getattr(nv, "nvmlClocksThrottleReasonHwThermalSlowdown", 0x40): "hw_thermal_slowdown",
+            getattr(nv, "nvmlClocksThrottleReasonSwThermalSlowdown", 0x20): "sw_thermal_slowdown",
+            getattr(nv, "nvmlClocksThrottleReasonSwPowerCap", 0x4): "sw_power_cap",
+            getattr(nv, "nvmlClocksThrottleReasonHwPowerBrakeSlowdown", 0x80): "hw_power_brake_slowdown",
+        }
+        while not self._halt.is_set():
+            try:
+                self.samples.append(int(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM)))
+                mask = int(nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h))
+                for bit, name in names.items():
+                    if mask & bit:
+                        self.reasons.add(name)
+            except Exception:
+                pass
+            self._halt.wait(self.period)
+
+    def stop(self) -> dict:
+        self._halt.set()
+        if self.is_alive():
+            self.join(timeout=2)
+        med = float(np.median(self.samples)) if self.samples else None
+        return {"sm_mhz": med, "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons), "samples": len(self.samples)}
+
+
+def physical_gpu_index(local: int) -> int:
+    vis = os.environ.get("CUDA_VISIBLE_DEVICES")
+    if vis:
+        try:
+            return int(vis.split(",")[local])
+        except Exception:
+            return local
+    return local
+
+
+# ------------------------------------------------------------------------------------
+def run_reference(args, rank: int, world: int) -> None:
+    """The CPU oracle, as it stands, on the host cores (rank 0 only)."""
+    if rank != 0:
+        return
+    import oracle
+    wl = Workload(args.workload, 0)
+    offsets, padded_P = W.padded_offsets(wl.numel)
+    threads = oracle.max_threads()
+    oracle.set_threads(threads)
+    params, opt = wl.host_stacks(offsets, padded_P)
+    if wl.schedule == "decreasing":
+        wl.p_layer = oracle.layer_probs(wl.T, wl.p, oracle.SCHEDULE_DECREASING)
+
+    def one_step(pop, a, b, out, step, p_layer):
+        p = wl.p if p_layer is None else p_layer
+        st = oracle.shuffle(pop, a, p, seed=SEED, step=step, stack2=b)
+        oracle.papa_ema(pop, a, ALPHA)
+        oracle.population_average(pop, a, out)
+        return st
+
+    full = oracle.Population(wl.N, wl.numel, offsets, padded_P, oracle.LAYOUT_NP, wl.tensor_id)
+    out = np.zeros(padded_P, dtype=params.dtype)
+    t0 = time.perf_counter()
+    one_step(full, params, opt, out, 0, wl.p_layer)
+    t_full = time.perf_counter() - t0
+    # bounded sample: a prefix of the tensor table, so that warmup + steps stay near a minute
+    budget = 60.0
+    frac = min(1.0, budget / max(t_full * (args.steps + args.warmup), 1e-9))
+    cum = np.cumsum(wl.numel)
+    n_t = int(np.searchsorted(cum, frac * wl.P, side="left")) + 1 if frac < 1.0 else wl.T
+    n_t = max(1, min(wl.T, n_t))
+    sub_numel = wl.numel[:n_t]
+    sub_P = int(sub_numel.sum())
+    sub_off, sub_padded = W.padded_offsets(sub_numel)
+    rows = params.reshape(wl.N, padded_P)
+    sp = np.ascontiguousarray(rows[:, :sub_padded])
+    so = np.ascontiguousarray(opt.reshape(wl.N, padded_P)[:, :sub_padded]) if opt is not None else None
+    sub = oracle.Population(wl.N, sub_numel, sub_off, sub_padded, oracle.LAYOUT_NP, wl.tensor_id[:n_t])
+    sub_pl = None if wl.p_layer is None else wl.p_layer[:n_t]
+    sout = np.zeros(sub_padded, dtype=params.dtype)
+    for w in range(args.warmup):
+        one_step(sub, sp, so, sout, w, sub_pl)
+    sel = 0
+    t0 = time.perf_counter()
+    for k in range(args.steps):
+        sel += one_step(sub, sp, so, sout, args.warmup + k, sub_pl)[0]
+    dt = time.perf_counter() - t0
+    scale = sub_P / wl.P
+    bytes_step = wl.algorithmic_bytes(sel / max(args.steps, 1) / scale)["step"] * scale
+    gbs = bytes_step * args.steps / dt / 1e9
+    sample = "first %d of %d tensors (%d of %d coordinates per model) per step" % (n_t, wl.T, sub_P, wl.P)
+    line = {
+        "impl": "reference", "metric": METRIC, "value": gbs, "unit": "GB/s", "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": dt / max(args.steps, 1) * 1e3, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "bf16+f32" if wl.bf16 else "f32", "data": "synthetic",
+        "config": {"workload": wl.name, "N": wl.N, "tensors": wl.T, "P": wl.P, "p": wl.p, "sample": sample},
+        "param_swaps_per_s": sel * wl.N / dt,
+        "cpu_baseline": {"value": gbs, "unit": "GB/s", "cores": threads, "kind": "oracle", "sample": sample},
+        "e2e": {"value": gbs, "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+# ------------------------------------------------------------------------------------
+def run_ours(args, rank: int, world: int, local_rank: int) -> None:
+    import torch
+    from paper_2405_17517_b200 import binding as B
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU path)")
+    if not os.path.exists(B.LIB_PATH):
+        if rank == 0:
+            from paper_2405_17517_b200 import build as wash_build
+            wash_build.build()
+    dist = None
+    if world > 1:
+        import torch.distributed as dist_mod
+        dist = dist_mod
+        torch.cuda.set_device(local_rank)
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+        dist.barrier()
+    else:
+        torch.cuda.set_device(local_rank)
+    B.load()
+    dev = local_rank
+    wl = Workload(args.workload, rank)
+    pop = B.Population(wl.N, wl.numel, B.WASH_LAYOUT_NP, dev, wl.tensor_id)
+    params_h, opt_h = wl.host_stacks(pop.offsets, pop.padded_P)
+
+    def to_torch(a):
+        t = torch.from_numpy(a.reshape(-1).view(np.int16) if a.dtype == np.uint16 else a.reshape(-1))
+        return t.view(torch.bfloat16) if a.dtype == np.uint16 else t
+
+    params_pin = to_torch(params_h).pin_memory()
+    opt_pin = to_torch(opt_h).pin_memory() if opt_h is not None else None
+    params_d = params_pin.cuda(non_blocking=True)
+    opt_d = opt_pin.cuda(non_blocking=True) if opt_pin is not None else None
+    avg_d = torch.zeros(pop.padded_P, dtype=params_d.dtype, device="cuda")
+    avg_pin = torch.zeros(pop.padded_P, dtype=params_d.dtype).pin_memory()
+    stats_d = torch.zeros(2, dtype=torch.int64, device="cuda")
+    pop.bind(B.WASH_STACK_PARAMS, params_d)
+    if opt_d is not None:
+        pop.bind(B.WASH_STACK_OPT, opt_d)
+    if args.mode == "sparse":
+        B.wash_set_mode(pop.ctx, B.WASH_MODE_SPARSE)
+    if args.threads or args.blocks_per_sm:
+        B.wash_set_launch(pop.ctx, args.threads, args.blocks_per_sm)
+    pdt = B.WASH_BF16 if wl.bf16 else B.WASH_F32
+    if wl.schedule == "decreasing":
+        wl.p_layer = B.wash_layer_probs(wl.T, wl.p, B.WASH_SCHEDULE_DECREASING)
+    p_layer = wl.p_layer
+    stream = torch.cuda.current_stream()
+
+    def step(i, ev=None):
+        if ev is not None:
+            ev[0].record(stream)
+        if opt_d is not None:
+            B.wash_shuffle_both(pop.ctx, i, wl.p, p_layer, SEED, stream, stats_d)
+        else:
+            B.wash_shuffle(pop.ctx, i, wl.p, p_layer, SEED, stream, stats_d)
+        if ev is not None:
+            ev[1].record(stream)
+        B.papa_ema(pop.ctx, B.WASH_STACK_PARAMS, ALPHA, stream)
+        if ev is not None:
+            ev[2].record(stream)
+        B.population_average(pop.ctx, B.WASH_STACK_PARAMS, avg_d, pdt, stream)
+        if ev is not None:
+            ev[3].record(stream)
+
+    def fence():
+        torch.cuda.synchronize()
+        if dist is not None:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    for w in range(args.warmup):
+        step(w)
+    fence()
+    stats_d.zero_()
+    launches0 = B.wash_launch_count()
+    events = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(args.steps)]
+    sampler = ClockSampler(physical_gpu_index(local_rank))
+    sampler.start()
+    fence()
+    t_begin = torch.cuda.Event(enable_timing=True)
+    t_end = torch.cuda.Event(enable_timing=True)
+    t_begin.record(stream)
+    for k in range(args.steps):
+        step(args.warmup + k, events[k])
+    t_end.record(stream)
+    fence()
+    clocks = sampler.stop()
+    launches = B.wash_launch_count() - launches0
+    B.wash_check(pop.ctx)
+    total_ms = t_begin.elapsed_time(t_end)
+    st = stats_d.cpu().numpy().view(np.uint64)
+    selected_total, moved_total = int(st[0]), int(st[1])
+    k_ms = np.array([[e[i].elapsed_time(e[i + 1]) for i in range(3)] for e in events])   # shuffle, ema, average
+    mean_ms = k_ms.mean(axis=0)
+
+    # ---- end to end through the host-buffer entry point --------------------------------
+    e2e_steps = max(1, min(args.steps, 5))
+    ops = B.WASH_OP_SHUFFLE | B.WASH_OP_EMA | B.WASH_OP_AVERAGE
+    B.wash_step_host(pop.ctx, ops, params_pin, opt_pin, avg_pin, 0, wl.p, p_layer, SEED, ALPHA, stream)   # warm
+    fence()
+    e0 = torch.cuda.Event(enable_timing=True)
+    e1 = torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for k in range(e2e_steps):
+        B.wash_step_host(pop.ctx, ops, params_pin, opt_pin, avg_pin, 1 + k, wl.p, p_layer, SEED, ALPHA, stream)
+    e1.record(stream)
+    fence()
+    e2e_ms = e0.elapsed_time(e1)
+    stack_bytes = params_pin.numel() * params_pin.element_size() + (opt_pin.numel() * opt_pin.element_size() if opt_pin is not None else 0)
+    h2d = stack_bytes
+    d2h = stack_bytes + avg_pin.numel() * avg_pin.element_size() + 16
+
+    # ---- max over ranks ------------------------------------------------------------------
+    if dist is not None:
+        t = torch.tensor([total_ms, e2e_ms, mean_ms[0], mean_ms[1], mean_ms[2]], dtype=torch.float64, device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms, e2e_ms = float(t[0]), float(t[1])
+        mean_ms = t[2:].cpu().numpy()
+        c = torch.tensor([selected_total, moved_total], dtype=torch.int64, device="cuda")
+        dist.all_reduce(c, op=dist.ReduceOp.SUM)
+        selected_total, moved_total = int(c[0]), int(c[1])
+
+    if rank == 0:
+        sel_per_step_rank = selected_total / args.steps / world
+        ab = wl.algorithmic_bytes(sel_per_step_rank)
+        step_ms = total_ms / args.steps
+        value = ab["step"] * world / (step_ms * 1e-3) / 1e9
+        peak, peak_src = measured_peak()
+        shuffle_gbs = ab["shuffle"] / (mean_ms[0] * 1e-3) / 1e9
+        line = {
+            "metric": METRIC, "value": value, "unit": "GB/s", "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+            "ms_per_step": step_ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "bf16+f32" if wl.bf16 else "f32", "data": "synthetic",
+            "value_definition": "bytes the three kernels of one step must stream (shuffle: read both stacks + write selected; "
+                                "EMA: read+write parameters; average: read parameters + write one row) / step time, all ranks",
+            "config": {"workload": wl.name, "N": wl.N, "tensors": wl.T, "P": wl.P, "p": wl.p,
+                       "per_layer_p": wl.p_layer is not None, "opt_state": wl.opt, "layout": "[N][P]", "mode": args.mode,
+                       "footprint_bytes_per_gpu": stack_bytes, "l2": "inputs larger than L2 (no flush)" if stack_bytes > 2.5e8 else "L2-resident: footprint below 2x L2",
+                       "sharding": "one population shard per rank, no collective"},
+            "param_swaps_per_s": selected_total * wl.N / (total_ms * 1e-3),
+            "moved_values_per_s": moved_total / (total_ms * 1e-3),
+            "selected_coords_per_step": selected_total / args.steps,
+            "kernels": {
+                "shuffle": {"ms": float(mean_ms[0]), "GBps": shuffle_gbs, "frac_of_hbm": shuffle_gbs / peak},
+                "papa_ema": {"ms": float(mean_ms[1]), "GBps": ab["ema"] / (mean_ms[1] * 1e-3) / 1e9},
+                "population_average": {"ms": float(mean_ms[2]), "GBps": ab["average"] / (mean_ms[2] * 1e-3) / 1e9},
+            },
+            "roofline": {"kernel": "shuffle_kernel (params + momentum, streaming)", "bound": "hbm", "achieved": shuffle_gbs,
+                         "peak": peak, "peak_source": peak_src, "unit": "GB/s", "frac": shuffle_gbs / peak,
+                         "traffic": TRAFFIC.get(wl.name)},
+            "e2e": {"value": ab["step"] * world / (e2e_ms / e2e_steps * 1e-3) / 1e9, "unit": "GB/s",
+                    "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": e2e_steps,
+                    "api": "wash_step_host (pinned host stacks)"},
+            "gpu_launches": int(launches),
+            "clocks": clocks,
+        }
+        if world == 1 and not args.no_cpu_baseline:
+            line["cpu_baseline"] = cpu_baseline(wl)
+        print(json.dumps(line), flush=True)
+    pop.close()
+    if dist is not None:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+# DRAM bytes per shuffle launch from the ncu capture summarised under profiles/ (None
+# until a capture of the current kernel exists).
+TRAFFIC = {}
+
+
+def cpu_baseline(wl: Workload) -> dict:
+    """The oracle as it stands on the host cores, on a bounded number of full steps."""
+    import oracle
+    offsets, padded_P = W.padded_offsets(wl.numel)
+    params, opt = wl.host_stacks(offsets, padded_P)
+    pop = oracle.Population(wl.N, wl.numel, offsets, padded_P, oracle.LAYOUT_NP, wl.tensor_id)
+    out = np.zeros(padded_P, dtype=params.dtype)
+    threads = oracle.max_threads()
+    oracle.set_threads(threads)
+    p = wl.p if wl.schedule is None else oracle.layer_probs(wl.T, wl.p, oracle.SCHEDULE_DECREASING)
+    steps, sel, t0 = 0, 0, time.perf_counter()
+    while True:
+        sel += oracle.shuffle(pop, params, p, seed=SEED, step=steps, stack2=opt)[0]
+        oracle.papa_ema(pop, params, ALPHA)
+        oracle.population_average(pop, params, out)
+        steps += 1
+        dt = time.perf_counter() - t0
+        if dt > 10.0 or steps >= 50:
+            break
+    gbs = wl.algorithmic_bytes(sel / steps)["step"] * steps / dt / 1e9
+    return {"value": gbs, "unit": "GB/s", "cores": threads, "kind": "oracle",
+            "sample": "%d full steps of the same workload (%.1f s)" % (steps, dt), "ms_per_step": dt / steps * 1e3}
+
+
+def main() -> None:
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="cfg2_resnet18_n5", choices=sorted(W.CONFIGS))
+    ap.add_argument("--mode", default="stream", choices=["stream", "sparse"])
+    ap.add_argument("--threads", type=int, default=0)
+    ap.add_argument("--blocks-per-sm", type=int, default=0)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.warmup < 3 and args.impl == "ours":
+        args.warmup = 3
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if args.impl == "reference":
+        run_reference(args, rank, world)
+    else:
+        run_ours(args, rank, world, local_rank)
+
+
+if __name__ == "__main__":
+    main()
