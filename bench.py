@@ -90,7 +90,7 @@ class Workload:
 class ClockSampler(threading.Thread):
     """Samples SM clock and throttle reasons (read-only NVML queries) while running."""
 
-    def __init__(self, index: int, period: float = 0.02):
+    def __init__(self, index: int, period: float = 0.01):
         super().__init__(daemon=True)
         self.index, self.period = index, period
         self.samples, self.reasons = [], set()
@@ -411,7 +411,7 @@ def cpu_baseline(wl: Workload) -> dict:
 def main() -> None:
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--steps", type=int, default=2000)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="cfg2_resnet18_n5", choices=sorted(W.CONFIGS))

@@ -114,8 +114,9 @@ int wash_bind(wash_ctx *ctx, int32_t stack, int32_t dtype, void *dev_ptr, int64_
 int wash_set_mode(wash_ctx *ctx, int32_t mode);
 
 /* Launch shape override for tuning: threads per block (multiple of 32 in 64..256;
- * 0 = default) and blocks per SM for the persistent grids (0 = as many as fit;
- * negative = no persistence, one group per thread). */
+ * 0 = default) and grid style: blocks_per_sm <= 0 (default) launches one group of 4
+ * coordinates per thread; blocks_per_sm > 0 launches a persistent grid of SM count x
+ * min(blocks_per_sm, resident blocks per SM) blocks that stride over the groups. */
 int wash_set_launch(wash_ctx *ctx, int32_t threads, int32_t blocks_per_sm);
 
 /* ---- the shuffling step ----------------------------------------------------------- */

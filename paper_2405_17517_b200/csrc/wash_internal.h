@@ -58,7 +58,7 @@ enum ReduceOp { kOpEma = 0, kOpAverage = 1, kOpPapaAll = 2, kOpConsensus = 3 };
 
 struct LaunchShape {
     int threads;         // 0 = default
-    int blocks_per_sm;   // 0 = as many as fit, < 0 = one group per thread
+    int blocks_per_sm;   // <= 0: one group per thread; > 0: persistent grid, that many blocks per SM
     int sm_count;
 };
 

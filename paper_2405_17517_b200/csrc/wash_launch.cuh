@@ -1,5 +1,7 @@
-// Grid sizing for the grid-stride kernels: a persistent grid of (SM count x resident
-// blocks per SM), or fewer blocks when the work is smaller.
+// Grid sizing for the grid-stride kernels.  By default one work item per thread (the
+// block scheduler then balances the SMs; measured faster than a persistent grid for
+// these short streaming kernels); on request a persistent grid of SM count x blocks
+// per SM.
 #pragma once
 #include <cstdint>
 #include <map>
@@ -60,9 +62,9 @@ cudaError_t launch_grid_stride(void (*kernel)(Args), const Args &args, uint64_t 
     if (fit.occupancy < 1) return cudaErrorLaunchOutOfResources;
     const uint64_t need = (n_items + threads - 1) / threads;
     uint64_t grid = need;
-    if (shape.blocks_per_sm >= 0) {   // persistent grid; negative = one trip per thread
+    if (shape.blocks_per_sm > 0) {   // persistent grid; otherwise one trip per thread
         int bps = fit.occupancy;
-        if (shape.blocks_per_sm > 0 && shape.blocks_per_sm < bps) bps = shape.blocks_per_sm;
+        if (shape.blocks_per_sm < bps) bps = shape.blocks_per_sm;
         const uint64_t resident = static_cast<uint64_t>(shape.sm_count > 0 ? shape.sm_count : 148) * bps;
         if (grid > resident) grid = resident;
     }
