@@ -194,6 +194,54 @@ int wash_step_host(wash_ctx *ctx, int32_t ops, void *host_params, void *host_opt
                    uint64_t step, double p, const double *p_layer, uint64_t seed, float alpha,
                    void *stream, wash_stats *host_stats);
 
+/* ---- for callers that must not allocate ------------------------------------------- */
+
+#define WASH_NOALLOC_MAX_TENSORS 1024                 /* most tensors per model            */
+#define WASH_NOALLOC_MAX_ROW_ELEMS (1ll << 26)        /* longest padded row, in elements   */
+
+/* The paper has no counterpart to this call; it exists for deployment reasons only.
+ *
+ * wash_create puts the context's lookup tables in device memory with cudaMalloc.  Two
+ * kinds of caller cannot afford that: a process in which a framework's memory pool has
+ * already taken the whole GPU (an allocation from this library would fail or compete
+ * with the pool), and a latency-critical loop in which cudaMalloc / cudaFree, which
+ * synchronise the whole device, would stall work that other streams have in flight.
+ * wash_shuffle_noalloc runs the same streaming shuffle as wash_shuffle on ONE stack
+ * without any context and without allocating device or pinned memory: its tables live
+ * in a fixed 288 KiB array inside the library image (32 KiB segment table + 256 KiB tile
+ * index), which every GPU that loads libwash.so holds until the process exits.
+ *
+ *   N, n_tensors, numel, layout     as for wash_create (row geometry is the same:
+ *                                   tensors start on multiples of 8 elements);
+ *   dtype, dev_stack, n_elems       as for wash_bind: a DEVICE stack of N * padded_P
+ *                                   elements, 16-byte aligned, borrowed for the call;
+ *   step, p, p_layer, seed, stats   as for wash_shuffle (stats: DEVICE-accessible,
+ *                                   added to, may be NULL);
+ *   device                          ordinal of the GPU that owns dev_stack.
+ *
+ * Limits: n_tensors <= WASH_NOALLOC_MAX_TENSORS and padded_P <=
+ * WASH_NOALLOC_MAX_ROW_ELEMS; anything larger is refused with WASH_ERR_ARG (use a
+ * context instead).  The result is bit-identical to wash_shuffle with the same
+ * arguments.  The message of a failure is returned by wash_noalloc_last_error().
+ *
+ * Sharing: all calls on a GPU use the one array.  Each call rewrites the tables it
+ * needs in full, in stream order, so nothing has to be cleared between calls and the
+ * previous call's contents never leak into the next; but two calls that can overlap on
+ * the GPU (different streams without an ordering between them, or two host threads)
+ * race on the tables and give undefined results.  Issue them on one stream, or order
+ * them with events.
+ *
+ * First use: the first call on each device looks up that device's address of the array
+ * (cudaGetSymbolAddress, with the device made current for the duration of the call).
+ * Make that first call before any stream capture begins. */
+int wash_shuffle_noalloc(int32_t N, int32_t n_tensors, const int64_t *numel, int32_t layout,
+                         int32_t dtype, void *dev_stack, int64_t n_elems, uint64_t step, double p,
+                         const double *p_layer, uint64_t seed, int32_t device, void *stream,
+                         wash_stats *stats);
+
+/* Message for the calling thread's most recent wash_shuffle_noalloc failure. */
+const char *wash_noalloc_last_error(void);
+
 /* ---- diagnostics ------------------------------------------------------------------ */
 
 /* Waits for `stream` and returns WASH_ERR_DEVICE_CHECK if a kernel recorded an

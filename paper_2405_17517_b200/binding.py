@@ -70,9 +70,8 @@ def load() -> ctypes.CDLL:
     L.wash_check.argtypes = [vp, vp]
     L.wash_last_error.restype = ctypes.c_char_p
     L.wash_launch_count.restype = ctypes.c_uint64
-    for name in ("wash_shuffle_noalloc",):
-        if hasattr(L, name):
-            getattr(L, name).restype = ctypes.c_int
+    L.wash_shuffle_noalloc.argtypes = [i32, i32, i64p, i32, i32, vp, i64, u64, dbl, dblp, u64, i32, vp, vp]
+    L.wash_noalloc_last_error.restype = ctypes.c_char_p
     _lib = L
     return L
 
@@ -208,6 +207,21 @@ def wash_step_host(ctx, ops: int, host_params, host_opt, host_avg, step, p, p_la
     _check(load().wash_step_host(ctx, ops, _ptr(host_params), _ptr(host_opt), _ptr(host_avg), step, float(p), pl,
                                  seed, ctypes.c_float(alpha), _stream(stream), ctypes.byref(st)))
     return int(st.selected_coords), int(st.moved_values)
+
+
+def wash_shuffle_noalloc(N: int, numel, layout: int, dtype: int, dev_stack, n_elems: int, step: int, p: float,
+                         p_layer=None, seed: int = 0, device: int = 0, stream=None, stats=None) -> None:
+    """The streaming shuffle without a context and without any allocation (see wash.h)."""
+    arr, np_ = _i64(numel)
+    keep, pl = _dbl_or_null(p_layer)
+    rc = load().wash_shuffle_noalloc(N, arr.size, np_, layout, dtype, _ptr(dev_stack), n_elems, step, float(p), pl,
+                                     seed, device, _stream(stream), _ptr(stats))
+    if rc != WASH_OK:
+        raise WashError(rc, load().wash_noalloc_last_error().decode())
+
+
+def wash_noalloc_last_error() -> str:
+    return load().wash_noalloc_last_error().decode()
 
 
 def wash_check(ctx, stream=None) -> None:
