@@ -57,7 +57,9 @@ enum wash_stack { WASH_STACK_PARAMS = 0, WASH_STACK_OPT = 1 };
 enum wash_schedule { WASH_SCHEDULE_DECREASING = 0, WASH_SCHEDULE_CONSTANT = 1, WASH_SCHEDULE_INCREASING = 2 };
 enum wash_mode {
     WASH_MODE_STREAM = 0, /* one pass that reads the whole stack; writes selected coordinates */
-    WASH_MODE_SPARSE = 1  /* draws the mask first; touches only selected coordinates          */
+    WASH_MODE_SPARSE = 1, /* draws the mask first; touches only selected coordinates          */
+    WASH_MODE_STREAM_STAGED = 2 /* as STREAM, the stack staged through shared memory by bulk
+                                   asynchronous copies instead of through registers          */
 };
 
 #define WASH_MAX_N 64            /* largest population                                     */

@@ -367,7 +367,7 @@ int wash_bind(wash_ctx *ctx, int32_t stack, int32_t dtype, void *dev_ptr, int64_
 int wash_set_mode(wash_ctx *ctx, int32_t mode)
 {
     if (!ctx) return fail(WASH_ERR_ARG, "ctx is NULL");
-    if (mode != WASH_MODE_STREAM && mode != WASH_MODE_SPARSE) return fail(WASH_ERR_ARG, "unknown mode %d", mode);
+    if (mode != WASH_MODE_STREAM && mode != WASH_MODE_SPARSE && mode != WASH_MODE_STREAM_STAGED) return fail(WASH_ERR_ARG, "unknown mode %d", mode);
     ctx->mode = mode;
     return WASH_OK;
 }
@@ -375,7 +375,7 @@ int wash_set_mode(wash_ctx *ctx, int32_t mode)
 int wash_set_launch(wash_ctx *ctx, int32_t threads, int32_t blocks_per_sm)
 {
     if (!ctx) return fail(WASH_ERR_ARG, "ctx is NULL");
-    if (threads != 0 && (threads < 64 || threads > 256 || (threads & 31))) return fail(WASH_ERR_ARG, "threads = %d: need 0 or a multiple of 32 in [64, 256]", threads);
+    if (threads != 0 && (threads < 32 || threads > 256 || (threads & 31))) return fail(WASH_ERR_ARG, "threads = %d: need 0 or a multiple of 32 in [32, 256]", threads);
     ctx->shape.threads = threads;
     ctx->shape.blocks_per_sm = blocks_per_sm;
     return WASH_OK;

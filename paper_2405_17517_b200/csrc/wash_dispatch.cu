@@ -11,6 +11,7 @@ namespace wash {
 WASH_N_LIST(WASH_DECL)
 #undef WASH_DECL
 cudaError_t launch_shuffle_sparse(const ShuffleArgs &, int, int, const LaunchShape &, cudaStream_t, bool *);
+cudaError_t launch_shuffle_staged(const ShuffleArgs &, int, int, const LaunchShape &, cudaStream_t, bool *);
 cudaError_t launch_reduce_n0(const ReduceArgs &, int, int, int, const LaunchShape &, cudaStream_t, bool *);
 
 static std::atomic<uint64_t> g_launches{0};
@@ -32,6 +33,7 @@ bool has_unrolled_kernels(int N)
 cudaError_t launch_shuffle(const ShuffleArgs &args, int a_dtype, int b_dtype, int mode,
                            const LaunchShape &shape, cudaStream_t stream, bool *supported)
 {
+    if (mode == kModeStreamStaged) return launch_shuffle_staged(args, a_dtype, b_dtype, shape, stream, supported);
     if (mode == kModeStream) {
         switch (args.pop.N) {
 #define WASH_CASE(n) case n: return launch_shuffle_stream_n##n(args, a_dtype, b_dtype, shape, stream, supported);

@@ -9,7 +9,7 @@ constexpr int kMaxN = 64;          // largest population (WASH_MAX_N)
 constexpr int kTileShift = 8;      // lookup tile = 256 groups = 1024 coordinates
 constexpr int kDtypeF32 = 0, kDtypeBF16 = 1, kDtypeNone = -1;
 constexpr int kLayoutNP = 0, kLayoutPN = 1;
-constexpr int kModeStream = 0, kModeSparse = 1;
+constexpr int kModeStream = 0, kModeSparse = 1, kModeStreamStaged = 2;
 
 // One row of a stack is cut into groups of 4 consecutive elements; a group never
 // straddles two tensors because tensors start on multiples of 8 elements.

@@ -1,0 +1,320 @@
+// Streaming shuffle with the stack staged through shared memory by the bulk-copy
+// engine (TMA, cp.async.bulk) instead of through registers.
+//
+// Why: the register-resident kernel keeps N (or 2N) vectors per thread in flight and is
+// limited by how many such threads fit on an SM (measured: 24 warps, ~120 KB in flight
+// per SM, 85 % of the bandwidth a pure read reaches).  Here one producer warp per CTA
+// streams tiles of the stack into a ring of shared-memory stages with bulk asynchronous
+// copies that complete on mbarriers; ~200 KB per SM are in flight with no register
+// cost, and the consumer warps spend their time on the Philox mask, which needs no data
+// at all.  A consumer touches a stage only for a selected coordinate (it then reads the
+// N values from shared memory and writes the moved ones to global memory) and to hand
+// the stage back.  N is a run-time value: one instantiation serves every population size.
+//
+// Tile = G consecutive groups (G = threads of one consumer team).  [N][P]: one bulk copy
+// per model row and stack (G*16 bytes of fp32).  [P][N]: the tile's G*4N elements are
+// contiguous, one copy per stack.  Every copy starts on a 16-byte boundary and has a
+// size that is a multiple of 16 bytes (rows start on multiples of 8 elements, a group
+// is 16 or 8 bytes, G is a multiple of 32).
+//
+// All waits are bounded: a wait that exceeds kWaitLimitNs sets bit 1 of the status word
+// and an abort flag that every loop checks; the producer then still waits (bounded) for
+// the copies it has issued before the CTA returns.
+#pragma once
+#include "wash_device.cuh"
+#include "wash_launch.cuh"
+
+namespace wash {
+
+constexpr unsigned long long kWaitLimitNs = 2000000000ull;   // 2 s
+constexpr int kMaxStages = 12;
+
+struct ShuffleTmaArgs {
+    ShuffleArgs s;
+    uint32_t n_tiles;        // ceil(n_groups / G)
+    int G;                   // groups per tile = threads per consumer team
+    int teams;               // consumer teams per CTA (tile i of a CTA goes to team i % teams)
+    int stages;
+    uint32_t stage_bytes;    // bytes of one stage (both stacks)
+    uint32_t b_offset;       // byte offset of the second stack inside a stage
+};
+
+__device__ __forceinline__ uint32_t smem_addr(const void *p) { return static_cast<uint32_t>(__cvta_generic_to_shared(p)); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
+{
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar)
+{
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+                 : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+__device__ __forceinline__ unsigned long long global_timer_ns()
+{
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+// Waits for the phase of parity `parity` to complete.  Returns false if the CTA is
+// aborting or the wait ran out of time (then it sets the abort flag and the status bit).
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag, uint32_t *status)
+{
+    if (mbar_try_wait(bar, parity)) return true;
+    const unsigned long long t0 = global_timer_ns();
+    for (uint32_t polls = 1;; ++polls) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if ((polls & 255u) == 0) {
+            if (*abort_flag) return false;
+            if (global_timer_ns() - t0 > kWaitLimitNs) {
+                *abort_flag = 1;
+                if (status) atomicOr(status, 2u);
+                return false;
+            }
+        }
+    }
+}
+// global -> shared bulk copy that reports its bytes to an mbarrier of this CTA
+__device__ __forceinline__ void bulk_load(uint32_t dst_smem, const void *src, uint32_t bytes, uint32_t bar)
+{
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(dst_smem), "l"(src), "r"(bytes), "r"(bar) : "memory");
+}
+
+// pi for coordinate i in a column of bytes: s_perm[n * stride]
+static __device__ __noinline__ void draw_permutation_u8(uint8_t *s_perm, int stride, int n_models, uint32_t i,
+                                                        uint32_t tensor, uint32_t step_lo, uint32_t step_hi8,
+                                                        uint32_t k0, uint32_t k1)
+{
+    for (int n = 0; n < n_models; ++n) s_perm[n * stride] = static_cast<uint8_t>(n);
+    Philox4 w{0, 0, 0, 0};
+    for (int k = n_models - 1, m = 0; k >= 1; --k, ++m) {
+        if ((m & 3) == 0) w = philox4x32_10(i, tensor, step_lo, step_hi8 | (1u + (static_cast<uint32_t>(m) >> 2)), k0, k1);
+        const uint32_t r = w.x;
+        w.x = w.y; w.y = w.z; w.z = w.w;
+        const uint32_t j = __umulhi(r, static_cast<uint32_t>(k + 1));
+        const uint8_t pk = s_perm[k * stride], pj = s_perm[j * stride];
+        s_perm[k * stride] = pj;
+        s_perm[j * stride] = pk;
+    }
+}
+
+// raw bits of (model n, coordinate c) of the tile's group j, read from a stage
+template <class T, int LAYOUT>
+__device__ __forceinline__ uint32_t stage_value(const unsigned char *stage, int G, int n_models, int n, int j, int c)
+{
+    const uint32_t elem = LAYOUT == kLayoutNP ? (static_cast<uint32_t>(n) * G + j) * 4u + c
+                                              : (static_cast<uint32_t>(j) * 4u + c) * n_models + n;
+    if (T::kBytes == 4) return reinterpret_cast<const uint32_t *>(stage)[elem];
+    return reinterpret_cast<const uint16_t *>(stage)[elem];
+}
+
+template <class TA, class TB, int LAYOUT>
+__global__ void __launch_bounds__(544) shuffle_tma_kernel(const __grid_constant__ ShuffleTmaArgs a)
+{
+    extern __shared__ __align__(128) unsigned char smem_raw[];
+    constexpr bool kHasB = TB::kCode != kDtypeNone;
+    // shared memory: [0,256) barriers + abort flag | stages | permutation columns
+    uint64_t *bars = reinterpret_cast<uint64_t *>(smem_raw);
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(smem_raw + 8 * 2 * kMaxStages);
+    unsigned char *stage0 = smem_raw + 256;
+    const int S = a.stages, G = a.G, n_models = a.s.pop.N;
+    const int consumers = G * a.teams;
+    uint8_t *perm_base = stage0 + static_cast<size_t>(S) * a.stage_bytes;
+    const uint32_t full0 = smem_addr(bars), empty0 = smem_addr(bars + kMaxStages);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int warps_per_team = G >> 5;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < S; ++s) {
+            mbar_init(full0 + 8 * s, 1);
+            mbar_init(empty0 + 8 * s, warps_per_team);
+        }
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
+
+    // tiles of this CTA: blockIdx.x, blockIdx.x + gridDim.x, ...
+    const uint32_t my_tiles = blockIdx.x < a.n_tiles ? (a.n_tiles - 1 - blockIdx.x) / gridDim.x + 1 : 0;
+    const uint32_t vec_a = TA::kBytes * 4, vec_b = kHasB ? TB::kBytes * 4 : 0;
+
+    if (warp == 0) {
+        // ---------------- producer ----------------
+        uint32_t issued = 0;
+        for (uint32_t i = 0; i < my_tiles; ++i) {
+            const int s = static_cast<int>(i % S);
+            // lane 0 waits for the stage to be free; the verdict is made warp-uniform
+            int go = 1;
+            if (lane == 0) {
+                if (i >= static_cast<uint32_t>(S)) go = mbar_wait(empty0 + 8 * s, ((i / S) - 1) & 1u, abort_flag, a.s.status) ? 1 : 0;
+                else go = *abort_flag ? 0 : 1;
+            }
+            go = __shfl_sync(0xFFFFFFFFu, go, 0);
+            if (!go) break;
+            const uint64_t tile = blockIdx.x + static_cast<uint64_t>(i) * gridDim.x;
+            const uint64_t g0 = tile * G;
+            const uint32_t groups = static_cast<uint32_t>(min(static_cast<uint64_t>(G), a.s.pop.n_groups - g0));
+            const uint32_t dst = smem_addr(stage0 + static_cast<size_t>(s) * a.stage_bytes);
+            const uint32_t bar = full0 + 8 * s;
+            if (LAYOUT == kLayoutNP) {
+                if (lane == 0) mbar_arrive_expect_tx(bar, groups * (vec_a + vec_b) * n_models);
+                __syncwarp();
+                const int rows = kHasB ? 2 * n_models : n_models;
+                for (int r = lane; r < rows; r += 32) {
+                    if (r < n_models) {
+                        const char *src = static_cast<const char *>(a.s.a) + (static_cast<long long>(r) * a.s.pop.padded_P + 4ll * g0) * TA::kBytes;
+                        bulk_load(dst + r * G * vec_a, src, groups * vec_a, bar);
+                    } else {
+                        const int rb = r - n_models;
+                        const char *src = static_cast<const char *>(a.s.b) + (static_cast<long long>(rb) * a.s.pop.padded_P + 4ll * g0) * TB::kBytes;
+                        bulk_load(dst + a.b_offset + rb * G * vec_b, src, groups * vec_b, bar);
+                    }
+                }
+            } else {
+                if (lane == 0) {
+                    mbar_arrive_expect_tx(bar, groups * (vec_a + vec_b) * n_models);
+                    bulk_load(dst, static_cast<const char *>(a.s.a) + 4ll * g0 * n_models * TA::kBytes, groups * vec_a * n_models, bar);
+                    if (kHasB)
+                        bulk_load(dst + a.b_offset, static_cast<const char *>(a.s.b) + 4ll * g0 * n_models * TB::kBytes, groups * vec_b * n_models, bar);
+                }
+            }
+            __syncwarp();
+            issued = i + 1;
+        }
+        // Do not leave while copies into this CTA's shared memory may be in flight: in
+        // the normal case these phases completed long ago and the checks return at once.
+        if (lane == 0) {
+            const uint32_t first = issued > static_cast<uint32_t>(S) ? issued - S : 0;
+            for (uint32_t i = first; i < issued; ++i) {
+                const uint32_t bar = full0 + 8 * (i % S);
+                const unsigned long long t0 = global_timer_ns();
+                while (!mbar_try_wait(bar, (i / S) & 1u))
+                    if (global_timer_ns() - t0 > kWaitLimitNs) { if (a.s.status) atomicOr(a.s.status, 4u); break; }
+            }
+        }
+        return;
+    }
+
+    // ---------------- consumers ----------------
+    const int ct = threadIdx.x - 32;                 // consumer thread index
+    if (ct >= consumers) return;
+    const int team = ct / G, j = ct - team * G;      // j: group of the tile this thread owns
+    uint8_t *s_perm = perm_base + ct;                // column [n][consumers]
+    uint32_t selected = 0, moved = 0;
+    for (uint32_t i = team; i < my_tiles; i += a.teams) {
+        if (*abort_flag) break;
+        const int s = static_cast<int>(i % S);
+        const uint32_t parity = (i / S) & 1u;
+        const uint32_t full = full0 + 8 * s;
+        const uint64_t tile = blockIdx.x + static_cast<uint64_t>(i) * gridDim.x;
+        const uint64_t g = tile * G + j;
+        uint32_t sel = 0;
+        GroupInfo gi{0, 0, 0, 0};
+        if (g < a.s.pop.n_groups) {
+            gi = find_group(a.s.pop, static_cast<uint32_t>(g), a.s.status);
+            if (gi.thr != 0 && gi.valid != 0) {
+                const Philox4 w = philox4x32_10(gi.cgroup, gi.tensor_id, a.s.step_lo, a.s.step_hi8, a.s.key0, a.s.key1);
+                sel |= (static_cast<uint64_t>(w.x) < gi.thr && gi.valid > 0) ? 1u : 0u;
+                sel |= (static_cast<uint64_t>(w.y) < gi.thr && gi.valid > 1) ? 2u : 0u;
+                sel |= (static_cast<uint64_t>(w.z) < gi.thr && gi.valid > 2) ? 4u : 0u;
+                sel |= (static_cast<uint64_t>(w.w) < gi.thr && gi.valid > 3) ? 8u : 0u;
+            }
+        }
+        if (sel != 0 && mbar_wait(full, parity, abort_flag, a.s.status)) {
+            const unsigned char *stage = stage0 + static_cast<size_t>(s) * a.stage_bytes;
+#pragma unroll 1
+            for (int c = 0; c < 4; ++c) {
+                if (!((sel >> c) & 1u)) continue;
+                draw_permutation_u8(s_perm, consumers, n_models, 4u * gi.cgroup + c, gi.tensor_id, a.s.step_lo, a.s.step_hi8, a.s.key0, a.s.key1);
+                const long long e = 4ll * static_cast<long long>(g) + c;
+                for (int n = 0; n < n_models; ++n) {
+                    const int src = s_perm[n * consumers];
+                    if (src == n) continue;
+                    TA::store_elem(a.s.a, elem_index<LAYOUT>(a.s.pop, n, e), stage_value<TA, LAYOUT>(stage, G, n_models, src, j, c));
+                    if constexpr (kHasB)
+                        TB::store_elem(a.s.b, elem_index<LAYOUT>(a.s.pop, n, e), stage_value<TB, LAYOUT>(stage + a.b_offset, G, n_models, src, j, c));
+                    ++moved;
+                }
+                ++selected;
+            }
+        }
+        __syncwarp();
+        // hand the stage back, but only once its copies have landed
+        if (lane == 0 && mbar_wait(full, parity, abort_flag, a.s.status)) mbar_arrive(empty0 + 8 * s);
+    }
+    if (a.s.stats) {
+        selected = __reduce_add_sync(0xFFFFFFFFu, selected);
+        moved = __reduce_add_sync(0xFFFFFFFFu, moved);
+        if (lane == 0 && selected) {
+            atomicAdd(a.s.stats, static_cast<unsigned long long>(selected));
+            atomicAdd(a.s.stats + 1, static_cast<unsigned long long>(moved));
+        }
+    }
+}
+
+// Picks tile size, stage count and grid for the population and launches.
+template <class TA, class TB>
+cudaError_t launch_shuffle_tma_typed(const ShuffleArgs &args, const LaunchShape &shape, cudaStream_t stream)
+{
+    constexpr bool kHasB = TB::kCode != kDtypeNone;
+    const int N = args.pop.N;
+    const uint32_t group_bytes = static_cast<uint32_t>(N) * (TA::kBytes * 4 + (kHasB ? TB::kBytes * 4 : 0));
+    const size_t budget = 200 * 1024;
+    ShuffleTmaArgs t;
+    t.s = args;
+    int G = 256;
+    if (shape.threads == 128 || shape.threads == 64 || shape.threads == 32) G = shape.threads;
+    while (G > 32 && 3ull * G * group_bytes + static_cast<size_t>(N) * G > budget) G >>= 1;
+    t.G = G;
+    t.teams = G >= 256 ? 1 : (G == 128 ? 2 : 4);
+    if (shape.blocks_per_sm > 0) t.teams = shape.blocks_per_sm;   // tuning: consumer teams per CTA
+    if (t.teams * G > 512) t.teams = 512 / G;
+    t.stage_bytes = static_cast<uint32_t>(G) * group_bytes;
+    t.b_offset = static_cast<uint32_t>(G) * N * TA::kBytes * 4;
+    const size_t perm_bytes = static_cast<size_t>(N) * G * t.teams;
+    int stages = static_cast<int>((budget - perm_bytes) / t.stage_bytes);
+    if (stages > kMaxStages) stages = kMaxStages;
+    if (stages < 2) return cudaErrorInvalidConfiguration;
+    t.stages = stages;
+    t.n_tiles = (args.pop.n_groups + G - 1) / G;
+    const size_t smem = 256 + static_cast<size_t>(stages) * t.stage_bytes + perm_bytes;
+    const int threads = 32 + G * t.teams;
+    auto kernel = args.pop.layout == kLayoutNP ? shuffle_tma_kernel<TA, TB, kLayoutNP> : shuffle_tma_kernel<TA, TB, kLayoutPN>;
+    KernelFit fit;
+    cudaError_t err = kernel_fit(reinterpret_cast<const void *>(kernel), threads, smem, &fit);
+    if (err != cudaSuccess) return err;
+    if (fit.occupancy < 1) return cudaErrorLaunchOutOfResources;
+    uint64_t grid = static_cast<uint64_t>(shape.sm_count > 0 ? shape.sm_count : 148) * fit.occupancy;
+    if (grid > t.n_tiles) grid = t.n_tiles;
+    if (grid == 0) return cudaSuccess;
+    kernel<<<static_cast<unsigned>(grid), threads, smem, stream>>>(t);
+    count_launch();
+    return cudaGetLastError();
+}
+
+inline cudaError_t launch_shuffle_tma(const ShuffleArgs &args, int a_dtype, int b_dtype, const LaunchShape &shape,
+                                      cudaStream_t stream, bool *supported)
+{
+    *supported = true;
+    if (a_dtype == kDtypeF32 && b_dtype == kDtypeNone) return launch_shuffle_tma_typed<F32, NoStack>(args, shape, stream);
+    if (a_dtype == kDtypeBF16 && b_dtype == kDtypeNone) return launch_shuffle_tma_typed<BF16, NoStack>(args, shape, stream);
+    if (a_dtype == kDtypeF32 && b_dtype == kDtypeF32) return launch_shuffle_tma_typed<F32, F32>(args, shape, stream);
+    if (a_dtype == kDtypeBF16 && b_dtype == kDtypeF32) return launch_shuffle_tma_typed<BF16, F32>(args, shape, stream);
+    if (a_dtype == kDtypeBF16 && b_dtype == kDtypeBF16) return launch_shuffle_tma_typed<BF16, BF16>(args, shape, stream);
+    if (a_dtype == kDtypeF32 && b_dtype == kDtypeBF16) return launch_shuffle_tma_typed<F32, BF16>(args, shape, stream);
+    *supported = false;
+    return cudaSuccess;
+}
+
+}  // namespace wash

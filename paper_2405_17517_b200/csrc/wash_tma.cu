@@ -1,0 +1,12 @@
+// Translation unit of the shared-memory-staged (bulk copy) streaming shuffle.
+#include "wash_shuffle_tma.cuh"
+
+namespace wash {
+
+cudaError_t launch_shuffle_staged(const ShuffleArgs &args, int a_dtype, int b_dtype, const LaunchShape &shape,
+                                  cudaStream_t stream, bool *supported)
+{
+    return launch_shuffle_tma(args, a_dtype, b_dtype, shape, stream, supported);
+}
+
+}  // namespace wash
