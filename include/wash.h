@@ -115,10 +115,12 @@ int wash_bind(wash_ctx *ctx, int32_t stack, int32_t dtype, void *dev_ptr, int64_
  * Results are bit-identical across modes. */
 int wash_set_mode(wash_ctx *ctx, int32_t mode);
 
-/* Launch shape override for tuning: threads per block (multiple of 32 in 64..256;
- * 0 = default) and grid style: blocks_per_sm <= 0 (default) launches one group of 4
- * coordinates per thread; blocks_per_sm > 0 launches a persistent grid of SM count x
- * min(blocks_per_sm, resident blocks per SM) blocks that stride over the groups. */
+/* Launch shape override for tuning: threads per block (multiple of 32 in 32..256;
+ * 0 = each kernel's default) and grid style: blocks_per_sm == 0 each kernel's default,
+ * > 0 a persistent grid of SM count x min(blocks_per_sm, resident blocks per SM) blocks
+ * that stride over the groups, < 0 one group of 4 coordinates per thread.  For
+ * WASH_MODE_STREAM_STAGED `threads` is the tile size in groups (32, 64, 128 or 256)
+ * and blocks_per_sm the number of consumer teams per block. */
 int wash_set_launch(wash_ctx *ctx, int32_t threads, int32_t blocks_per_sm);
 
 /* ---- the shuffling step ----------------------------------------------------------- */

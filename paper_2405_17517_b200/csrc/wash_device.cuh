@@ -129,6 +129,9 @@ struct GroupInfo {
     uint64_t thr;
 };
 
+// Describes group g given its segment's table entry (two 16-byte halves).
+__device__ __forceinline__ GroupInfo group_info(uint4 lo, uint4 hi, uint32_t g, uint32_t *status);
+
 __device__ __forceinline__ GroupInfo find_group(const PopView &pop, uint32_t g, uint32_t *status)
 {
     uint32_t s = __ldg(pop.tile_first + (g >> kTileShift));
@@ -136,6 +139,26 @@ __device__ __forceinline__ GroupInfo find_group(const PopView &pop, uint32_t g, 
     while (s < last && g >= __ldg(&pop.seg[s].group_end)) ++s;
     const uint4 lo = __ldg(reinterpret_cast<const uint4 *>(pop.seg + s));       // begin, end, tensor, cgroup_begin
     const uint4 hi = __ldg(reinterpret_cast<const uint4 *>(pop.seg + s) + 1);   // numel, -, thr
+    return group_info(lo, hi, g, status);
+}
+
+// As find_group, for a caller that visits groups in increasing order: `cursor` is the
+// segment of the previous group (or any segment not after g's) and is advanced; `seg`
+// may be a copy of the table in shared memory.
+__device__ __forceinline__ GroupInfo find_group_forward(const SegEntry *seg, int n_seg, uint32_t &cursor, uint32_t g,
+                                                        uint32_t *status)
+{
+    const uint32_t last = static_cast<uint32_t>(n_seg) - 1u;
+    uint32_t s = cursor;
+    while (s < last && g >= seg[s].group_end) ++s;
+    cursor = s;
+    const uint4 lo = reinterpret_cast<const uint4 *>(seg + s)[0];
+    const uint4 hi = reinterpret_cast<const uint4 *>(seg + s)[1];
+    return group_info(lo, hi, g, status);
+}
+
+__device__ __forceinline__ GroupInfo group_info(uint4 lo, uint4 hi, uint32_t g, uint32_t *status)
+{
     GroupInfo gi;
     if (g < lo.x || g >= lo.y) {   // table inconsistent with the row: report, touch nothing
         if (status) atomicOr(status, 1u);

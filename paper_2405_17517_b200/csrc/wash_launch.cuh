@@ -1,7 +1,8 @@
-// Grid sizing for the grid-stride kernels.  By default one work item per thread (the
-// block scheduler then balances the SMs; measured faster than a persistent grid for
-// these short streaming kernels); on request a persistent grid of SM count x blocks
-// per SM.
+// Grid sizing for the grid-stride kernels: either one work item per thread (the block
+// scheduler balances the SMs) or a persistent grid of SM count x resident blocks per SM.
+// Each kernel family states the default that measured faster for it; wash_set_launch
+// overrides (blocks_per_sm > 0: persistent with at most that many blocks per SM,
+// < 0: one item per thread).
 #pragma once
 #include <cstdint>
 #include <map>
@@ -29,8 +30,15 @@ inline cudaError_t kernel_fit(const void *kernel, int threads, size_t smem, Kern
         auto it = cache.find(key);
         if (it != cache.end()) { *fit = it->second; return cudaSuccess; }
     }
-    if (smem > 48 * 1024) {
-        err = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
+    if (smem > 32 * 1024) {   // static shared memory counts against the default 48 KiB too
+        // raise the kernel's limit to the device's opt-in maximum (never lower it: other
+        // launch shapes of the same kernel may already rely on a larger value)
+        int optin = 0;
+        err = cudaDeviceGetAttribute(&optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
+        if (err != cudaSuccess) return err;
+        optin -= 1024;   // room for the kernels' few bytes of static shared memory
+        if (optin < 0 || smem > static_cast<size_t>(optin)) return cudaErrorInvalidConfiguration;
+        err = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, optin);
         if (err != cudaSuccess) return err;
     }
     int occ = 0;
@@ -47,12 +55,18 @@ inline cudaError_t kernel_fit(const void *kernel, int threads, size_t smem, Kern
 
 // Launch `kernel(args)` over n_items work items, one item per thread per loop trip.
 // smem_per_thread bytes of dynamic shared memory are given to every thread.
+struct GridDefault {
+    int threads;        // block size when the caller gave none
+    bool persistent;    // grid style when the caller gave none
+};
+
 template <typename Args>
 cudaError_t launch_grid_stride(void (*kernel)(Args), const Args &args, uint64_t n_items,
-                               size_t smem_per_thread, const LaunchShape &shape, cudaStream_t stream)
+                               size_t smem_per_thread, const LaunchShape &shape, cudaStream_t stream,
+                               GridDefault dflt = GridDefault{256, false})
 {
     if (n_items == 0) return cudaSuccess;
-    int threads = shape.threads > 0 ? shape.threads : 256;
+    int threads = shape.threads > 0 ? shape.threads : dflt.threads;
     if (threads > 256) threads = 256;
     while (smem_per_thread * threads > 96 * 1024 && threads > 64) threads /= 2;
     const size_t smem = smem_per_thread * threads;
@@ -62,9 +76,10 @@ cudaError_t launch_grid_stride(void (*kernel)(Args), const Args &args, uint64_t 
     if (fit.occupancy < 1) return cudaErrorLaunchOutOfResources;
     const uint64_t need = (n_items + threads - 1) / threads;
     uint64_t grid = need;
-    if (shape.blocks_per_sm > 0) {   // persistent grid; otherwise one trip per thread
+    const bool persistent = shape.blocks_per_sm > 0 || (shape.blocks_per_sm == 0 && dflt.persistent);
+    if (persistent) {   // otherwise one trip per thread
         int bps = fit.occupancy;
-        if (shape.blocks_per_sm < bps) bps = shape.blocks_per_sm;
+        if (shape.blocks_per_sm > 0 && shape.blocks_per_sm < bps) bps = shape.blocks_per_sm;
         const uint64_t resident = static_cast<uint64_t>(shape.sm_count > 0 ? shape.sm_count : 148) * bps;
         if (grid > resident) grid = resident;
     }

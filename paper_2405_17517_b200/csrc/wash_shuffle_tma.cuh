@@ -17,7 +17,7 @@
 // size that is a multiple of 16 bytes (rows start on multiples of 8 elements, a group
 // is 16 or 8 bytes, G is a multiple of 32).
 //
-// All waits are bounded: a wait that exceeds kWaitLimitNs sets bit 1 of the status word
+// All waits are bounded: a wait that exceeds kWaitLimitCycles sets bit 1 of the status word
 // and an abort flag that every loop checks; the producer then still waits (bounded) for
 // the copies it has issued before the CTA returns.
 #pragma once
@@ -26,17 +26,18 @@
 
 namespace wash {
 
-constexpr unsigned long long kWaitLimitNs = 2000000000ull;   // 2 s
+constexpr long long kWaitLimitCycles = 4000000000ll;   // about 2 s of SM clock
 constexpr int kMaxStages = 12;
 
 struct ShuffleTmaArgs {
     ShuffleArgs s;
     uint32_t n_tiles;        // ceil(n_groups / G)
     int G;                   // groups per tile = threads per consumer team
-    int teams;               // consumer teams per CTA (tile i of a CTA goes to team i % teams)
+    int teams;               // consumer teams per CTA (tile i of a CTA goes to team i % teams); divides stages
     int stages;
     uint32_t stage_bytes;    // bytes of one stage (both stacks)
     uint32_t b_offset;       // byte offset of the second stack inside a stage
+    uint32_t seg_smem_bytes; // bytes reserved for a shared-memory copy of the segment table (0: read it from global)
 };
 
 __device__ __forceinline__ uint32_t smem_addr(const void *p) { return static_cast<uint32_t>(__cvta_generic_to_shared(p)); }
@@ -60,23 +61,20 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
                  : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
     return ok != 0;
 }
-__device__ __forceinline__ unsigned long long global_timer_ns()
-{
-    unsigned long long t;
-    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
-    return t;
-}
 // Waits for the phase of parity `parity` to complete.  Returns false if the CTA is
 // aborting or the wait ran out of time (then it sets the abort flag and the status bit).
+// Time is measured with the SM's cycle counter, read only every 1024 polls.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag, uint32_t *status)
 {
     if (mbar_try_wait(bar, parity)) return true;
-    const unsigned long long t0 = global_timer_ns();
+    long long t0 = 0;
     for (uint32_t polls = 1;; ++polls) {
         if (mbar_try_wait(bar, parity)) return true;
-        if ((polls & 255u) == 0) {
+        if ((polls & 1023u) == 0) {
             if (*abort_flag) return false;
-            if (global_timer_ns() - t0 > kWaitLimitNs) {
+            const long long now = clock64();
+            if (t0 == 0) t0 = now;
+            if (now - t0 > kWaitLimitCycles) {
                 *abort_flag = 1;
                 if (status) atomicOr(status, 2u);
                 return false;
@@ -131,6 +129,14 @@ __global__ void __launch_bounds__(544) shuffle_tma_kernel(const __grid_constant_
     const int S = a.stages, G = a.G, n_models = a.s.pop.N;
     const int consumers = G * a.teams;
     uint8_t *perm_base = stage0 + static_cast<size_t>(S) * a.stage_bytes;
+    // optional copy of the segment table, so that the lookup costs no global round trip
+    const SegEntry *seg = a.s.pop.seg;
+    if (a.seg_smem_bytes) {
+        uint4 *dst = reinterpret_cast<uint4 *>(perm_base + ((static_cast<size_t>(n_models) * consumers + 15) & ~static_cast<size_t>(15)));
+        const uint4 *src = reinterpret_cast<const uint4 *>(a.s.pop.seg);
+        for (int k = threadIdx.x; k < a.s.pop.n_seg * 2; k += blockDim.x) dst[k] = __ldg(src + k);
+        seg = reinterpret_cast<const SegEntry *>(dst);
+    }
     const uint32_t full0 = smem_addr(bars), empty0 = smem_addr(bars + kMaxStages);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int warps_per_team = G >> 5;
@@ -198,9 +204,9 @@ __global__ void __launch_bounds__(544) shuffle_tma_kernel(const __grid_constant_
             const uint32_t first = issued > static_cast<uint32_t>(S) ? issued - S : 0;
             for (uint32_t i = first; i < issued; ++i) {
                 const uint32_t bar = full0 + 8 * (i % S);
-                const unsigned long long t0 = global_timer_ns();
+                const long long t0 = clock64();
                 while (!mbar_try_wait(bar, (i / S) & 1u))
-                    if (global_timer_ns() - t0 > kWaitLimitNs) { if (a.s.status) atomicOr(a.s.status, 4u); break; }
+                    if (clock64() - t0 > kWaitLimitCycles) { if (a.s.status) atomicOr(a.s.status, 4u); break; }
             }
         }
         return;
@@ -212,6 +218,12 @@ __global__ void __launch_bounds__(544) shuffle_tma_kernel(const __grid_constant_
     const int team = ct / G, j = ct - team * G;      // j: group of the tile this thread owns
     uint8_t *s_perm = perm_base + ct;                // column [n][consumers]
     uint32_t selected = 0, moved = 0;
+    // this thread's groups come in increasing order: the segment cursor only moves forward
+    uint32_t cursor = 0;
+    {
+        const uint64_t g_first = (blockIdx.x + static_cast<uint64_t>(team) * gridDim.x) * G + j;
+        if (static_cast<uint32_t>(team) < my_tiles && g_first < a.s.pop.n_groups) cursor = __ldg(a.s.pop.tile_first + (g_first >> kTileShift));
+    }
     for (uint32_t i = team; i < my_tiles; i += a.teams) {
         if (*abort_flag) break;
         const int s = static_cast<int>(i % S);
@@ -222,7 +234,7 @@ __global__ void __launch_bounds__(544) shuffle_tma_kernel(const __grid_constant_
         uint32_t sel = 0;
         GroupInfo gi{0, 0, 0, 0};
         if (g < a.s.pop.n_groups) {
-            gi = find_group(a.s.pop, static_cast<uint32_t>(g), a.s.status);
+            gi = find_group_forward(seg, a.s.pop.n_seg, cursor, static_cast<uint32_t>(g), a.s.status);
             if (gi.thr != 0 && gi.valid != 0) {
                 const Philox4 w = philox4x32_10(gi.cgroup, gi.tensor_id, a.s.step_lo, a.s.step_hi8, a.s.key0, a.s.key1);
                 sel |= (static_cast<uint64_t>(w.x) < gi.thr && gi.valid > 0) ? 1u : 0u;
@@ -250,8 +262,12 @@ __global__ void __launch_bounds__(544) shuffle_tma_kernel(const __grid_constant_
             }
         }
         __syncwarp();
-        // hand the stage back, but only once its copies have landed
+        // Hand the stage back, but only once its copies have landed.  The second
+        // __syncwarp keeps the other lanes from running ahead of lane 0: a lane that
+        // reached this stage's next phase while the barrier was still in the current one
+        // would see its parity test pass at once and read the old tile.
         if (lane == 0 && mbar_wait(full, parity, abort_flag, a.s.status)) mbar_arrive(empty0 + 8 * s);
+        __syncwarp();
     }
     if (a.s.stats) {
         selected = __reduce_add_sync(0xFFFFFFFFu, selected);
@@ -277,18 +293,24 @@ cudaError_t launch_shuffle_tma_typed(const ShuffleArgs &args, const LaunchShape 
     if (shape.threads == 128 || shape.threads == 64 || shape.threads == 32) G = shape.threads;
     while (G > 32 && 3ull * G * group_bytes + static_cast<size_t>(N) * G > budget) G >>= 1;
     t.G = G;
-    t.teams = G >= 256 ? 1 : (G == 128 ? 2 : 4);
+    t.teams = G >= 256 ? 2 : (G == 128 ? 4 : 8);
     if (shape.blocks_per_sm > 0) t.teams = shape.blocks_per_sm;   // tuning: consumer teams per CTA
     if (t.teams * G > 512) t.teams = 512 / G;
     t.stage_bytes = static_cast<uint32_t>(G) * group_bytes;
     t.b_offset = static_cast<uint32_t>(G) * N * TA::kBytes * 4;
-    const size_t perm_bytes = static_cast<size_t>(N) * G * t.teams;
-    int stages = static_cast<int>((budget - perm_bytes) / t.stage_bytes);
+    const size_t perm_bytes = (static_cast<size_t>(N) * G * t.teams + 15) & ~static_cast<size_t>(15);   // sized for the most teams considered
+    const size_t seg_bytes = sizeof(SegEntry) * static_cast<size_t>(args.pop.n_seg);
+    t.seg_smem_bytes = seg_bytes <= 16 * 1024 ? static_cast<uint32_t>(seg_bytes) : 0;
+    int stages = static_cast<int>((budget - perm_bytes - t.seg_smem_bytes) / t.stage_bytes);
     if (stages > kMaxStages) stages = kMaxStages;
+    // A stage must always be consumed by the same team: a waiter may only wait for the
+    // phase that follows the one it saw last, so it has to see every phase of its stages.
+    while (t.teams > 1 && stages / t.teams * t.teams < 2) t.teams >>= 1;
+    stages = stages / t.teams * t.teams;
     if (stages < 2) return cudaErrorInvalidConfiguration;
     t.stages = stages;
     t.n_tiles = (args.pop.n_groups + G - 1) / G;
-    const size_t smem = 256 + static_cast<size_t>(stages) * t.stage_bytes + perm_bytes;
+    const size_t smem = 256 + static_cast<size_t>(stages) * t.stage_bytes + perm_bytes + t.seg_smem_bytes;
     const int threads = 32 + G * t.teams;
     auto kernel = args.pop.layout == kLayoutNP ? shuffle_tma_kernel<TA, TB, kLayoutNP> : shuffle_tma_kernel<TA, TB, kLayoutPN>;
     KernelFit fit;
