@@ -3,8 +3,8 @@
 //
 // Why: the register-resident kernel keeps N (or 2N) vectors per thread in flight and is
 // limited by how many such threads fit on an SM (measured: 24 warps, ~120 KB in flight
-// per SM, 85 % of the bandwidth a pure read reaches).  Here one producer warp per CTA
-// streams tiles of the stack into a ring of shared-memory stages with bulk asynchronous
+// per SM, 85 % of the bandwidth a pure read reaches).  Here the producer warps of a CTA
+// stream tiles of the stack into a ring of shared-memory stages with bulk asynchronous
 // copies that complete on mbarriers; ~200 KB per SM are in flight with no register
 // cost, and the consumer warps spend their time on the Philox mask, which needs no data
 // at all.  A consumer touches a stage only for a selected coordinate (it then reads the
@@ -28,6 +28,8 @@ namespace wash {
 
 constexpr long long kWaitLimitCycles = 4000000000ll;   // about 2 s of SM clock
 constexpr int kMaxStages = 12;
+constexpr int kProducerWarps = 4;
+constexpr int kPieceBytes = 4096;   // largest single bulk copy
 
 struct ShuffleTmaArgs {
     ShuffleArgs s;
@@ -50,9 +52,9 @@ __device__ __forceinline__ void mbar_arrive(uint32_t bar)
 {
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
-__device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes)
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes)
 {
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+    asm volatile("mbarrier.expect_tx.relaxed.cta.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
 }
 __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
 {
@@ -118,7 +120,7 @@ __device__ __forceinline__ uint32_t stage_value(const unsigned char *stage, int 
 }
 
 template <class TA, class TB, int LAYOUT>
-__global__ void __launch_bounds__(544) shuffle_tma_kernel(const __grid_constant__ ShuffleTmaArgs a)
+__global__ void __launch_bounds__(32 * kProducerWarps + 512) shuffle_tma_kernel(const __grid_constant__ ShuffleTmaArgs a)
 {
     extern __shared__ __align__(128) unsigned char smem_raw[];
     constexpr bool kHasB = TB::kCode != kDtypeNone;
@@ -143,7 +145,7 @@ __global__ void __launch_bounds__(544) shuffle_tma_kernel(const __grid_constant_
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < S; ++s) {
-            mbar_init(full0 + 8 * s, 1);
+            mbar_init(full0 + 8 * s, kProducerWarps);
             mbar_init(empty0 + 8 * s, warps_per_team);
         }
         *abort_flag = 0;
@@ -155,8 +157,17 @@ __global__ void __launch_bounds__(544) shuffle_tma_kernel(const __grid_constant_
     const uint32_t my_tiles = blockIdx.x < a.n_tiles ? (a.n_tiles - 1 - blockIdx.x) / gridDim.x + 1 : 0;
     const uint32_t vec_a = TA::kBytes * 4, vec_b = kHasB ? TB::kBytes * 4 : 0;
 
-    if (warp == 0) {
-        // ---------------- producer ----------------
+    if (warp < kProducerWarps) {
+        // ---------------- producers ----------------
+        // A tile is a list of contiguous regions ([N][P]: one per model row and stack;
+        // [P][N]: one per stack), cut into pieces of at most kPieceBytes.  Piece q goes to
+        // producer thread q: each bulk copy occupies its issuing warp for some tens of
+        // nanoseconds, so the pieces are spread over several warps.  A thread announces
+        // its bytes (expect_tx) before it issues its copy; lane 0 of every producer warp
+        // then arrives, so a stage's "full" barrier counts kProducerWarps arrivals.
+        const int regions_a = LAYOUT == kLayoutNP ? n_models : 1;
+        const int regions_b = kHasB ? regions_a : 0;
+        const int pt = threadIdx.x;                      // producer thread index, 0 .. 32*kProducerWarps-1
         uint32_t issued = 0;
         for (uint32_t i = 0; i < my_tiles; ++i) {
             const int s = static_cast<int>(i % S);
@@ -173,29 +184,29 @@ __global__ void __launch_bounds__(544) shuffle_tma_kernel(const __grid_constant_
             const uint32_t groups = static_cast<uint32_t>(min(static_cast<uint64_t>(G), a.s.pop.n_groups - g0));
             const uint32_t dst = smem_addr(stage0 + static_cast<size_t>(s) * a.stage_bytes);
             const uint32_t bar = full0 + 8 * s;
-            if (LAYOUT == kLayoutNP) {
-                if (lane == 0) mbar_arrive_expect_tx(bar, groups * (vec_a + vec_b) * n_models);
-                __syncwarp();
-                const int rows = kHasB ? 2 * n_models : n_models;
-                for (int r = lane; r < rows; r += 32) {
-                    if (r < n_models) {
-                        const char *src = static_cast<const char *>(a.s.a) + (static_cast<long long>(r) * a.s.pop.padded_P + 4ll * g0) * TA::kBytes;
-                        bulk_load(dst + r * G * vec_a, src, groups * vec_a, bar);
-                    } else {
-                        const int rb = r - n_models;
-                        const char *src = static_cast<const char *>(a.s.b) + (static_cast<long long>(rb) * a.s.pop.padded_P + 4ll * g0) * TB::kBytes;
-                        bulk_load(dst + a.b_offset + rb * G * vec_b, src, groups * vec_b, bar);
-                    }
-                }
-            } else {
-                if (lane == 0) {
-                    mbar_arrive_expect_tx(bar, groups * (vec_a + vec_b) * n_models);
-                    bulk_load(dst, static_cast<const char *>(a.s.a) + 4ll * g0 * n_models * TA::kBytes, groups * vec_a * n_models, bar);
-                    if (kHasB)
-                        bulk_load(dst + a.b_offset, static_cast<const char *>(a.s.b) + 4ll * g0 * n_models * TB::kBytes, groups * vec_b * n_models, bar);
-                }
+            // bytes of one region of each stack, and how many pieces that makes
+            const uint32_t bytes_a = groups * vec_a * (LAYOUT == kLayoutNP ? 1 : n_models);
+            const uint32_t bytes_b = groups * vec_b * (LAYOUT == kLayoutNP ? 1 : n_models);
+            const uint32_t pieces_a = (bytes_a + kPieceBytes - 1) / kPieceBytes;
+            const uint32_t pieces_b = kHasB ? (bytes_b + kPieceBytes - 1) / kPieceBytes : 0;
+            const uint32_t total = regions_a * pieces_a + regions_b * pieces_b;
+            for (uint32_t q = pt; q < total; q += 32 * kProducerWarps) {
+                const bool in_a = q < regions_a * pieces_a;
+                const uint32_t qq = in_a ? q : q - regions_a * pieces_a;
+                const uint32_t per = in_a ? pieces_a : pieces_b;
+                const uint32_t region = qq / per, off = (qq - region * per) * kPieceBytes;
+                const uint32_t bytes = min(static_cast<uint32_t>(kPieceBytes), (in_a ? bytes_a : bytes_b) - off);
+                const int eb = in_a ? TA::kBytes : (kHasB ? TB::kBytes : 1);
+                // first element of the region in the stack, and its place in the stage
+                const long long elem0 = LAYOUT == kLayoutNP ? static_cast<long long>(region) * a.s.pop.padded_P + 4ll * g0
+                                                            : 4ll * g0 * n_models;
+                const char *src = static_cast<const char *>(in_a ? a.s.a : a.s.b) + elem0 * eb + off;
+                const uint32_t region_dst = (in_a ? 0u : a.b_offset) + (LAYOUT == kLayoutNP ? region * G * (in_a ? vec_a : vec_b) : 0u);
+                mbar_expect_tx(bar, bytes);
+                bulk_load(dst + region_dst + off, src, bytes, bar);
             }
             __syncwarp();
+            if (lane == 0) mbar_arrive(bar);
             issued = i + 1;
         }
         // Do not leave while copies into this CTA's shared memory may be in flight: in
@@ -213,7 +224,7 @@ __global__ void __launch_bounds__(544) shuffle_tma_kernel(const __grid_constant_
     }
 
     // ---------------- consumers ----------------
-    const int ct = threadIdx.x - 32;                 // consumer thread index
+    const int ct = threadIdx.x - 32 * kProducerWarps;   // consumer thread index
     if (ct >= consumers) return;
     const int team = ct / G, j = ct - team * G;      // j: group of the tile this thread owns
     uint8_t *s_perm = perm_base + ct;                // column [n][consumers]
@@ -311,7 +322,7 @@ cudaError_t launch_shuffle_tma_typed(const ShuffleArgs &args, const LaunchShape 
     t.stages = stages;
     t.n_tiles = (args.pop.n_groups + G - 1) / G;
     const size_t smem = 256 + static_cast<size_t>(stages) * t.stage_bytes + perm_bytes + t.seg_smem_bytes;
-    const int threads = 32 + G * t.teams;
+    const int threads = 32 * kProducerWarps + G * t.teams;
     auto kernel = args.pop.layout == kLayoutNP ? shuffle_tma_kernel<TA, TB, kLayoutNP> : shuffle_tma_kernel<TA, TB, kLayoutPN>;
     KernelFit fit;
     cudaError_t err = kernel_fit(reinterpret_cast<const void *>(kernel), threads, smem, &fit);
