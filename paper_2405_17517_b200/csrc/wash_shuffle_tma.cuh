@@ -8,8 +8,10 @@
 // copies that complete on mbarriers; ~200 KB per SM are in flight with no register
 // cost, and the consumer warps spend their time on the Philox mask, which needs no data
 // at all.  A consumer touches a stage only for a selected coordinate (it then reads the
-// N values from shared memory and writes the moved ones to global memory) and to hand
-// the stage back.  N is a run-time value: one instantiation serves every population size.
+// N values from shared memory and writes the moved ones to global memory); a warp hands
+// a stage back as soon as it has drawn the tile's mask and served its selected lanes,
+// whether or not the tile has landed -- the producers wait for the landing themselves
+// before they reuse the stage.  N is a run-time value: one instantiation serves every population size.
 //
 // Tile = G consecutive groups (G = threads of one consumer team).  [N][P]: one bulk copy
 // per model row and stack (G*16 bytes of fp32).  [P][N]: the tile's G*4N elements are
@@ -28,6 +30,7 @@ namespace wash {
 
 constexpr long long kWaitLimitCycles = 4000000000ll;   // about 2 s of SM clock
 constexpr int kMaxStages = 12;
+constexpr int kHeaderBytes = 512;   // three barriers per stage and the abort flag
 constexpr int kProducerWarps = 4;
 constexpr int kPieceBytes = 4096;   // largest single bulk copy
 
@@ -120,14 +123,14 @@ __device__ __forceinline__ uint32_t stage_value(const unsigned char *stage, int 
 }
 
 template <class TA, class TB, int LAYOUT>
-__global__ void __launch_bounds__(32 * kProducerWarps + 512) shuffle_tma_kernel(const __grid_constant__ ShuffleTmaArgs a)
+__global__ void __launch_bounds__(32 * kProducerWarps + 512, 1) shuffle_tma_kernel(const __grid_constant__ ShuffleTmaArgs a)
 {
     extern __shared__ __align__(128) unsigned char smem_raw[];
     constexpr bool kHasB = TB::kCode != kDtypeNone;
-    // shared memory: [0,256) barriers + abort flag | stages | permutation columns
+    // shared memory: [0,512) barriers + abort flag | stages | permutation columns | segment table
     uint64_t *bars = reinterpret_cast<uint64_t *>(smem_raw);
-    volatile int *abort_flag = reinterpret_cast<volatile int *>(smem_raw + 8 * 2 * kMaxStages);
-    unsigned char *stage0 = smem_raw + 256;
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(smem_raw + 8 * 3 * kMaxStages);
+    unsigned char *stage0 = smem_raw + kHeaderBytes;
     const int S = a.stages, G = a.G, n_models = a.s.pop.N;
     const int consumers = G * a.teams;
     uint8_t *perm_base = stage0 + static_cast<size_t>(S) * a.stage_bytes;
@@ -139,7 +142,9 @@ __global__ void __launch_bounds__(32 * kProducerWarps + 512) shuffle_tma_kernel(
         for (int k = threadIdx.x; k < a.s.pop.n_seg * 2; k += blockDim.x) dst[k] = __ldg(src + k);
         seg = reinterpret_cast<const SegEntry *>(dst);
     }
-    const uint32_t full0 = smem_addr(bars), empty0 = smem_addr(bars + kMaxStages);
+    // per stage: full (the tile's bytes have landed), empty (every consumer warp has let go of
+    // the stage), issued (the producers have started the tile's copies)
+    const uint32_t full0 = smem_addr(bars), empty0 = smem_addr(bars + kMaxStages), issued0 = smem_addr(bars + 2 * kMaxStages);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int warps_per_team = G >> 5;
 
@@ -147,6 +152,7 @@ __global__ void __launch_bounds__(32 * kProducerWarps + 512) shuffle_tma_kernel(
         for (int s = 0; s < S; ++s) {
             mbar_init(full0 + 8 * s, kProducerWarps);
             mbar_init(empty0 + 8 * s, warps_per_team);
+            mbar_init(issued0 + 8 * s, kProducerWarps);
         }
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -161,20 +167,23 @@ __global__ void __launch_bounds__(32 * kProducerWarps + 512) shuffle_tma_kernel(
         // ---------------- producers ----------------
         // A tile is a list of contiguous regions ([N][P]: one per model row and stack;
         // [P][N]: one per stack), cut into pieces of at most kPieceBytes.  Piece q goes to
-        // producer thread q: each bulk copy occupies its issuing warp for some tens of
+        // a producer thread, warps taking turns: each bulk copy occupies its issuing warp for some tens of
         // nanoseconds, so the pieces are spread over several warps.  A thread announces
         // its bytes (expect_tx) before it issues its copy; lane 0 of every producer warp
         // then arrives, so a stage's "full" barrier counts kProducerWarps arrivals.
         const int regions_a = LAYOUT == kLayoutNP ? n_models : 1;
         const int regions_b = kHasB ? regions_a : 0;
-        const int pt = threadIdx.x;                      // producer thread index, 0 .. 32*kProducerWarps-1
         uint32_t issued = 0;
         for (uint32_t i = 0; i < my_tiles; ++i) {
             const int s = static_cast<int>(i % S);
             // lane 0 waits for the stage to be free; the verdict is made warp-uniform
+            // (the stage's previous tile must have landed, so that the barrier's byte count
+            // is settled, and every consumer warp must have let go of it)
             int go = 1;
             if (lane == 0) {
-                if (i >= static_cast<uint32_t>(S)) go = mbar_wait(empty0 + 8 * s, ((i / S) - 1) & 1u, abort_flag, a.s.status) ? 1 : 0;
+                if (i >= static_cast<uint32_t>(S))
+                    go = (mbar_wait(full0 + 8 * s, ((i / S) - 1) & 1u, abort_flag, a.s.status) &&
+                          mbar_wait(empty0 + 8 * s, ((i / S) - 1) & 1u, abort_flag, a.s.status)) ? 1 : 0;
                 else go = *abort_flag ? 0 : 1;
             }
             go = __shfl_sync(0xFFFFFFFFu, go, 0);
@@ -190,7 +199,7 @@ __global__ void __launch_bounds__(32 * kProducerWarps + 512) shuffle_tma_kernel(
             const uint32_t pieces_a = (bytes_a + kPieceBytes - 1) / kPieceBytes;
             const uint32_t pieces_b = kHasB ? (bytes_b + kPieceBytes - 1) / kPieceBytes : 0;
             const uint32_t total = regions_a * pieces_a + regions_b * pieces_b;
-            for (uint32_t q = pt; q < total; q += 32 * kProducerWarps) {
+            for (uint32_t q = lane * kProducerWarps + warp; q < total; q += 32 * kProducerWarps) {   // neighbouring pieces go to different warps
                 const bool in_a = q < regions_a * pieces_a;
                 const uint32_t qq = in_a ? q : q - regions_a * pieces_a;
                 const uint32_t per = in_a ? pieces_a : pieces_b;
@@ -206,7 +215,10 @@ __global__ void __launch_bounds__(32 * kProducerWarps + 512) shuffle_tma_kernel(
                 bulk_load(dst + region_dst + off, src, bytes, bar);
             }
             __syncwarp();
-            if (lane == 0) mbar_arrive(bar);
+            if (lane == 0) {
+                mbar_arrive(bar);
+                mbar_arrive(issued0 + 8 * s);
+            }
             issued = i + 1;
         }
         // Do not leave while copies into this CTA's shared memory may be in flight: in
@@ -254,7 +266,12 @@ __global__ void __launch_bounds__(32 * kProducerWarps + 512) shuffle_tma_kernel(
                 sel |= (static_cast<uint64_t>(w.w) < gi.thr && gi.valid > 3) ? 8u : 0u;
             }
         }
-        if (sel != 0 && mbar_wait(full, parity, abort_flag, a.s.status)) {
+        // Only a thread with a selected coordinate needs the tile's data.  It first makes
+        // sure the stage's previous phase is over (its warp may have released that tile
+        // before it had landed), then waits for this tile's phase.
+        const uint32_t k = i / S;
+        if (sel != 0 && (k == 0 || mbar_wait(full, parity ^ 1u, abort_flag, a.s.status)) &&
+            mbar_wait(full, parity, abort_flag, a.s.status)) {
             const unsigned char *stage = stage0 + static_cast<size_t>(s) * a.stage_bytes;
 #pragma unroll 1
             for (int c = 0; c < 4; ++c) {
@@ -273,11 +290,17 @@ __global__ void __launch_bounds__(32 * kProducerWarps + 512) shuffle_tma_kernel(
             }
         }
         __syncwarp();
-        // Hand the stage back, but only once its copies have landed.  The second
-        // __syncwarp keeps the other lanes from running ahead of lane 0: a lane that
-        // reached this stage's next phase while the barrier was still in the current one
-        // would see its parity test pass at once and read the old tile.
-        if (lane == 0 && mbar_wait(full, parity, abort_flag, a.s.status)) mbar_arrive(empty0 + 8 * s);
+        // Release the stage for this tile.  An arrival counts toward the barrier's current
+        // phase, so the previous phase (every warp's release of the stage's previous tile)
+        // has to be over first.  The warp does not wait for the tile's data: a stage whose
+        // tile nobody needs is handed back before it has even landed, and the producers
+        // check the landing themselves.
+        // Nor may the consumers get more than one phase ahead of the producers (a parity wait
+        // can only tell two neighbouring phases apart): the release also waits until the
+        // producers have issued this tile, which they do long before it lands.
+        if (lane == 0 && (k == 0 || mbar_wait(empty0 + 8 * s, parity ^ 1u, abort_flag, a.s.status)) &&
+            mbar_wait(issued0 + 8 * s, parity, abort_flag, a.s.status))
+            mbar_arrive(empty0 + 8 * s);
         __syncwarp();
     }
     if (a.s.stats) {
@@ -321,7 +344,7 @@ cudaError_t launch_shuffle_tma_typed(const ShuffleArgs &args, const LaunchShape 
     if (stages < 2) return cudaErrorInvalidConfiguration;
     t.stages = stages;
     t.n_tiles = (args.pop.n_groups + G - 1) / G;
-    const size_t smem = 256 + static_cast<size_t>(stages) * t.stage_bytes + perm_bytes + t.seg_smem_bytes;
+    const size_t smem = kHeaderBytes + static_cast<size_t>(stages) * t.stage_bytes + perm_bytes + t.seg_smem_bytes;
     const int threads = 32 * kProducerWarps + G * t.teams;
     auto kernel = args.pop.layout == kLayoutNP ? shuffle_tma_kernel<TA, TB, kLayoutNP> : shuffle_tma_kernel<TA, TB, kLayoutPN>;
     KernelFit fit;
