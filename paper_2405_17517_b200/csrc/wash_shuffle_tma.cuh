@@ -55,9 +55,9 @@ __device__ __forceinline__ void mbar_arrive(uint32_t bar)
 {
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes)
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes)
 {
-    asm volatile("mbarrier.expect_tx.relaxed.cta.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
 }
 __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
 {
@@ -69,7 +69,7 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
 // Waits for the phase of parity `parity` to complete.  Returns false if the CTA is
 // aborting or the wait ran out of time (then it sets the abort flag and the status bit).
 // Time is measured with the SM's cycle counter, read only every 1024 polls.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag, uint32_t *status)
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag, uint32_t *status, uint32_t site = 0)
 {
     if (mbar_try_wait(bar, parity)) return true;
     long long t0 = 0;
@@ -81,7 +81,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
             if (t0 == 0) t0 = now;
             if (now - t0 > kWaitLimitCycles) {
                 *abort_flag = 1;
-                if (status) atomicOr(status, 2u);
+                if (status) atomicOr(status, 2u | site);
                 return false;
             }
         }
@@ -168,9 +168,9 @@ __global__ void __launch_bounds__(32 * kProducerWarps + 512, 1) shuffle_tma_kern
         // A tile is a list of contiguous regions ([N][P]: one per model row and stack;
         // [P][N]: one per stack), cut into pieces of at most kPieceBytes.  Piece q goes to
         // a producer thread, warps taking turns: each bulk copy occupies its issuing warp for some tens of
-        // nanoseconds, so the pieces are spread over several warps.  A thread announces
-        // its bytes (expect_tx) before it issues its copy; lane 0 of every producer warp
-        // then arrives, so a stage's "full" barrier counts kProducerWarps arrivals.
+        // nanoseconds, so the pieces are spread over several warps.  Lane 0 of every producer
+        // warp announces the warp's bytes with its arrival (arrive.expect_tx) before the
+        // warp issues its copies, so a stage's "full" barrier counts kProducerWarps arrivals.
         const int regions_a = LAYOUT == kLayoutNP ? n_models : 1;
         const int regions_b = kHasB ? regions_a : 0;
         uint32_t issued = 0;
@@ -182,8 +182,8 @@ __global__ void __launch_bounds__(32 * kProducerWarps + 512, 1) shuffle_tma_kern
             int go = 1;
             if (lane == 0) {
                 if (i >= static_cast<uint32_t>(S))
-                    go = (mbar_wait(full0 + 8 * s, ((i / S) - 1) & 1u, abort_flag, a.s.status) &&
-                          mbar_wait(empty0 + 8 * s, ((i / S) - 1) & 1u, abort_flag, a.s.status)) ? 1 : 0;
+                    go = (mbar_wait(full0 + 8 * s, ((i / S) - 1) & 1u, abort_flag, a.s.status, 16u) &&
+                          mbar_wait(empty0 + 8 * s, ((i / S) - 1) & 1u, abort_flag, a.s.status, 32u)) ? 1 : 0;
                 else go = *abort_flag ? 0 : 1;
             }
             go = __shfl_sync(0xFFFFFFFFu, go, 0);
@@ -199,6 +199,18 @@ __global__ void __launch_bounds__(32 * kProducerWarps + 512, 1) shuffle_tma_kern
             const uint32_t pieces_a = (bytes_a + kPieceBytes - 1) / kPieceBytes;
             const uint32_t pieces_b = kHasB ? (bytes_b + kPieceBytes - 1) / kPieceBytes : 0;
             const uint32_t total = regions_a * pieces_a + regions_b * pieces_b;
+            // this warp's share of the bytes, announced by lane 0 together with its arrival
+            uint32_t my_bytes = 0;
+            for (uint32_t q = lane * kProducerWarps + warp; q < total; q += 32 * kProducerWarps) {
+                const bool in_a = q < regions_a * pieces_a;
+                const uint32_t qq = in_a ? q : q - regions_a * pieces_a;
+                const uint32_t per = in_a ? pieces_a : pieces_b;
+                const uint32_t off = (qq % per) * kPieceBytes;
+                my_bytes += min(static_cast<uint32_t>(kPieceBytes), (in_a ? bytes_a : bytes_b) - off);
+            }
+            my_bytes = __reduce_add_sync(0xFFFFFFFFu, my_bytes);
+            if (lane == 0) mbar_arrive_expect_tx(bar, my_bytes);
+            __syncwarp();
             for (uint32_t q = lane * kProducerWarps + warp; q < total; q += 32 * kProducerWarps) {   // neighbouring pieces go to different warps
                 const bool in_a = q < regions_a * pieces_a;
                 const uint32_t qq = in_a ? q : q - regions_a * pieces_a;
@@ -211,14 +223,10 @@ __global__ void __launch_bounds__(32 * kProducerWarps + 512, 1) shuffle_tma_kern
                                                             : 4ll * g0 * n_models;
                 const char *src = static_cast<const char *>(in_a ? a.s.a : a.s.b) + elem0 * eb + off;
                 const uint32_t region_dst = (in_a ? 0u : a.b_offset) + (LAYOUT == kLayoutNP ? region * G * (in_a ? vec_a : vec_b) : 0u);
-                mbar_expect_tx(bar, bytes);
                 bulk_load(dst + region_dst + off, src, bytes, bar);
             }
             __syncwarp();
-            if (lane == 0) {
-                mbar_arrive(bar);
-                mbar_arrive(issued0 + 8 * s);
-            }
+            if (lane == 0) mbar_arrive(issued0 + 8 * s);
             issued = i + 1;
         }
         // Do not leave while copies into this CTA's shared memory may be in flight: in
@@ -266,12 +274,14 @@ __global__ void __launch_bounds__(32 * kProducerWarps + 512, 1) shuffle_tma_kern
                 sel |= (static_cast<uint64_t>(w.w) < gi.thr && gi.valid > 3) ? 8u : 0u;
             }
         }
-        // Only a thread with a selected coordinate needs the tile's data.  It first makes
-        // sure the stage's previous phase is over (its warp may have released that tile
-        // before it had landed), then waits for this tile's phase.
+        // Only a thread with a selected coordinate needs the tile's data.  Its warp may have
+        // released the stage's previous tile before that tile had landed, and a parity wait
+        // cannot tell "previous phase still open" from "this phase already over".  So it
+        // first waits until the producers have issued this tile -- which they only do once
+        // the previous one has landed -- and then for this tile's bytes.
         const uint32_t k = i / S;
-        if (sel != 0 && (k == 0 || mbar_wait(full, parity ^ 1u, abort_flag, a.s.status)) &&
-            mbar_wait(full, parity, abort_flag, a.s.status)) {
+        if (sel != 0 && mbar_wait(issued0 + 8 * s, parity, abort_flag, a.s.status, 64u) &&
+            mbar_wait(full, parity, abort_flag, a.s.status, 128u)) {
             const unsigned char *stage = stage0 + static_cast<size_t>(s) * a.stage_bytes;
 #pragma unroll 1
             for (int c = 0; c < 4; ++c) {
@@ -298,8 +308,8 @@ __global__ void __launch_bounds__(32 * kProducerWarps + 512, 1) shuffle_tma_kern
         // Nor may the consumers get more than one phase ahead of the producers (a parity wait
         // can only tell two neighbouring phases apart): the release also waits until the
         // producers have issued this tile, which they do long before it lands.
-        if (lane == 0 && (k == 0 || mbar_wait(empty0 + 8 * s, parity ^ 1u, abort_flag, a.s.status)) &&
-            mbar_wait(issued0 + 8 * s, parity, abort_flag, a.s.status))
+        if (lane == 0 && (k == 0 || mbar_wait(empty0 + 8 * s, parity ^ 1u, abort_flag, a.s.status, 256u)) &&
+            mbar_wait(issued0 + 8 * s, parity, abort_flag, a.s.status, 512u))
             mbar_arrive(empty0 + 8 * s);
         __syncwarp();
     }
