@@ -3,7 +3,10 @@
 //
 // Why: the register-resident kernel keeps N (or 2N) vectors per thread in flight and is
 // limited by how many such threads fit on an SM (measured: 24 warps, ~120 KB in flight
-// per SM, 85 % of the bandwidth a pure read reaches).  Here the producer warps of a CTA
+// per SM, 85 % of the bandwidth a pure read reaches).  Measured outcome on B200: every
+// 1-D bulk copy costs its CTA about 85 ns whatever its size, so with rows of a few KiB
+// this kernel reaches 76-80 % of the measured copy bandwidth on the ResNet populations
+// and does not beat the register kernel (83-92 %); it is kept as a selectable mode.  Here the producer warps of a CTA
 // stream tiles of the stack into a ring of shared-memory stages with bulk asynchronous
 // copies that complete on mbarriers; ~200 KB per SM are in flight with no register
 // cost, and the consumer warps spend their time on the Philox mask, which needs no data
@@ -31,7 +34,8 @@ namespace wash {
 constexpr long long kWaitLimitCycles = 4000000000ll;   // about 2 s of SM clock
 constexpr int kMaxStages = 12;
 constexpr int kHeaderBytes = 512;   // three barriers per stage and the abort flag
-constexpr int kProducerWarps = 4;
+constexpr int kProducerWarps = 1;
+constexpr int kCtasPerSm = 3;
 constexpr int kPieceBytes = 4096;   // largest single bulk copy
 
 struct ShuffleTmaArgs {
@@ -123,7 +127,7 @@ __device__ __forceinline__ uint32_t stage_value(const unsigned char *stage, int 
 }
 
 template <class TA, class TB, int LAYOUT>
-__global__ void __launch_bounds__(32 * kProducerWarps + 512, 1) shuffle_tma_kernel(const __grid_constant__ ShuffleTmaArgs a)
+__global__ void __launch_bounds__(32 * kProducerWarps + 512) shuffle_tma_kernel(const __grid_constant__ ShuffleTmaArgs a)
 {
     extern __shared__ __align__(128) unsigned char smem_raw[];
     constexpr bool kHasB = TB::kCode != kDtypeNone;
@@ -330,28 +334,40 @@ cudaError_t launch_shuffle_tma_typed(const ShuffleArgs &args, const LaunchShape 
     constexpr bool kHasB = TB::kCode != kDtypeNone;
     const int N = args.pop.N;
     const uint32_t group_bytes = static_cast<uint32_t>(N) * (TA::kBytes * 4 + (kHasB ? TB::kBytes * 4 : 0));
-    const size_t budget = 200 * 1024;
+    // Each bulk copy costs its CTA a fixed ~85 ns whatever its size (measured), so one CTA
+    // cannot keep an SM's share of HBM busy with copies of a few KiB: aim for kCtasPerSm
+    // CTAs per SM, each with its own ring, and fall back to fewer when a population's
+    // stages are too large for that.
+    int ctas = kCtasPerSm;
     ShuffleTmaArgs t;
     t.s = args;
-    int G = 256;
-    if (shape.threads == 128 || shape.threads == 64 || shape.threads == 32) G = shape.threads;
-    while (G > 32 && 3ull * G * group_bytes + static_cast<size_t>(N) * G > budget) G >>= 1;
-    t.G = G;
-    t.teams = G >= 256 ? 2 : (G == 128 ? 4 : 8);
-    if (shape.blocks_per_sm > 0) t.teams = shape.blocks_per_sm;   // tuning: consumer teams per CTA
-    if (t.teams * G > 512) t.teams = 512 / G;
-    t.stage_bytes = static_cast<uint32_t>(G) * group_bytes;
-    t.b_offset = static_cast<uint32_t>(G) * N * TA::kBytes * 4;
-    const size_t perm_bytes = (static_cast<size_t>(N) * G * t.teams + 15) & ~static_cast<size_t>(15);   // sized for the most teams considered
+    int stages = 0;
+    size_t perm_bytes = 0;
     const size_t seg_bytes = sizeof(SegEntry) * static_cast<size_t>(args.pop.n_seg);
     t.seg_smem_bytes = seg_bytes <= 16 * 1024 ? static_cast<uint32_t>(seg_bytes) : 0;
-    int stages = static_cast<int>((budget - perm_bytes - t.seg_smem_bytes) / t.stage_bytes);
-    if (stages > kMaxStages) stages = kMaxStages;
-    // A stage must always be consumed by the same team: a waiter may only wait for the
-    // phase that follows the one it saw last, so it has to see every phase of its stages.
-    while (t.teams > 1 && stages / t.teams * t.teams < 2) t.teams >>= 1;
-    stages = stages / t.teams * t.teams;
+    for (; ctas >= 1; --ctas) {
+        const size_t budget = 200 * 1024 / ctas;
+        int G = 256;
+        if (shape.threads == 128 || shape.threads == 64 || shape.threads == 32) G = shape.threads;
+        while (G > 32 && 2ull * G * group_bytes + static_cast<size_t>(N) * G + t.seg_smem_bytes > budget) G >>= 1;
+        t.G = G;
+        t.teams = 1;
+        if (shape.blocks_per_sm > 0) t.teams = shape.blocks_per_sm;   // tuning: consumer teams per CTA
+        if (t.teams * G > 512) t.teams = 512 / G;
+        t.stage_bytes = static_cast<uint32_t>(G) * group_bytes;
+        t.b_offset = static_cast<uint32_t>(G) * N * TA::kBytes * 4;
+        perm_bytes = (static_cast<size_t>(N) * G * t.teams + 15) & ~static_cast<size_t>(15);   // sized for the most teams considered
+        if (perm_bytes + t.seg_smem_bytes >= budget) continue;
+        stages = static_cast<int>((budget - perm_bytes - t.seg_smem_bytes) / t.stage_bytes);
+        if (stages > kMaxStages) stages = kMaxStages;
+        // A stage must always be consumed by the same team: a waiter has to see every
+        // phase of the barriers it waits on.
+        while (t.teams > 1 && stages / t.teams * t.teams < 2) t.teams >>= 1;
+        stages = stages / t.teams * t.teams;
+        if (stages >= 2) break;
+    }
     if (stages < 2) return cudaErrorInvalidConfiguration;
+    const int G = t.G;
     t.stages = stages;
     t.n_tiles = (args.pop.n_groups + G - 1) / G;
     const size_t smem = kHeaderBytes + static_cast<size_t>(stages) * t.stage_bytes + perm_bytes + t.seg_smem_bytes;
