@@ -58,8 +58,10 @@ enum wash_schedule { WASH_SCHEDULE_DECREASING = 0, WASH_SCHEDULE_CONSTANT = 1, W
 enum wash_mode {
     WASH_MODE_STREAM = 0, /* one pass that reads the whole stack; writes selected coordinates */
     WASH_MODE_SPARSE = 1, /* draws the mask first; touches only selected coordinates          */
-    WASH_MODE_STREAM_STAGED = 2 /* as STREAM, the stack staged through shared memory by bulk
-                                   asynchronous copies instead of through registers          */
+    WASH_MODE_STREAM_STAGED = 2, /* as STREAM, the stack staged through shared memory by bulk
+                                    asynchronous copies (TMA) instead of through registers   */
+    WASH_MODE_STREAM_ASYNC = 3   /* as STREAM, staged through shared memory by per-thread
+                                    asynchronous copies (cp.async)                           */
 };
 
 #define WASH_MAX_N 64            /* largest population                                     */

@@ -12,6 +12,7 @@ WASH_N_LIST(WASH_DECL)
 #undef WASH_DECL
 cudaError_t launch_shuffle_sparse(const ShuffleArgs &, int, int, const LaunchShape &, cudaStream_t, bool *);
 cudaError_t launch_shuffle_staged(const ShuffleArgs &, int, int, const LaunchShape &, cudaStream_t, bool *);
+cudaError_t launch_shuffle_async_staged(const ShuffleArgs &, int, int, const LaunchShape &, cudaStream_t, bool *);
 cudaError_t launch_reduce_n0(const ReduceArgs &, int, int, int, const LaunchShape &, cudaStream_t, bool *);
 
 static std::atomic<uint64_t> g_launches{0};
@@ -34,6 +35,7 @@ cudaError_t launch_shuffle(const ShuffleArgs &args, int a_dtype, int b_dtype, in
                            const LaunchShape &shape, cudaStream_t stream, bool *supported)
 {
     if (mode == kModeStreamStaged) return launch_shuffle_staged(args, a_dtype, b_dtype, shape, stream, supported);
+    if (mode == kModeStreamAsync) return launch_shuffle_async_staged(args, a_dtype, b_dtype, shape, stream, supported);
     if (mode == kModeStream) {
         switch (args.pop.N) {
 #define WASH_CASE(n) case n: return launch_shuffle_stream_n##n(args, a_dtype, b_dtype, shape, stream, supported);
