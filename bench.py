@@ -253,7 +253,7 @@ def run_ours(args, rank: int, world: int, local_rank: int) -> None:
     if opt_d is not None:
         pop.bind(B.WASH_STACK_OPT, opt_d)
     if args.mode != "stream":
-        B.wash_set_mode(pop.ctx, {"sparse": B.WASH_MODE_SPARSE, "staged": B.WASH_MODE_STREAM_STAGED, "async": B.WASH_MODE_STREAM_ASYNC}[args.mode])
+        B.wash_set_mode(pop.ctx, {"sparse": B.WASH_MODE_SPARSE, "staged": B.WASH_MODE_STREAM_STAGED, "registers": B.WASH_MODE_STREAM_REGISTERS}[args.mode])
     if args.threads or args.blocks_per_sm:
         B.wash_set_launch(pop.ctx, args.threads, args.blocks_per_sm)
     pdt = B.WASH_BF16 if wl.bf16 else B.WASH_F32
@@ -361,7 +361,7 @@ def run_ours(args, rank: int, world: int, local_rank: int) -> None:
                 "papa_ema": {"ms": float(mean_ms[1]), "GBps": ab["ema"] / (mean_ms[1] * 1e-3) / 1e9},
                 "population_average": {"ms": float(mean_ms[2]), "GBps": ab["average"] / (mean_ms[2] * 1e-3) / 1e9},
             },
-            "roofline": {"kernel": "shuffle_kernel (params + momentum, streaming)", "bound": "hbm", "achieved": shuffle_gbs,
+            "roofline": {"kernel": "shuffle kernel, mode %s (params + momentum)" % args.mode, "bound": "hbm", "achieved": shuffle_gbs,
                          "peak": peak, "peak_source": peak_src, "unit": "GB/s", "frac": shuffle_gbs / peak,
                          "traffic": TRAFFIC.get(wl.name)},
             "e2e": {"value": ab["step"] * world / (e2e_ms / e2e_steps * 1e-3) / 1e9, "unit": "GB/s",
@@ -415,7 +415,7 @@ def main() -> None:
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="cfg2_resnet18_n5", choices=sorted(W.CONFIGS))
-    ap.add_argument("--mode", default="stream", choices=["stream", "sparse", "staged", "async"])
+    ap.add_argument("--mode", default="stream", choices=["stream", "sparse", "staged", "registers"])
     ap.add_argument("--threads", type=int, default=0)
     ap.add_argument("--blocks-per-sm", type=int, default=0)
     ap.add_argument("--no-cpu-baseline", action="store_true")

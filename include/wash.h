@@ -56,12 +56,14 @@ enum wash_dtype { WASH_F32 = 0, WASH_BF16 = 1 };
 enum wash_stack { WASH_STACK_PARAMS = 0, WASH_STACK_OPT = 1 };
 enum wash_schedule { WASH_SCHEDULE_DECREASING = 0, WASH_SCHEDULE_CONSTANT = 1, WASH_SCHEDULE_INCREASING = 2 };
 enum wash_mode {
-    WASH_MODE_STREAM = 0, /* one pass that reads the whole stack; writes selected coordinates */
+    WASH_MODE_STREAM = 0, /* one pass that reads the whole stack and writes the selected
+                             coordinates; the stack travels global -> shared memory by
+                             per-thread asynchronous copies (cp.async).  Default.            */
     WASH_MODE_SPARSE = 1, /* draws the mask first; touches only selected coordinates          */
-    WASH_MODE_STREAM_STAGED = 2, /* as STREAM, the stack staged through shared memory by bulk
-                                    asynchronous copies (TMA) instead of through registers   */
-    WASH_MODE_STREAM_ASYNC = 3   /* as STREAM, staged through shared memory by per-thread
-                                    asynchronous copies (cp.async)                           */
+    WASH_MODE_STREAM_STAGED = 2,   /* as STREAM, staged by bulk asynchronous copies (TMA)     */
+    WASH_MODE_STREAM_REGISTERS = 3 /* as STREAM, the loads held in registers (kernels unrolled
+                                      for N in {2,3,4,5,6,8,10,12,16,20,24,32}; other N run
+                                      the default kernel)                                     */
 };
 
 #define WASH_MAX_N 64            /* largest population                                     */

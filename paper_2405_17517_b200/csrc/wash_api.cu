@@ -3,7 +3,6 @@
 #include <cmath>
 #include <cstdarg>
 #include <cstdio>
-#include <cstdlib>
 #include <cstring>
 #include <new>
 #include <string>
@@ -88,7 +87,6 @@ struct wash_ctx {
     size_t avg_bytes = 0;
 
     int mode = WASH_MODE_STREAM;
-    int prefetch_ahead = getenv("WASH_PREFETCH") ? atoi(getenv("WASH_PREFETCH")) : 0;
     wash::LaunchShape shape{0, 0, 148};
 };
 
@@ -203,7 +201,6 @@ int shuffle_impl(wash_ctx *ctx, int which, uint64_t step, double p, const double
     args.step_hi8 = static_cast<uint32_t>(step >> 32) << 8;
     args.stats = reinterpret_cast<unsigned long long *>(stats);
     args.status = ctx->status_dev;
-    args.prefetch_ahead = ctx->prefetch_ahead;
     bool supported = false;
     cudaError_t err = wash::launch_shuffle(args, a_dtype, b_dtype, ctx->mode, ctx->shape, stream, &supported);
     if (err != cudaSuccess) return cuda_fail(err, "shuffle kernel launch");
@@ -232,7 +229,6 @@ int reduce_impl(wash_ctx *ctx, int op, int stack, void *out, int out_dtype, floa
     args.group_hi = ctx->seg_host[static_cast<size_t>(tensor_hi) - 1].group_end;
     args.sq_out = sq_out;
     args.status = ctx->status_dev;
-    args.prefetch_ahead = ctx->prefetch_ahead;
     bool supported = false;
     cudaError_t err = wash::launch_reduce(args, op, ctx->stack_dtype[stack], out_dtype, ctx->shape, stream, &supported);
     if (err != cudaSuccess) return cuda_fail(err, "kernel launch");
@@ -371,7 +367,7 @@ int wash_bind(wash_ctx *ctx, int32_t stack, int32_t dtype, void *dev_ptr, int64_
 int wash_set_mode(wash_ctx *ctx, int32_t mode)
 {
     if (!ctx) return fail(WASH_ERR_ARG, "ctx is NULL");
-    if (mode < WASH_MODE_STREAM || mode > WASH_MODE_STREAM_ASYNC) return fail(WASH_ERR_ARG, "unknown mode %d", mode);
+    if (mode < WASH_MODE_STREAM || mode > WASH_MODE_STREAM_REGISTERS) return fail(WASH_ERR_ARG, "unknown mode %d", mode);
     ctx->mode = mode;
     return WASH_OK;
 }

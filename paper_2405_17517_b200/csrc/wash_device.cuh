@@ -112,23 +112,6 @@ __device__ __forceinline__ char *group_vec_ptr(void *base, const PopView &pop, u
     return static_cast<char *>(base) + e * T::kBytes;
 }
 
-// Asks L2 for the lines that hold group g of every model (n_vecs vectors of T).  Called
-// by all threads of a warp for their own (consecutive) groups; one thread per 128-byte
-// line issues the prefetch.  Only a hint: no register, no shared memory, no completion.
-template <class T, int LAYOUT>
-__device__ __forceinline__ void prefetch_group_l2(void *base, const PopView &pop, uint64_t g, int n_vecs)
-{
-    constexpr int kVecBytes = T::kBytes * 4;
-    if (LAYOUT == kLayoutNP) {
-        if ((threadIdx.x & (128 / kVecBytes - 1)) != 0) return;
-        for (int j = 0; j < n_vecs; ++j)
-            asm volatile("prefetch.global.L2 [%0];" ::"l"(group_vec_ptr<T, LAYOUT>(base, pop, g, j)));
-    } else {
-        for (int j = 0; j < n_vecs; j += 128 / kVecBytes)
-            asm volatile("prefetch.global.L2 [%0];" ::"l"(group_vec_ptr<T, LAYOUT>(base, pop, g, j)));
-    }
-}
-
 // raw bits of (model n, coordinate c of the group) out of the group's N vectors
 template <class T, int LAYOUT, int CAP>
 __device__ __forceinline__ uint32_t group_value(const typename T::vec (&v)[CAP], int n_models, int n, int c)

@@ -34,18 +34,19 @@ bool has_unrolled_kernels(int N)
 cudaError_t launch_shuffle(const ShuffleArgs &args, int a_dtype, int b_dtype, int mode,
                            const LaunchShape &shape, cudaStream_t stream, bool *supported)
 {
+    if (mode == kModeSparse) return launch_shuffle_sparse(args, a_dtype, b_dtype, shape, stream, supported);
     if (mode == kModeStreamStaged) return launch_shuffle_staged(args, a_dtype, b_dtype, shape, stream, supported);
-    if (mode == kModeStreamAsync) return launch_shuffle_async_staged(args, a_dtype, b_dtype, shape, stream, supported);
-    if (mode == kModeStream) {
+    if (mode == kModeStreamRegisters) {
         switch (args.pop.N) {
 #define WASH_CASE(n) case n: return launch_shuffle_stream_n##n(args, a_dtype, b_dtype, shape, stream, supported);
             WASH_N_LIST(WASH_CASE)
 #undef WASH_CASE
         default:
-            break;   // no unrolled kernel for this N: the sparse kernel gives the same bits
+            break;   // no unrolled kernel for this N: the default kernel gives the same bits
         }
     }
-    return launch_shuffle_sparse(args, a_dtype, b_dtype, shape, stream, supported);
+    // default streaming kernel: staged through shared memory with cp.async, any N
+    return launch_shuffle_async_staged(args, a_dtype, b_dtype, shape, stream, supported);
 }
 
 cudaError_t launch_reduce(const ReduceArgs &args, int op, int dtype, int out_dtype,

@@ -9,7 +9,7 @@ constexpr int kMaxN = 64;          // largest population (WASH_MAX_N)
 constexpr int kTileShift = 8;      // lookup tile = 256 groups = 1024 coordinates
 constexpr int kDtypeF32 = 0, kDtypeBF16 = 1, kDtypeNone = -1;
 constexpr int kLayoutNP = 0, kLayoutPN = 1;
-constexpr int kModeStream = 0, kModeSparse = 1, kModeStreamStaged = 2, kModeStreamAsync = 3;
+constexpr int kModeStream = 0, kModeSparse = 1, kModeStreamStaged = 2, kModeStreamRegisters = 3;
 
 // One row of a stack is cut into groups of 4 consecutive elements; a group never
 // straddles two tensors because tensors start on multiples of 8 elements.
@@ -42,7 +42,6 @@ struct ShuffleArgs {
     uint32_t step_lo, step_hi8;   // step & 0xFFFFFFFF, (step >> 32) << 8
     unsigned long long *stats;    // device-accessible {selected, moved} or nullptr
     uint32_t *status;             // device status word
-    int prefetch_ahead;           // loop trips ahead whose lines are prefetched into L2 (0 = none)
 };
 
 struct ReduceArgs {
@@ -53,7 +52,6 @@ struct ReduceArgs {
     uint32_t group_lo, group_hi;  // range of groups to process
     double *sq_out;               // consensus: N doubles (device) or nullptr
     uint32_t *status;
-    int prefetch_ahead;           // as in ShuffleArgs
 };
 
 enum ReduceOp { kOpEma = 0, kOpAverage = 1, kOpPapaAll = 2, kOpConsensus = 3 };

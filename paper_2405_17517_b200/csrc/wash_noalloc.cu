@@ -148,7 +148,6 @@ extern "C" int wash_shuffle_noalloc(int32_t N, int32_t n_tensors, const int64_t 
             args.step_hi8 = static_cast<uint32_t>(step >> 32) << 8;
             args.stats = reinterpret_cast<unsigned long long *>(stats);
             args.status = nullptr;
-            args.prefetch_ahead = 0;
             const wash::LaunchShape shape{0, 0, sm_count};
             bool supported = false;
             err = wash::launch_shuffle(args, dtype, wash::kDtypeNone, wash::kModeStream, shape, stream, &supported);

@@ -27,10 +27,6 @@ __global__ void __launch_bounds__(256) reduce_kernel(const __grid_constant__ Red
     const uint64_t stride = static_cast<uint64_t>(gridDim.x) * blockDim.x;
     for (uint64_t g = a.group_lo + static_cast<uint64_t>(blockIdx.x) * blockDim.x + threadIdx.x; g < a.group_hi; g += stride) {
         typename T::vec v[kCap];
-        if (a.prefetch_ahead > 0) {
-            const uint64_t g_ahead = g + stride * a.prefetch_ahead;
-            if (g_ahead < a.group_hi) prefetch_group_l2<T, LAYOUT>(a.stack, a.pop, g_ahead, n_models);
-        }
         if constexpr (N > 0) {
 #pragma unroll
             for (int j = 0; j < N; ++j) v[j] = T::load_group(group_vec_ptr<T, LAYOUT>(a.stack, a.pop, g, j));

@@ -58,15 +58,6 @@ __global__ void __launch_bounds__(256) shuffle_kernel(const __grid_constant__ Sh
         typename TA::vec va[kRegs];
         typename TB::vec vb[kRegs];
         if constexpr (STREAM) {
-            // deepen the memory pipeline beyond what the registers hold: ask L2 for the
-            // lines of a later trip of this loop
-            if (a.prefetch_ahead > 0) {
-                const uint64_t g_ahead = g + stride * a.prefetch_ahead;
-                if (g_ahead < a.pop.n_groups) {
-                    prefetch_group_l2<TA, LAYOUT>(a.a, a.pop, g_ahead, N);
-                    if constexpr (kHasB) prefetch_group_l2<TB, LAYOUT>(a.b, a.pop, g_ahead, N);
-                }
-            }
 #pragma unroll
             for (int j = 0; j < N; ++j) va[j] = TA::load_group(group_vec_ptr<TA, LAYOUT>(a.a, a.pop, g, j));
             if constexpr (kHasB) {

@@ -140,7 +140,7 @@ cudaError_t launch_shuffle_async_typed(const ShuffleArgs &args, const LaunchShap
     const size_t per_thread = static_cast<size_t>(args.pop.N) * (TA::kBytes * 4 + (kHasB ? TB::kBytes * 4 : 0) + 1);
     // block size: as many threads as keep a block's image near 44 KiB, so that five blocks
     // (about 200 KiB in flight) share an SM
-    int threads = shape.threads > 0 ? shape.threads : 256;
+    int threads = shape.threads > 0 ? shape.threads : 128;   // measured: 64-128 beat 256 (a block waits for its slowest thread)
     if (threads > 256) threads = 256;
     if (shape.threads <= 0)
         while (threads > 32 && per_thread * threads > 44 * 1024) threads >>= 1;
