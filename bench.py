@@ -381,7 +381,11 @@ def run_ours(args, rank: int, world: int, local_rank: int) -> None:
 
 # DRAM bytes per shuffle launch from the ncu capture summarised under profiles/ (None
 # until a capture of the current kernel exists).
-TRAFFIC = {}
+TRAFFIC = {
+    # shuffle_async_kernel<F32, F32, [N][P]>, two launches: 448.88 MB read + 6.66..7.18 MB written
+    "cfg2_resnet18_n5": {"dram_bytes_read": 448.88e6, "dram_bytes_write": 6.9e6,
+                         "source": "profiles/shuffle_async_kernel_cfg2_resnet18_n5.md"},
+}
 
 
 def cpu_baseline(wl: Workload) -> dict:
@@ -401,7 +405,7 @@ def cpu_baseline(wl: Workload) -> dict:
         oracle.population_average(pop, params, out)
         steps += 1
         dt = time.perf_counter() - t0
-        if dt > 10.0 or steps >= 50:
+        if dt > 10.0 or steps >= 2000:
             break
     gbs = wl.algorithmic_bytes(sel / steps)["step"] * steps / dt / 1e9
     return {"value": gbs, "unit": "GB/s", "cores": threads, "kind": "oracle",

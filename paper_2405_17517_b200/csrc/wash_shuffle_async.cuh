@@ -43,9 +43,14 @@ __device__ __forceinline__ void async_fetch(uint32_t image, void *base, const Po
     constexpr int kVec = T::kBytes * 4;
     const uint32_t t = threadIdx.x, T_ = blockDim.x;
     if (LAYOUT == kLayoutNP) {
-        if (t < groups_in_block)
-            for (int j = 0; j < n_models; ++j)
-                cp_async<kVec>(image + (j * T_ + t) * kVec, group_vec_ptr<T, LAYOUT>(base, pop, g_block + t, j));
+        if (t < groups_in_block) {
+            // model j's vector of this thread's group: one row further in global memory,
+            // one row of T vectors further in the image
+            const char *src = group_vec_ptr<T, LAYOUT>(base, pop, g_block + t, 0);
+            const size_t row_bytes = static_cast<size_t>(pop.padded_P) * T::kBytes;
+            uint32_t dst = image + t * kVec;
+            for (int j = 0; j < n_models; ++j, src += row_bytes, dst += T_ * kVec) cp_async<kVec>(dst, src);
+        }
     } else {
         const uint32_t vecs = groups_in_block * n_models;
         const char *src = static_cast<const char *>(base) + 4ll * static_cast<long long>(g_block) * n_models * T::kBytes;
@@ -65,7 +70,7 @@ __device__ __forceinline__ uint32_t image_value(const unsigned char *image, int 
 }
 
 template <class TA, class TB, int LAYOUT>
-__global__ void __launch_bounds__(256) shuffle_async_kernel(const __grid_constant__ ShuffleArgs a)
+__global__ void __launch_bounds__(256, 5) shuffle_async_kernel(const __grid_constant__ ShuffleArgs a)
 {
     extern __shared__ __align__(128) unsigned char smem_raw[];
     constexpr bool kHasB = TB::kCode != kDtypeNone;
@@ -140,7 +145,7 @@ cudaError_t launch_shuffle_async_typed(const ShuffleArgs &args, const LaunchShap
     const size_t per_thread = static_cast<size_t>(args.pop.N) * (TA::kBytes * 4 + (kHasB ? TB::kBytes * 4 : 0) + 1);
     // block size: as many threads as keep a block's image near 44 KiB, so that five blocks
     // (about 200 KiB in flight) share an SM
-    int threads = shape.threads > 0 ? shape.threads : 128;   // measured: 64-128 beat 256 (a block waits for its slowest thread)
+    int threads = shape.threads > 0 ? shape.threads : 64;   // measured: 64 beats 128 and 256 (a block holds its shared memory until its slowest thread is done)
     if (threads > 256) threads = 256;
     if (shape.threads <= 0)
         while (threads > 32 && per_thread * threads > 44 * 1024) threads >>= 1;
