@@ -363,7 +363,8 @@ def run_ours(args, rank: int, world: int, local_rank: int) -> None:
             },
             "roofline": {"kernel": "shuffle kernel, mode %s (params + momentum)" % args.mode, "bound": "hbm", "achieved": shuffle_gbs,
                          "peak": peak, "peak_source": peak_src, "unit": "GB/s", "frac": shuffle_gbs / peak,
-                         "traffic": TRAFFIC.get(wl.name)},
+                         "traffic": TRAFFIC.get(wl.name, {}).get("dram_bytes") if args.mode == "stream" else None,
+                         "traffic_source": TRAFFIC.get(wl.name, {}).get("source") if args.mode == "stream" else None},
             "e2e": {"value": ab["step"] * world / (e2e_ms / e2e_steps * 1e-3) / 1e9, "unit": "GB/s",
                     "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": e2e_steps,
                     "api": "wash_step_host (pinned host stacks)"},
@@ -383,7 +384,7 @@ def run_ours(args, rank: int, world: int, local_rank: int) -> None:
 # until a capture of the current kernel exists).
 TRAFFIC = {
     # shuffle_async_kernel<F32, F32, [N][P]>, two launches: 448.88 MB read + 6.66..7.18 MB written
-    "cfg2_resnet18_n5": {"dram_bytes_read": 448.88e6, "dram_bytes_write": 6.9e6,
+    "cfg2_resnet18_n5": {"dram_bytes": 448.88e6 + 6.9e6,
                          "source": "profiles/shuffle_async_kernel_cfg2_resnet18_n5.md"},
 }
 
@@ -412,6 +413,59 @@ def cpu_baseline(wl: Workload) -> dict:
             "sample": "%d full steps of the same workload (%.1f s)" % (steps, dt), "ms_per_step": dt / steps * 1e3}
 
 
+def run_sweep(args) -> None:
+    """Config 5: flat fp32 populations, N x P x p x layout, shuffle only.  One JSON line
+    per cell (not the default bench line)."""
+    import torch
+    from paper_2405_17517_b200 import binding as B
+
+    torch.cuda.set_device(0)
+    B.load()
+    peak, _ = measured_peak()
+    modes = {"stream": B.WASH_MODE_STREAM, "sparse": B.WASH_MODE_SPARSE, "registers": B.WASH_MODE_STREAM_REGISTERS,
+             "staged": B.WASH_MODE_STREAM_STAGED}
+    stream = torch.cuda.current_stream()
+    for N in (2, 4, 8, 16, 32):
+        for logP in (20, 24, 27):
+            P = 1 << logP
+            for layout, lname in ((B.WASH_LAYOUT_NP, "[N][P]"), (B.WASH_LAYOUT_PN, "[P][N]")):
+                pop = B.Population(N, [P], layout, 0)
+                gen = torch.Generator(device="cuda").manual_seed(N * 100 + logP)
+                stack = torch.randn(N * pop.padded_P, generator=gen, device="cuda", dtype=torch.float32) * 0.05
+                pop.bind(B.WASH_STACK_PARAMS, stack)
+                stats = torch.zeros(2, dtype=torch.int64, device="cuda")
+                for p in (1e-4, 1e-3, 1e-2, 1e-1, 1.0):
+                    for mode in args.sweep_modes.split(","):
+                        B.wash_set_mode(pop.ctx, modes[mode])
+                        for w in range(3):
+                            B.wash_shuffle(pop.ctx, w, p, None, SEED, stream, stats)
+                        torch.cuda.synchronize()
+                        stats.zero_()
+                        reps = 20 if N * P * 4 < (4 << 30) else 8
+                        ev = [torch.cuda.Event(enable_timing=True) for _ in range(reps + 1)]
+                        ev[0].record(stream)
+                        for k in range(reps):
+                            B.wash_shuffle(pop.ctx, 3 + k, p, None, SEED, stream, stats)
+                            ev[k + 1].record(stream)
+                        torch.cuda.synchronize()
+                        ms = float(np.median([ev[k].elapsed_time(ev[k + 1]) for k in range(reps)]))
+                        sel = int(stats[0]) / reps
+                        footprint = N * P * 4
+                        streamed = footprint + sel * N * 4
+                        line = {"N": N, "P": P, "p": p, "layout": lname, "mode": mode, "ms": ms,
+                                "selected_per_launch": sel, "param_swaps_per_s": sel * N / (ms * 1e-3),
+                                "algorithmic_GBps": 2 * 4 * N * sel / (ms * 1e-3) / 1e9}
+                        if mode != "sparse":
+                            line["streamed_GBps"] = streamed / (ms * 1e-3) / 1e9
+                            line["frac_of_hbm"] = line["streamed_GBps"] / peak
+                        line["l2"] = "L2-influenced" if footprint < (256 << 20) else "beyond L2"
+                        print(json.dumps(line), flush=True)
+                B.wash_check(pop.ctx)
+                pop.close()
+                del stack
+                torch.cuda.empty_cache()
+
+
 def main() -> None:
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -423,12 +477,17 @@ def main() -> None:
     ap.add_argument("--threads", type=int, default=0)
     ap.add_argument("--blocks-per-sm", type=int, default=0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--sweep", action="store_true", help="config-5 sweep of the shuffle kernel (many JSON lines)")
+    ap.add_argument("--sweep-modes", default="stream,sparse")
     args = ap.parse_args()
     if args.warmup < 3 and args.impl == "ours":
         args.warmup = 3
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if args.sweep:
+        run_sweep(args)
+        return
     if args.impl == "reference":
         run_reference(args, rank, world)
     else:

@@ -1,0 +1,122 @@
+"""GPU parity at the benchmark's full sizes: the ResNet populations of configs 2-4 in the
+launch configuration bench.py times (default mode and launch shape), compared with the
+oracle bit for bit, and a multi-gigabyte flat population of config 5 checked on sampled
+coordinate ranges that the oracle recomputes on its own."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2405_17517_b200 import binding as B
+from paper_2405_17517_b200 import workloads as W
+from gpu_util import Case, bits, to_host_bits
+
+pytestmark = pytest.mark.gpu
+
+
+def _resnet_case(name):
+    cfg = W.CONFIGS[name]
+    table = W.table_from_spec(cfg["table"])
+    N = cfg["N"]
+    dense = W.init_population(table, N, seed=0)
+    mom = W.init_momentum(table, N, seed=1)
+    c = Case(N, W.numels(table), 0, cfg["dtype"], "f32", dense=dense, dense_opt=mom)
+    return cfg, c, len(table)
+
+
+def test_config2_resnet18_n5_full_size():
+    cfg, c, T = _resnet_case("cfg2_resnet18_n5")
+    oracle.set_threads(oracle.max_threads())
+    tot = [0, 0]
+    for step in range(4):
+        B.wash_shuffle_both(c.gpu.ctx, step, cfg["p"], None, seed=0, stats=c.stats_dev)
+        s = oracle.shuffle(c.ora, c.host, cfg["p"], seed=0, step=step, stack2=c.host_opt)
+        tot[0] += s[0]; tot[1] += s[1]
+    c.assert_equal("cfg2 shuffle")
+    assert c.gpu_stats() == tuple(tot)
+    B.papa_ema(c.gpu.ctx, B.WASH_STACK_PARAMS, 0.99)
+    oracle.papa_ema(c.ora, c.host, 0.99)
+    c.assert_equal("cfg2 ema")
+    out = torch.zeros(c.P, dtype=torch.float32, device="cuda")
+    B.population_average(c.gpu.ctx, B.WASH_STACK_PARAMS, out, B.WASH_F32)
+    want = np.zeros(c.P, dtype=np.float32)
+    oracle.population_average(c.ora, c.host, want)
+    assert (to_host_bits(out) == want.view(np.uint32)).all()
+    oracle.set_threads(1)
+    c.close()
+
+
+def test_config3_resnet50_n10_thousand_steps_per_layer_p():
+    """N = 10, 161 tensors, p_t = 0.01 (1 - t/160), momentum shuffled along, 1000 steps;
+    compared at steps 0, 1, 10, 100 and 999, counters at the end."""
+    cfg, c, T = _resnet_case("cfg3_resnet50_n10")
+    oracle.set_threads(oracle.max_threads())
+    pl = B.wash_layer_probs(T, cfg["p"], B.WASH_SCHEDULE_DECREASING)
+    assert np.array_equal(pl, oracle.layer_probs(T, cfg["p"]))
+    tot = [0, 0]
+    for step in range(1000):
+        B.wash_shuffle_both(c.gpu.ctx, step, cfg["p"], pl, seed=3, stats=c.stats_dev)
+        s = oracle.shuffle(c.ora, c.host, pl, seed=3, step=step, stack2=c.host_opt)
+        tot[0] += s[0]; tot[1] += s[1]
+        if step in (0, 1, 10, 100, 999):
+            c.assert_equal("cfg3 step %d" % step)
+    assert c.gpu_stats() == tuple(tot)
+    # the paper's communicated fraction for this schedule, measured: sum_t q_t d_t / P per step
+    numel = np.asarray(c.numel, dtype=np.float64)
+    expect = (np.floor(pl * 2.0 ** 32) / 2.0 ** 32 * numel).sum() * 1000
+    assert abs(tot[0] - expect) < 5 * np.sqrt(expect)
+    oracle.set_threads(1)
+    c.close()
+
+
+def test_config4_resnet50_bf16_weights_fp32_momentum():
+    cfg, c, T = _resnet_case("cfg4_resnet50_bf16_n8")
+    oracle.set_threads(oracle.max_threads())
+    for step in range(3):
+        B.wash_shuffle_both(c.gpu.ctx, step, cfg["p"], None, seed=5, stats=c.stats_dev)
+        oracle.shuffle(c.ora, c.host, cfg["p"], seed=5, step=step, stack2=c.host_opt)
+    c.assert_equal("cfg4 shuffle")
+    for alpha in (0.999, 0.001):
+        B.papa_ema(c.gpu.ctx, B.WASH_STACK_PARAMS, alpha)
+        oracle.papa_ema(c.ora, c.host, alpha)
+        c.assert_equal("cfg4 ema %g" % alpha)
+    for code, np_dtype, t_dtype in ((B.WASH_F32, np.float32, torch.float32), (B.WASH_BF16, np.uint16, torch.bfloat16)):
+        out = torch.zeros(c.P, dtype=t_dtype, device="cuda")
+        B.population_average(c.gpu.ctx, B.WASH_STACK_PARAMS, out, code)
+        want = np.zeros(c.P, dtype=np_dtype)
+        oracle.population_average(c.ora, c.host, want)
+        assert (to_host_bits(out) == bits(want)).all()
+    oracle.set_threads(1)
+    c.close()
+
+
+@pytest.mark.parametrize("layout", [0, 1])
+@pytest.mark.parametrize("N,logP,p", [(8, 27, 0.01), (32, 24, 0.1), (2, 27, 1.0)])
+def test_config5_large_flat_population_on_sampled_ranges(N, logP, p, layout):
+    """A flat fp32 population far larger than L2 (up to 4.3 GB), generated on the device.
+    64 random coordinate ranges are copied out before and after the shuffle; the oracle
+    shuffles each range on its own (segment of tensor 0 starting at that coordinate) and
+    must reproduce it.  The counters are checked against the binomial law."""
+    P = 1 << logP
+    pop = B.Population(N, [P], layout, 0)
+    gen = torch.Generator(device="cuda").manual_seed(1234 + N)
+    stack = torch.randn(N * pop.padded_P, generator=gen, device="cuda", dtype=torch.float32) * 0.05
+    pop.bind(B.WASH_STACK_PARAMS, stack)
+    view = stack.view(N, P) if layout == 0 else stack.view(P, N).t()
+    rng = np.random.default_rng(7)
+    starts = (rng.integers(0, (P - 4096) // 4, 62) * 4).tolist() + [0, P - 4096]
+    before = [view[:, s:s + 4096].contiguous().cpu().numpy() for s in starts]
+    stats = torch.zeros(2, dtype=torch.int64, device="cuda")
+    B.wash_shuffle(pop.ctx, 17, p, None, seed=99, stats=stats)
+    torch.cuda.synchronize()
+    B.wash_check(pop.ctx)
+    for s, b in zip(starts, before):
+        seg = oracle.Population(N, [4096], tensor_id=[0], coord_begin=[s])
+        want = np.ascontiguousarray(b)
+        oracle.shuffle(seg, want, p, seed=99, step=17)
+        got = view[:, s:s + 4096].contiguous().cpu().numpy()
+        assert (got.view(np.uint32) == want.view(np.uint32)).all(), s
+    sel = int(stats[0])
+    q = oracle.threshold(p) / 2.0 ** 32
+    assert abs(sel - P * q) <= 5 * np.sqrt(P * q * (1 - q)) + 1e-9
+    pop.close()
