@@ -216,8 +216,8 @@ int wash_step_host(wash_ctx *ctx, int32_t ops, void *host_params, void *host_opt
  * synchronise the whole device, would stall work that other streams have in flight.
  * wash_shuffle_noalloc runs the same streaming shuffle as wash_shuffle on ONE stack
  * without any context and without allocating device or pinned memory: its tables live
- * in a fixed 288 KiB array inside the library image (32 KiB segment table + 256 KiB tile
- * index), which every GPU that loads libwash.so holds until the process exits.
+ * in a fixed 296 KiB array inside the library image (32 KiB segment table, 256 KiB tile
+ * index, 8 KiB of partial sums for the counters), which every GPU that loads libwash.so holds until the process exits.
  *
  *   N, n_tensors, numel, layout     as for wash_create (row geometry is the same:
  *                                   tensors start on multiples of 8 elements);
@@ -233,8 +233,8 @@ int wash_step_host(wash_ctx *ctx, int32_t ops, void *host_params, void *host_opt
  * arguments.  The message of a failure is returned by wash_noalloc_last_error().
  *
  * Sharing: all calls on a GPU use the one array.  Each call rewrites the tables it
- * needs in full, in stream order, so nothing has to be cleared between calls and the
- * previous call's contents never leak into the next; but two calls that can overlap on
+ * needs in full and zeroes the partial sums, in stream order, so the previous call's
+ * contents never leak into the next; but two calls that can overlap on
  * the GPU (different streams without an ordering between them, or two host threads)
  * race on the tables and give undefined results.  Issue them on one stream, or order
  * them with events.

@@ -83,6 +83,7 @@ struct wash_ctx {
 
     uint32_t *status_dev = nullptr;
     wash_stats *stats_dev = nullptr;       // for wash_step_host
+    wash::StatSlot *stat_slots_dev = nullptr;
     void *avg_dev = nullptr;               // for wash_step_host, allocated on first use
     size_t avg_bytes = 0;
 
@@ -100,6 +101,7 @@ void release(wash_ctx *ctx)
     if (ctx->tile_first_dev) cudaFree(ctx->tile_first_dev);
     if (ctx->status_dev) cudaFree(ctx->status_dev);
     if (ctx->stats_dev) cudaFree(ctx->stats_dev);
+    if (ctx->stat_slots_dev) cudaFree(ctx->stat_slots_dev);
     if (ctx->avg_dev) cudaFree(ctx->avg_dev);
     for (int s = 0; s < kSlots; ++s) {
         if (ctx->seg_pinned[s]) cudaFreeHost(ctx->seg_pinned[s]);
@@ -200,6 +202,7 @@ int shuffle_impl(wash_ctx *ctx, int which, uint64_t step, double p, const double
     args.step_lo = static_cast<uint32_t>(step);
     args.step_hi8 = static_cast<uint32_t>(step >> 32) << 8;
     args.stats = reinterpret_cast<unsigned long long *>(stats);
+    args.stat_slots = ctx->stat_slots_dev;
     args.status = ctx->status_dev;
     bool supported = false;
     cudaError_t err = wash::launch_shuffle(args, a_dtype, b_dtype, ctx->mode, ctx->shape, stream, &supported);
@@ -305,7 +308,8 @@ int wash_create_segments(wash_ctx **out, int32_t N, int32_t n_segments, const in
     if ((err = cudaMalloc(&ctx->seg_dev, seg_bytes)) != cudaSuccess ||
         (err = cudaMalloc(&ctx->tile_first_dev, sizeof(uint32_t) * ctx->n_tiles)) != cudaSuccess ||
         (err = cudaMalloc(&ctx->status_dev, sizeof(uint32_t))) != cudaSuccess ||
-        (err = cudaMalloc(&ctx->stats_dev, sizeof(wash_stats))) != cudaSuccess) {
+        (err = cudaMalloc(&ctx->stats_dev, sizeof(wash_stats))) != cudaSuccess ||
+        (err = cudaMalloc(&ctx->stat_slots_dev, sizeof(wash::StatSlot) * wash::kStatSlots)) != cudaSuccess) {
         release(ctx);
         cudaGetLastError();
         return fail(WASH_ERR_ALLOC, "device allocation failed: %s", cudaGetErrorString(err));
@@ -320,7 +324,8 @@ int wash_create_segments(wash_ctx **out, int32_t N, int32_t n_segments, const in
     }
     if ((err = cudaMemcpy(ctx->tile_first_dev, tile_first.data(), sizeof(uint32_t) * ctx->n_tiles, cudaMemcpyHostToDevice)) != cudaSuccess ||
         (err = cudaMemset(ctx->status_dev, 0, sizeof(uint32_t))) != cudaSuccess ||
-        (err = cudaMemset(ctx->stats_dev, 0, sizeof(wash_stats))) != cudaSuccess) {
+        (err = cudaMemset(ctx->stats_dev, 0, sizeof(wash_stats))) != cudaSuccess ||
+        (err = cudaMemset(ctx->stat_slots_dev, 0, sizeof(wash::StatSlot) * wash::kStatSlots)) != cudaSuccess) {
         release(ctx);
         return cuda_fail(err, "table upload");
     }

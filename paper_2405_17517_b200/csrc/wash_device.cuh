@@ -121,6 +121,52 @@ __device__ __forceinline__ uint32_t group_value(const typename T::vec (&v)[CAP],
     return T::get(v[f >> 2], f & 3);
 }
 
+// ---- statistics -----------------------------------------------------------------------
+// Called by every thread of the block at the end of a shuffle kernel.  Warp sums go to
+// shared memory, the block's sums to slot (blockIdx mod kStatSlots); the last block to
+// report to a slot moves the slot's totals into the caller's counters and leaves the slot
+// zeroed for the next launch.
+__device__ __forceinline__ void publish_block_stats(unsigned long long *stats, StatSlot *slots, uint32_t selected, uint32_t moved)
+{
+    if (!stats) return;
+    __shared__ uint32_t block_sum[2];
+    if (threadIdx.x == 0) block_sum[0] = block_sum[1] = 0;
+    __syncthreads();
+    selected = __reduce_add_sync(0xFFFFFFFFu, selected);
+    moved = __reduce_add_sync(0xFFFFFFFFu, moved);
+    if ((threadIdx.x & 31) == 0 && selected) {
+        atomicAdd(&block_sum[0], selected);
+        atomicAdd(&block_sum[1], moved);
+    }
+    __syncthreads();
+    if (threadIdx.x != 0) return;
+    if (!slots) {
+        if (block_sum[0]) {
+            atomicAdd(stats, static_cast<unsigned long long>(block_sum[0]));
+            atomicAdd(stats + 1, static_cast<unsigned long long>(block_sum[1]));
+        }
+        return;
+    }
+    const uint32_t slot = blockIdx.x % kStatSlots;
+    StatSlot *s = slots + slot;
+    if (block_sum[0]) {
+        atomicAdd(&s->selected, static_cast<unsigned long long>(block_sum[0]));
+        atomicAdd(&s->moved, static_cast<unsigned long long>(block_sum[1]));
+    }
+    __threadfence();
+    const unsigned long long reporters = (gridDim.x - slot + kStatSlots - 1) / kStatSlots;   // blocks that map to this slot
+    if (atomicAdd(&s->blocks, 1ull) == reporters - 1) {
+        __threadfence();
+        const unsigned long long sel = atomicExch(&s->selected, 0ull);
+        const unsigned long long mov = atomicExch(&s->moved, 0ull);
+        atomicExch(&s->blocks, 0ull);
+        if (sel) {
+            atomicAdd(stats, sel);
+            atomicAdd(stats + 1, mov);
+        }
+    }
+}
+
 // ---- which segment does group g belong to ---------------------------------------------
 struct GroupInfo {
     uint32_t tensor_id;

@@ -24,6 +24,14 @@ struct SegEntry {
 };
 static_assert(sizeof(SegEntry) == 32, "SegEntry must stay 32 bytes");
 
+// Statistics are gathered in kStatSlots partial sums before they reach the caller's two
+// counters: per-block atomics on one address were measured to cost about 1 ns each and
+// to dominate the kernel once most blocks have a selected coordinate.
+constexpr int kStatSlots = 256;
+struct StatSlot {
+    unsigned long long selected, moved, blocks, reserved;
+};
+
 struct PopView {
     int N;
     int layout;
@@ -41,6 +49,7 @@ struct ShuffleArgs {
     uint32_t key0, key1;          // seed
     uint32_t step_lo, step_hi8;   // step & 0xFFFFFFFF, (step >> 32) << 8
     unsigned long long *stats;    // device-accessible {selected, moved} or nullptr
+    StatSlot *stat_slots;         // device, kStatSlots zeroed entries (left zeroed by every launch), or nullptr
     uint32_t *status;             // device status word
 };
 

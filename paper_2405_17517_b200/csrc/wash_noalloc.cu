@@ -29,7 +29,8 @@ constexpr long long kMaxRowElems = WASH_NOALLOC_MAX_ROW_ELEMS;
 constexpr size_t kMaxTiles = static_cast<size_t>(kMaxRowElems / 4) >> wash::kTileShift;
 constexpr size_t kSegBytes = sizeof(SegEntry) * kMaxTensors;          // 32 KiB
 constexpr size_t kTileBytes = sizeof(uint32_t) * kMaxTiles;           // 256 KiB
-constexpr size_t kScratchBytes = kSegBytes + kTileBytes;
+constexpr size_t kSlotBytes = sizeof(wash::StatSlot) * wash::kStatSlots;   // 8 KiB
+constexpr size_t kScratchBytes = kSegBytes + kTileBytes + kSlotBytes;
 
 // The scratch itself.  In host code this name is only a handle for the runtime's symbol
 // lookup -- it is NOT a device address and must never be passed to a kernel; the device
@@ -126,10 +127,13 @@ extern "C" int wash_shuffle_noalloc(int32_t N, int32_t n_tensors, const int64_t 
         cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
         SegEntry *seg_dev = reinterpret_cast<SegEntry *>(scratch);
         uint32_t *tile_dev = reinterpret_cast<uint32_t *>(scratch + kSegBytes);
-        // Both tables are rewritten in full, in stream order, before the kernel reads
-        // them; nothing in the scratch is carried over from the previous call.
+        // Both tables are rewritten in full and the counters' partial sums are zeroed, in
+        // stream order, before the kernel runs; nothing is carried over from the previous call.
         err = cudaMemcpyAsync(seg_dev, seg.data(), sizeof(SegEntry) * seg.size(), cudaMemcpyHostToDevice, stream);
         if (err == cudaSuccess) err = cudaMemcpyAsync(tile_dev, tile_first.data(), sizeof(uint32_t) * n_tiles, cudaMemcpyHostToDevice, stream);
+        // the partial sums of the statistics must start at zero
+        wash::StatSlot *slots_dev = reinterpret_cast<wash::StatSlot *>(scratch + kSegBytes + kTileBytes);
+        if (err == cudaSuccess && stats) err = cudaMemsetAsync(slots_dev, 0, kSlotBytes, stream);
         if (err != cudaSuccess) rc = fail(WASH_ERR_CUDA, cudaGetErrorString(err));
         if (rc == WASH_OK) {
             wash::ShuffleArgs args;
@@ -147,6 +151,7 @@ extern "C" int wash_shuffle_noalloc(int32_t N, int32_t n_tensors, const int64_t 
             args.step_lo = static_cast<uint32_t>(step);
             args.step_hi8 = static_cast<uint32_t>(step >> 32) << 8;
             args.stats = reinterpret_cast<unsigned long long *>(stats);
+            args.stat_slots = slots_dev;
             args.status = nullptr;
             const wash::LaunchShape shape{0, 0, sm_count};
             bool supported = false;

@@ -109,23 +109,7 @@ __global__ void __launch_bounds__(256) shuffle_kernel(const __grid_constant__ Sh
             ++selected;
         }
     }
-    if (a.stats) {
-        // warp sums -> block sums in shared memory -> one pair of global atomics per block
-        __shared__ uint32_t block_sum[2];
-        if (threadIdx.x == 0) block_sum[0] = block_sum[1] = 0;
-        __syncthreads();
-        selected = __reduce_add_sync(0xFFFFFFFFu, selected);
-        moved = __reduce_add_sync(0xFFFFFFFFu, moved);
-        if ((threadIdx.x & 31) == 0 && selected) {
-            atomicAdd(&block_sum[0], selected);
-            atomicAdd(&block_sum[1], moved);
-        }
-        __syncthreads();
-        if (threadIdx.x == 0 && block_sum[0]) {
-            atomicAdd(a.stats, static_cast<unsigned long long>(block_sum[0]));
-            atomicAdd(a.stats + 1, static_cast<unsigned long long>(block_sum[1]));
-        }
-    }
+    publish_block_stats(a.stats, a.stat_slots, selected, moved);
 }
 
 template <int N, class TA, class TB, bool STREAM>

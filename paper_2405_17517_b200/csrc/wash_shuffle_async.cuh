@@ -120,22 +120,7 @@ __global__ void __launch_bounds__(256, 5) shuffle_async_kernel(const __grid_cons
             ++selected;
         }
     }
-    if (a.stats) {
-        __shared__ uint32_t block_sum[2];
-        if (threadIdx.x == 0) block_sum[0] = block_sum[1] = 0;
-        __syncthreads();
-        selected = __reduce_add_sync(0xFFFFFFFFu, selected);
-        moved = __reduce_add_sync(0xFFFFFFFFu, moved);
-        if ((threadIdx.x & 31) == 0 && selected) {
-            atomicAdd(&block_sum[0], selected);
-            atomicAdd(&block_sum[1], moved);
-        }
-        __syncthreads();
-        if (threadIdx.x == 0 && block_sum[0]) {
-            atomicAdd(a.stats, static_cast<unsigned long long>(block_sum[0]));
-            atomicAdd(a.stats + 1, static_cast<unsigned long long>(block_sum[1]));
-        }
-    }
+    publish_block_stats(a.stats, a.stat_slots, selected, moved);
 }
 
 template <class TA, class TB>
