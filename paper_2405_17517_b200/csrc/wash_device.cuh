@@ -123,9 +123,9 @@ __device__ __forceinline__ uint32_t group_value(const typename T::vec (&v)[CAP],
 
 // ---- statistics -----------------------------------------------------------------------
 // Called by every thread of the block at the end of a shuffle kernel.  Warp sums go to
-// shared memory, the block's sums to slot (blockIdx mod kStatSlots); the last block to
-// report to a slot moves the slot's totals into the caller's counters and leaves the slot
-// zeroed for the next launch.
+// shared memory and a block that selected anything adds its sums to slot (blockIdx mod
+// kStatSlots).  flush_stats_kernel, launched right after the shuffle, moves the slots'
+// totals into the caller's counters and zeroes the slots.
 __device__ __forceinline__ void publish_block_stats(unsigned long long *stats, StatSlot *slots, uint32_t selected, uint32_t moved)
 {
     if (!stats) return;
@@ -139,32 +139,10 @@ __device__ __forceinline__ void publish_block_stats(unsigned long long *stats, S
         atomicAdd(&block_sum[1], moved);
     }
     __syncthreads();
-    if (threadIdx.x != 0) return;
-    if (!slots) {
-        if (block_sum[0]) {
-            atomicAdd(stats, static_cast<unsigned long long>(block_sum[0]));
-            atomicAdd(stats + 1, static_cast<unsigned long long>(block_sum[1]));
-        }
-        return;
-    }
-    const uint32_t slot = blockIdx.x % kStatSlots;
-    StatSlot *s = slots + slot;
-    if (block_sum[0]) {
-        atomicAdd(&s->selected, static_cast<unsigned long long>(block_sum[0]));
-        atomicAdd(&s->moved, static_cast<unsigned long long>(block_sum[1]));
-    }
-    __threadfence();
-    const unsigned long long reporters = (gridDim.x - slot + kStatSlots - 1) / kStatSlots;   // blocks that map to this slot
-    if (atomicAdd(&s->blocks, 1ull) == reporters - 1) {
-        __threadfence();
-        const unsigned long long sel = atomicExch(&s->selected, 0ull);
-        const unsigned long long mov = atomicExch(&s->moved, 0ull);
-        atomicExch(&s->blocks, 0ull);
-        if (sel) {
-            atomicAdd(stats, sel);
-            atomicAdd(stats + 1, mov);
-        }
-    }
+    if (threadIdx.x != 0 || block_sum[0] == 0) return;
+    unsigned long long *dst = slots ? &slots[blockIdx.x % kStatSlots].selected : stats;   // {selected, moved} are adjacent in both
+    atomicAdd(dst, static_cast<unsigned long long>(block_sum[0]));
+    atomicAdd(dst + 1, static_cast<unsigned long long>(block_sum[1]));
 }
 
 // ---- which segment does group g belong to ---------------------------------------------

@@ -31,8 +31,28 @@ bool has_unrolled_kernels(int N)
     }
 }
 
-cudaError_t launch_shuffle(const ShuffleArgs &args, int a_dtype, int b_dtype, int mode,
-                           const LaunchShape &shape, cudaStream_t stream, bool *supported)
+// Sums the partial statistics into the caller's counters and zeroes them again.
+__global__ void __launch_bounds__(kStatSlots) flush_stats_kernel(StatSlot *slots, unsigned long long *stats)
+{
+    __shared__ unsigned long long sum[2];
+    if (threadIdx.x == 0) sum[0] = sum[1] = 0;
+    __syncthreads();
+    const unsigned long long sel = slots[threadIdx.x].selected, mov = slots[threadIdx.x].moved;
+    if (sel) {
+        slots[threadIdx.x].selected = 0;
+        slots[threadIdx.x].moved = 0;
+        atomicAdd(&sum[0], sel);
+        atomicAdd(&sum[1], mov);
+    }
+    __syncthreads();
+    if (threadIdx.x == 0 && sum[0]) {
+        atomicAdd(stats, sum[0]);
+        atomicAdd(stats + 1, sum[1]);
+    }
+}
+
+static cudaError_t launch_shuffle_kernel(const ShuffleArgs &args, int a_dtype, int b_dtype, int mode,
+                                         const LaunchShape &shape, cudaStream_t stream, bool *supported)
 {
     if (mode == kModeSparse) return launch_shuffle_sparse(args, a_dtype, b_dtype, shape, stream, supported);
     if (mode == kModeStreamStaged) return launch_shuffle_staged(args, a_dtype, b_dtype, shape, stream, supported);
@@ -47,6 +67,16 @@ cudaError_t launch_shuffle(const ShuffleArgs &args, int a_dtype, int b_dtype, in
     }
     // default streaming kernel: staged through shared memory with cp.async, any N
     return launch_shuffle_async_staged(args, a_dtype, b_dtype, shape, stream, supported);
+}
+
+cudaError_t launch_shuffle(const ShuffleArgs &args, int a_dtype, int b_dtype, int mode,
+                           const LaunchShape &shape, cudaStream_t stream, bool *supported)
+{
+    cudaError_t err = launch_shuffle_kernel(args, a_dtype, b_dtype, mode, shape, stream, supported);
+    if (err != cudaSuccess || !*supported || !args.stats || !args.stat_slots) return err;
+    flush_stats_kernel<<<1, kStatSlots, 0, stream>>>(args.stat_slots, args.stats);
+    count_launch();
+    return cudaGetLastError();
 }
 
 cudaError_t launch_reduce(const ReduceArgs &args, int op, int dtype, int out_dtype,
