@@ -58,15 +58,33 @@ __device__ __forceinline__ void async_fetch(uint32_t image, void *base, const Po
     }
 }
 
-// raw bits of (model n, coordinate c) of this thread's group, out of the block image
+// raw bits of (model n, coordinate c) of the group of block thread t, out of the block image
 template <class T, int LAYOUT>
-__device__ __forceinline__ uint32_t image_value(const unsigned char *image, int n_models, int n, int c)
+__device__ __forceinline__ uint32_t image_value(const unsigned char *image, int n_models, uint32_t t, int n, int c)
 {
-    const uint32_t t = threadIdx.x, T_ = blockDim.x;
+    const uint32_t T_ = blockDim.x;
     const uint32_t elem = LAYOUT == kLayoutNP ? (static_cast<uint32_t>(n) * T_ + t) * 4u + c
                                               : (4u * t + c) * n_models + n;
     if (T::kBytes == 4) return reinterpret_cast<const uint32_t *>(image)[elem];
     return reinterpret_cast<const uint16_t *>(image)[elem];
+}
+
+// pi for coordinate i with pi(n) in nibble n of the result (N <= 16): the Fisher-Yates of
+// draw_permutation_u8 on a register instead of a shared-memory column.
+__device__ __forceinline__ uint64_t draw_permutation_packed(int n_models, uint32_t i, uint32_t tensor, uint32_t step_lo,
+                                                            uint32_t step_hi8, uint32_t k0, uint32_t k1)
+{
+    uint64_t perm = 0xFEDCBA9876543210ull;
+    Philox4 w{0, 0, 0, 0};
+    for (int k = n_models - 1, m = 0; k >= 1; --k, ++m) {
+        if ((m & 3) == 0) w = philox4x32_10(i, tensor, step_lo, step_hi8 | (1u + (static_cast<uint32_t>(m) >> 2)), k0, k1);
+        const uint32_t r = w.x;
+        w.x = w.y; w.y = w.z; w.z = w.w;
+        const uint32_t sk = 4u * k, sj = 4u * __umulhi(r, static_cast<uint32_t>(k + 1));
+        const uint64_t diff = ((perm >> sk) ^ (perm >> sj)) & 15ull;   // swap nibbles k and j
+        perm ^= (diff << sk) | (diff << sj);
+    }
+    return perm;
 }
 
 template <class TA, class TB, int LAYOUT>
@@ -78,7 +96,8 @@ __global__ void __launch_bounds__(256, 5) shuffle_async_kernel(const __grid_cons
     const uint32_t T_ = blockDim.x;
     unsigned char *image_a = smem_raw;
     unsigned char *image_b = image_a + static_cast<size_t>(n_models) * T_ * TA::kBytes * 4;
-    uint8_t *s_perm = image_b + (kHasB ? static_cast<size_t>(n_models) * T_ * TB::kBytes * 4 : 0) + threadIdx.x;   // column [n][T]
+    uint8_t *s_list = image_b + (kHasB ? static_cast<size_t>(n_models) * T_ * TB::kBytes * 4 : 0);   // 128 bytes per warp
+    uint8_t *s_perm = s_list + 4 * T_ + threadIdx.x;   // column [n][T], used when N > 16
 
     const uint64_t g_block = static_cast<uint64_t>(blockIdx.x) * T_;
     const uint32_t groups_in_block = static_cast<uint32_t>(min(static_cast<uint64_t>(T_), a.pop.n_groups - g_block));
@@ -99,23 +118,62 @@ __global__ void __launch_bounds__(256, 5) shuffle_async_kernel(const __grid_cons
         }
     }
     // Every thread waits for its own copies (none may be in flight when the block ends).
-    // In the [P][N] image a thread's values were copied by other threads, so a block with
-    // a selected coordinate also needs a block-wide barrier before it reads the image.
+    // A selected coordinate is served by whichever lane of the warp gets it (below), so
+    // the warp must see each other's copies; in the [P][N] image a group's values were
+    // copied by threads of other warps, so a block with a selected coordinate needs a
+    // block-wide barrier instead.
     cp_async_wait_all();
-    const bool block_has_work = LAYOUT == kLayoutPN ? (__syncthreads_or(sel != 0) != 0) : (sel != 0);
-    if (block_has_work && sel != 0) {
-#pragma unroll 1
-        for (int c = 0; c < 4; ++c) {
-            if (!((sel >> c) & 1u)) continue;
-            draw_permutation_u8(s_perm, T_, n_models, 4u * gi.cgroup + c, gi.tensor_id, a.step_lo, a.step_hi8, a.key0, a.key1);
-            const long long e = 4ll * static_cast<long long>(g) + c;
-            for (int n = 0; n < n_models; ++n) {
-                const int src = s_perm[n * T_];
-                if (src == n) continue;
-                TA::store_elem(a.a, elem_index<LAYOUT>(a.pop, n, e), image_value<TA, LAYOUT>(image_a, n_models, src, c));
-                if constexpr (kHasB)
-                    TB::store_elem(a.b, elem_index<LAYOUT>(a.pop, n, e), image_value<TB, LAYOUT>(image_b, n_models, src, c));
-                ++moved;
+    if (LAYOUT == kLayoutPN) __syncthreads_or(sel != 0);
+    else __syncwarp();
+
+    // The warp's selected coordinates are listed in shared memory and dealt out to the
+    // lanes 32 at a time: with a few selected coordinates per warp (p around 0.01-0.1)
+    // one round serves them all, instead of one divergent pass per coordinate slot.
+    const uint32_t lane = threadIdx.x & 31u, warp_base = threadIdx.x & ~31u;
+    const uint32_t mine = __popc(sel);
+    uint32_t upto = mine;   // inclusive prefix sum over the lanes
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+        const uint32_t v = __shfl_up_sync(0xFFFFFFFFu, upto, d);
+        if (lane >= static_cast<uint32_t>(d)) upto += v;
+    }
+    const uint32_t total = __shfl_sync(0xFFFFFFFFu, upto, 31);
+    if (total != 0) {
+        uint8_t *list = s_list + (threadIdx.x >> 5) * 128;   // entry = owner lane * 4 + coordinate slot
+        uint32_t pos = upto - mine;
+#pragma unroll
+        for (int c = 0; c < 4; ++c)
+            if ((sel >> c) & 1u) list[pos++] = static_cast<uint8_t>(lane * 4 + c);
+        __syncwarp();
+        for (uint32_t first = 0; first < total; first += 32) {
+            const bool active = first + lane < total;
+            const uint32_t entry = active ? list[first + lane] : 0u;
+            const uint32_t owner = entry >> 2, c = entry & 3u;
+            const uint32_t cgroup = __shfl_sync(0xFFFFFFFFu, gi.cgroup, owner);
+            const uint32_t tensor = __shfl_sync(0xFFFFFFFFu, gi.tensor_id, owner);
+            if (!active) continue;
+            const uint32_t t_owner = warp_base + owner;
+            const long long e = 4ll * static_cast<long long>(g_block + t_owner) + c;
+            if (n_models <= 16) {
+                const uint64_t perm = draw_permutation_packed(n_models, 4u * cgroup + c, tensor, a.step_lo, a.step_hi8, a.key0, a.key1);
+                for (int n = 0; n < n_models; ++n) {
+                    const int src = static_cast<int>((perm >> (4 * n)) & 15ull);
+                    if (src == n) continue;
+                    TA::store_elem(a.a, elem_index<LAYOUT>(a.pop, n, e), image_value<TA, LAYOUT>(image_a, n_models, t_owner, src, c));
+                    if constexpr (kHasB)
+                        TB::store_elem(a.b, elem_index<LAYOUT>(a.pop, n, e), image_value<TB, LAYOUT>(image_b, n_models, t_owner, src, c));
+                    ++moved;
+                }
+            } else {
+                draw_permutation_u8(s_perm, T_, n_models, 4u * cgroup + c, tensor, a.step_lo, a.step_hi8, a.key0, a.key1);
+                for (int n = 0; n < n_models; ++n) {
+                    const int src = s_perm[n * T_];
+                    if (src == n) continue;
+                    TA::store_elem(a.a, elem_index<LAYOUT>(a.pop, n, e), image_value<TA, LAYOUT>(image_a, n_models, t_owner, src, c));
+                    if constexpr (kHasB)
+                        TB::store_elem(a.b, elem_index<LAYOUT>(a.pop, n, e), image_value<TB, LAYOUT>(image_b, n_models, t_owner, src, c));
+                    ++moved;
+                }
             }
             ++selected;
         }
@@ -127,7 +185,8 @@ template <class TA, class TB>
 cudaError_t launch_shuffle_async_typed(const ShuffleArgs &args, const LaunchShape &shape, cudaStream_t stream)
 {
     constexpr bool kHasB = TB::kCode != kDtypeNone;
-    const size_t per_thread = static_cast<size_t>(args.pop.N) * (TA::kBytes * 4 + (kHasB ? TB::kBytes * 4 : 0) + 1);
+    // images of both stacks, 4 bytes of the warp's list, a byte per model for the permutation
+    const size_t per_thread = static_cast<size_t>(args.pop.N) * (TA::kBytes * 4 + (kHasB ? TB::kBytes * 4 : 0) + 1) + 4;
     // block size: as many threads as keep a block's image near 44 KiB, so that five blocks
     // (about 200 KiB in flight) share an SM
     int threads = shape.threads > 0 ? shape.threads : 64;   // measured: 64 beats 128 and 256 (a block holds its shared memory until its slowest thread is done)
