@@ -425,16 +425,19 @@ def run_sweep(args) -> None:
     modes = {"stream": B.WASH_MODE_STREAM, "sparse": B.WASH_MODE_SPARSE, "registers": B.WASH_MODE_STREAM_REGISTERS,
              "staged": B.WASH_MODE_STREAM_STAGED}
     stream = torch.cuda.current_stream()
-    for N in (2, 4, 8, 16, 32):
-        for logP in (20, 24, 27):
+    pick = lambda text, default, conv: [conv(x) for x in text.split(",")] if text else default
+    for N in pick(args.sweep_N, [2, 4, 8, 16, 32], int):
+        for logP in pick(args.sweep_logP, [20, 24, 27], int):
             P = 1 << logP
             for layout, lname in ((B.WASH_LAYOUT_NP, "[N][P]"), (B.WASH_LAYOUT_PN, "[P][N]")):
+                if args.sweep_layout and args.sweep_layout != ("np" if layout == B.WASH_LAYOUT_NP else "pn"):
+                    continue
                 pop = B.Population(N, [P], layout, 0)
                 gen = torch.Generator(device="cuda").manual_seed(N * 100 + logP)
                 stack = torch.randn(N * pop.padded_P, generator=gen, device="cuda", dtype=torch.float32) * 0.05
                 pop.bind(B.WASH_STACK_PARAMS, stack)
                 stats = torch.zeros(2, dtype=torch.int64, device="cuda")
-                for p in (1e-4, 1e-3, 1e-2, 1e-1, 1.0):
+                for p in pick(args.sweep_p, [1e-4, 1e-3, 1e-2, 1e-1, 1.0], float):
                     for mode in args.sweep_modes.split(","):
                         B.wash_set_mode(pop.ctx, modes[mode])
                         for w in range(3):
@@ -479,6 +482,10 @@ def main() -> None:
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--sweep", action="store_true", help="config-5 sweep of the shuffle kernel (many JSON lines)")
     ap.add_argument("--sweep-modes", default="stream,sparse")
+    ap.add_argument("--sweep-N", default="", help="comma list; default 2,4,8,16,32")
+    ap.add_argument("--sweep-logP", default="", help="comma list; default 20,24,27")
+    ap.add_argument("--sweep-p", default="", help="comma list; default 1e-4..1")
+    ap.add_argument("--sweep-layout", default="", choices=["", "np", "pn"])
     args = ap.parse_args()
     if args.warmup < 3 and args.impl == "ours":
         args.warmup = 3

@@ -1,6 +1,6 @@
 // One translation unit per population size: compiled with -DWASH_N=<n> for every n of
 // WASH_N_LIST (unrolled kernels) and with -DWASH_N=0 (run-time-N kernels, which include
-// the sparse shuffle).
+// the reduce kernels for population sizes without an unrolled instantiation).
 #include "wash_shuffle.cuh"
 #include "wash_reduce.cuh"
 
@@ -18,12 +18,6 @@ cudaError_t WASH_CAT(launch_shuffle_stream_n, WASH_N)(const ShuffleArgs &args, i
                                                       const LaunchShape &shape, cudaStream_t stream, bool *supported)
 {
     return launch_shuffle_n<WASH_N, true>(args, a_dtype, b_dtype, shape, stream, supported);
-}
-#else
-cudaError_t launch_shuffle_sparse(const ShuffleArgs &args, int a_dtype, int b_dtype, const LaunchShape &shape,
-                                  cudaStream_t stream, bool *supported)
-{
-    return launch_shuffle_n<0, false>(args, a_dtype, b_dtype, shape, stream, supported);
 }
 #endif
 

@@ -87,22 +87,29 @@ __device__ __forceinline__ uint64_t draw_permutation_packed(int n_models, uint32
     return perm;
 }
 
-template <class TA, class TB, int LAYOUT>
+// FETCH = true: the streaming kernel described above.  FETCH = false: the sparse mode --
+// nothing is copied up front; the mask is drawn first and a selected coordinate's N values
+// are loaded from global memory into a private shared-memory column when it is served.
+template <class TA, class TB, int LAYOUT, bool FETCH>
 __global__ void __launch_bounds__(256, 5) shuffle_async_kernel(const __grid_constant__ ShuffleArgs a)
 {
     extern __shared__ __align__(128) unsigned char smem_raw[];
     constexpr bool kHasB = TB::kCode != kDtypeNone;
     const int n_models = a.pop.N;
     const uint32_t T_ = blockDim.x;
+    // FETCH: images of the two stacks.  !FETCH: one column of N words per thread.
     unsigned char *image_a = smem_raw;
-    unsigned char *image_b = image_a + static_cast<size_t>(n_models) * T_ * TA::kBytes * 4;
-    uint8_t *s_list = image_b + (kHasB ? static_cast<size_t>(n_models) * T_ * TB::kBytes * 4 : 0);   // 128 bytes per warp
+    unsigned char *image_b = image_a + static_cast<size_t>(n_models) * T_ * (FETCH ? TA::kBytes * 4 : 4);
+    uint8_t *s_list = image_b + (FETCH && kHasB ? static_cast<size_t>(n_models) * T_ * TB::kBytes * 4 : 0);   // 128 bytes per warp
     uint8_t *s_perm = s_list + 4 * T_ + threadIdx.x;   // column [n][T], used when N > 16
+    uint32_t *s_col = reinterpret_cast<uint32_t *>(smem_raw) + threadIdx.x;   // !FETCH: column [n][T]
 
     const uint64_t g_block = static_cast<uint64_t>(blockIdx.x) * T_;
     const uint32_t groups_in_block = static_cast<uint32_t>(min(static_cast<uint64_t>(T_), a.pop.n_groups - g_block));
-    async_fetch<TA, LAYOUT>(smem_addr(image_a), a.a, a.pop, g_block, groups_in_block, n_models);
-    if constexpr (kHasB) async_fetch<TB, LAYOUT>(smem_addr(image_b), a.b, a.pop, g_block, groups_in_block, n_models);
+    if constexpr (FETCH) {
+        async_fetch<TA, LAYOUT>(smem_addr(image_a), a.a, a.pop, g_block, groups_in_block, n_models);
+        if constexpr (kHasB) async_fetch<TB, LAYOUT>(smem_addr(image_b), a.b, a.pop, g_block, groups_in_block, n_models);
+    }
 
     uint32_t selected = 0, moved = 0, sel = 0;
     GroupInfo gi{0, 0, 0, 0};
@@ -122,9 +129,11 @@ __global__ void __launch_bounds__(256, 5) shuffle_async_kernel(const __grid_cons
     // the warp must see each other's copies; in the [P][N] image a group's values were
     // copied by threads of other warps, so a block with a selected coordinate needs a
     // block-wide barrier instead.
-    cp_async_wait_all();
-    if (LAYOUT == kLayoutPN) __syncthreads_or(sel != 0);
-    else __syncwarp();
+    if constexpr (FETCH) {
+        cp_async_wait_all();
+        if (LAYOUT == kLayoutPN) __syncthreads_or(sel != 0);
+        else __syncwarp();
+    }
 
     // The warp's selected coordinates are listed in shared memory and dealt out to the
     // lanes 32 at a time: with a few selected coordinates per warp (p around 0.01-0.1)
@@ -154,10 +163,15 @@ __global__ void __launch_bounds__(256, 5) shuffle_async_kernel(const __grid_cons
             if (!active) continue;
             const uint32_t t_owner = warp_base + owner;
             const long long e = 4ll * static_cast<long long>(g_block + t_owner) + c;
-            if (n_models <= 16) {
-                const uint64_t perm = draw_permutation_packed(n_models, 4u * cgroup + c, tensor, a.step_lo, a.step_hi8, a.key0, a.key1);
+            uint64_t perm = 0;
+            if (n_models <= 16) perm = draw_permutation_packed(n_models, 4u * cgroup + c, tensor, a.step_lo, a.step_hi8, a.key0, a.key1);
+            else draw_permutation_u8(s_perm, T_, n_models, 4u * cgroup + c, tensor, a.step_lo, a.step_hi8, a.key0, a.key1);
+            auto source_of = [&](int n) -> int {
+                return n_models <= 16 ? static_cast<int>((perm >> (4 * n)) & 15ull) : static_cast<int>(s_perm[n * T_]);
+            };
+            if constexpr (FETCH) {
                 for (int n = 0; n < n_models; ++n) {
-                    const int src = static_cast<int>((perm >> (4 * n)) & 15ull);
+                    const int src = source_of(n);
                     if (src == n) continue;
                     TA::store_elem(a.a, elem_index<LAYOUT>(a.pop, n, e), image_value<TA, LAYOUT>(image_a, n_models, t_owner, src, c));
                     if constexpr (kHasB)
@@ -165,14 +179,20 @@ __global__ void __launch_bounds__(256, 5) shuffle_async_kernel(const __grid_cons
                     ++moved;
                 }
             } else {
-                draw_permutation_u8(s_perm, T_, n_models, 4u * cgroup + c, tensor, a.step_lo, a.step_hi8, a.key0, a.key1);
+                // all N old values first (the exchange is in place), then the moved ones back
+                for (int n = 0; n < n_models; ++n) s_col[n * T_] = TA::load_elem(a.a, elem_index<LAYOUT>(a.pop, n, e));
                 for (int n = 0; n < n_models; ++n) {
-                    const int src = s_perm[n * T_];
+                    const int src = source_of(n);
                     if (src == n) continue;
-                    TA::store_elem(a.a, elem_index<LAYOUT>(a.pop, n, e), image_value<TA, LAYOUT>(image_a, n_models, t_owner, src, c));
-                    if constexpr (kHasB)
-                        TB::store_elem(a.b, elem_index<LAYOUT>(a.pop, n, e), image_value<TB, LAYOUT>(image_b, n_models, t_owner, src, c));
+                    TA::store_elem(a.a, elem_index<LAYOUT>(a.pop, n, e), s_col[src * T_]);
                     ++moved;
+                }
+                if constexpr (kHasB) {
+                    for (int n = 0; n < n_models; ++n) s_col[n * T_] = TB::load_elem(a.b, elem_index<LAYOUT>(a.pop, n, e));
+                    for (int n = 0; n < n_models; ++n) {
+                        const int src = source_of(n);
+                        if (src != n) TB::store_elem(a.b, elem_index<LAYOUT>(a.pop, n, e), s_col[src * T_]);
+                    }
                 }
             }
             ++selected;
@@ -181,20 +201,21 @@ __global__ void __launch_bounds__(256, 5) shuffle_async_kernel(const __grid_cons
     publish_block_stats(a.stats, a.stat_slots, selected, moved);
 }
 
-template <class TA, class TB>
+template <class TA, class TB, bool FETCH>
 cudaError_t launch_shuffle_async_typed(const ShuffleArgs &args, const LaunchShape &shape, cudaStream_t stream)
 {
     constexpr bool kHasB = TB::kCode != kDtypeNone;
-    // images of both stacks, 4 bytes of the warp's list, a byte per model for the permutation
-    const size_t per_thread = static_cast<size_t>(args.pop.N) * (TA::kBytes * 4 + (kHasB ? TB::kBytes * 4 : 0) + 1) + 4;
+    // images of both stacks (or one column of words), 4 bytes of the warp's list, a byte
+    // per model for the permutation
+    const size_t per_thread = static_cast<size_t>(args.pop.N) * ((FETCH ? TA::kBytes * 4 + (kHasB ? TB::kBytes * 4 : 0) : 4) + 1) + 4;
     // block size: as many threads as keep a block's image near 44 KiB, so that five blocks
     // (about 200 KiB in flight) share an SM
-    int threads = shape.threads > 0 ? shape.threads : 64;   // measured: 64 beats 128 and 256 (a block holds its shared memory until its slowest thread is done)
+    int threads = shape.threads > 0 ? shape.threads : (FETCH ? 64 : 128);   // measured: 64 beats 128 and 256 when streaming (a block holds its shared memory until its slowest thread is done)
     if (threads > 256) threads = 256;
     if (shape.threads <= 0)
         while (threads > 32 && per_thread * threads > 44 * 1024) threads >>= 1;
     const size_t smem = (per_thread * threads + 15) & ~static_cast<size_t>(15);
-    auto kernel = args.pop.layout == kLayoutNP ? shuffle_async_kernel<TA, TB, kLayoutNP> : shuffle_async_kernel<TA, TB, kLayoutPN>;
+    auto kernel = args.pop.layout == kLayoutNP ? shuffle_async_kernel<TA, TB, kLayoutNP, FETCH> : shuffle_async_kernel<TA, TB, kLayoutPN, FETCH>;
     KernelFit fit;
     cudaError_t err = kernel_fit(reinterpret_cast<const void *>(kernel), threads, smem, &fit);
     if (err != cudaSuccess) return err;
@@ -207,16 +228,17 @@ cudaError_t launch_shuffle_async_typed(const ShuffleArgs &args, const LaunchShap
     return cudaGetLastError();
 }
 
-inline cudaError_t launch_shuffle_async(const ShuffleArgs &args, int a_dtype, int b_dtype, const LaunchShape &shape,
-                                        cudaStream_t stream, bool *supported)
+template <bool FETCH>
+cudaError_t launch_shuffle_async(const ShuffleArgs &args, int a_dtype, int b_dtype, const LaunchShape &shape,
+                                 cudaStream_t stream, bool *supported)
 {
     *supported = true;
-    if (a_dtype == kDtypeF32 && b_dtype == kDtypeNone) return launch_shuffle_async_typed<F32, NoStack>(args, shape, stream);
-    if (a_dtype == kDtypeBF16 && b_dtype == kDtypeNone) return launch_shuffle_async_typed<BF16, NoStack>(args, shape, stream);
-    if (a_dtype == kDtypeF32 && b_dtype == kDtypeF32) return launch_shuffle_async_typed<F32, F32>(args, shape, stream);
-    if (a_dtype == kDtypeBF16 && b_dtype == kDtypeF32) return launch_shuffle_async_typed<BF16, F32>(args, shape, stream);
-    if (a_dtype == kDtypeBF16 && b_dtype == kDtypeBF16) return launch_shuffle_async_typed<BF16, BF16>(args, shape, stream);
-    if (a_dtype == kDtypeF32 && b_dtype == kDtypeBF16) return launch_shuffle_async_typed<F32, BF16>(args, shape, stream);
+    if (a_dtype == kDtypeF32 && b_dtype == kDtypeNone) return launch_shuffle_async_typed<F32, NoStack, FETCH>(args, shape, stream);
+    if (a_dtype == kDtypeBF16 && b_dtype == kDtypeNone) return launch_shuffle_async_typed<BF16, NoStack, FETCH>(args, shape, stream);
+    if (a_dtype == kDtypeF32 && b_dtype == kDtypeF32) return launch_shuffle_async_typed<F32, F32, FETCH>(args, shape, stream);
+    if (a_dtype == kDtypeBF16 && b_dtype == kDtypeF32) return launch_shuffle_async_typed<BF16, F32, FETCH>(args, shape, stream);
+    if (a_dtype == kDtypeBF16 && b_dtype == kDtypeBF16) return launch_shuffle_async_typed<BF16, BF16, FETCH>(args, shape, stream);
+    if (a_dtype == kDtypeF32 && b_dtype == kDtypeBF16) return launch_shuffle_async_typed<F32, BF16, FETCH>(args, shape, stream);
     *supported = false;
     return cudaSuccess;
 }
