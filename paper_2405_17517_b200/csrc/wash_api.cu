@@ -84,6 +84,7 @@ struct wash_ctx {
     uint32_t *status_dev = nullptr;
     wash_stats *stats_dev = nullptr;       // for wash_step_host
     wash::StatSlot *stat_slots_dev = nullptr;
+    double expected_selected = 0.0;        // sum over tensors of numel * thr / 2^32, for the current thresholds
     void *avg_dev = nullptr;               // for wash_step_host, allocated on first use
     size_t avg_bytes = 0;
 
@@ -143,6 +144,9 @@ int sync_table(wash_ctx *ctx, double p, const double *p_layer, cudaStream_t stre
         }
     }
     if (!changed) return WASH_OK;
+    ctx->expected_selected = 0.0;
+    for (int s = 0; s < ctx->n_seg; ++s)
+        ctx->expected_selected += static_cast<double>(ctx->seg_host[s].numel) * static_cast<double>(ctx->seg_host[s].thr) / 4294967296.0;
     const int slot = ctx->next_slot;
     ctx->next_slot = (slot + 1) % kSlots;
     if (ctx->slot_used[slot]) {   // the copy that last read this slot must be done
@@ -202,7 +206,16 @@ int shuffle_impl(wash_ctx *ctx, int which, uint64_t step, double p, const double
     args.step_lo = static_cast<uint32_t>(step);
     args.step_hi8 = static_cast<uint32_t>(step >> 32) << 8;
     args.stats = reinterpret_cast<unsigned long long *>(stats);
-    args.stat_slots = ctx->stat_slots_dev;
+    // Counters: blocks that selected something add to the caller's two words directly when
+    // that stays well below one atomic per nanosecond on one address (measured limit);
+    // otherwise through the partial-sum slots and a small flush kernel.
+    {
+        const double bytes = static_cast<double>(ctx->N) * static_cast<double>(ctx->padded_P) *
+                             (elem_bytes(a_dtype) + (b ? elem_bytes(b_dtype) : 0));
+        const double kernel_ns = bytes / 6000.0 + 2000.0;
+        const double reporting_blocks = std::fmin(ctx->expected_selected, static_cast<double>(ctx->n_groups) / 64.0);
+        args.stat_slots = (2.0 * reporting_blocks / kernel_ns > 0.35) ? ctx->stat_slots_dev : nullptr;
+    }
     args.status = ctx->status_dev;
     bool supported = false;
     cudaError_t err = wash::launch_shuffle(args, a_dtype, b_dtype, ctx->mode, ctx->shape, stream, &supported);

