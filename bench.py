@@ -425,6 +425,20 @@ def run_sweep(args) -> None:
     modes = {"stream": B.WASH_MODE_STREAM, "sparse": B.WASH_MODE_SPARSE, "registers": B.WASH_MODE_STREAM_REGISTERS,
              "staged": B.WASH_MODE_STREAM_STAGED}
     stream = torch.cuda.current_stream()
+    # integer-pipe ceiling of the mask: Philox blocks per second with no memory traffic
+    chk = torch.zeros(1, dtype=torch.int32, device="cuda")
+    n_blocks = 1 << 28
+    for _ in range(3):
+        B.wash_philox_probe(n_blocks, SEED, chk, 0, stream)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for _ in range(5):
+        B.wash_philox_probe(n_blocks, SEED, chk, 0, stream)
+    e1.record(stream)
+    torch.cuda.synchronize()
+    rate = 5 * n_blocks / (e0.elapsed_time(e1) * 1e-3)
+    print(json.dumps({"philox_blocks_per_s": rate, "mask_coordinates_per_s": 4 * rate,
+                      "note": "ceiling of the mask draw alone; N*16 bytes of fp32 stack per block"}), flush=True)
     pick = lambda text, default, conv: [conv(x) for x in text.split(",")] if text else default
     for N in pick(args.sweep_N, [2, 4, 8, 16, 32], int):
         for logP in pick(args.sweep_logP, [20, 24, 27], int):

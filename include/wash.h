@@ -259,6 +259,14 @@ int wash_check(wash_ctx *ctx, void *stream);
 /* Message for the calling thread's most recent error (never NULL). */
 const char *wash_last_error(void);
 
+/* Integer-pipe ceiling of the shuffle's mask: a kernel that does nothing but draw
+ * n_blocks Philox4x32-10 blocks (the mask of 4*n_blocks coordinates, counters as in
+ * wash_shuffle for tensor 0 at step 0 with key = seed) and folds them into one word,
+ * which it adds to *dev_checksum (DEVICE, uint32, caller-zeroed; may be NULL).  Timing it
+ * gives the rate at which masks can be drawn when memory costs nothing, i.e. the bound
+ * that takes over from HBM for small N.  No stack is touched.  Diagnostic only. */
+int wash_philox_probe(uint64_t n_blocks, uint64_t seed, uint32_t *dev_checksum, int32_t device, void *stream);
+
 /* Number of kernels this library has launched in this process. */
 uint64_t wash_launch_count(void);
 

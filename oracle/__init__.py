@@ -28,7 +28,12 @@ SCHEDULE_DECREASING, SCHEDULE_CONSTANT, SCHEDULE_INCREASING = 0, 1, 2
 
 
 def build(force: bool = False) -> str:
-    """Compile the oracle (gcc, no fast-math, no FMA contraction) if it is stale."""
+    """Compile the oracle (gcc, no fast-math, no FMA contraction) if it is stale.
+    WASH_ORACLE_LIB names an already built library to load instead (used by the test
+    that checks the pins against deliberately broken copies of the oracle)."""
+    override = os.environ.get("WASH_ORACLE_LIB")
+    if override:
+        return override
     with _lock:
         stale = (not os.path.exists(_LIB)) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC)
         if force or stale:

@@ -68,6 +68,7 @@ def load() -> ctypes.CDLL:
     L.wash_consensus_sq.argtypes = [vp, i32, i32, i32, vp, vp]
     L.wash_step_host.argtypes = [vp, i32, vp, vp, vp, u64, dbl, dblp, u64, ctypes.c_float, vp, ctypes.POINTER(wash_stats)]
     L.wash_check.argtypes = [vp, vp]
+    L.wash_philox_probe.argtypes = [u64, u64, vp, i32, vp]
     L.wash_last_error.restype = ctypes.c_char_p
     L.wash_launch_count.restype = ctypes.c_uint64
     L.wash_shuffle_noalloc.argtypes = [i32, i32, i64p, i32, i32, vp, i64, u64, dbl, dblp, u64, i32, vp, vp]
@@ -222,6 +223,10 @@ def wash_shuffle_noalloc(N: int, numel, layout: int, dtype: int, dev_stack, n_el
 
 def wash_noalloc_last_error() -> str:
     return load().wash_noalloc_last_error().decode()
+
+
+def wash_philox_probe(n_blocks: int, seed: int = 0, dev_checksum=None, device: int = 0, stream=None) -> None:
+    _check(load().wash_philox_probe(n_blocks, seed, _ptr(dev_checksum), device, _stream(stream)))
 
 
 def wash_check(ctx, stream=None) -> None:

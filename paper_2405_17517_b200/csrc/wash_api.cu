@@ -538,6 +538,16 @@ int wash_check(wash_ctx *ctx, void *stream_v)
     return WASH_OK;
 }
 
+int wash_philox_probe(uint64_t n_blocks, uint64_t seed, uint32_t *dev_checksum, int32_t device, void *stream_v)
+{
+    if (device < 0) return fail(WASH_ERR_ARG, "device = %d", device);
+    DeviceGuard guard(device);
+    if (guard.err != cudaSuccess) return cuda_fail(guard.err, "cudaSetDevice");
+    cudaError_t err = wash::launch_philox_probe(n_blocks, seed, dev_checksum, static_cast<cudaStream_t>(stream_v));
+    if (err != cudaSuccess) return cuda_fail(err, "philox probe launch");
+    return WASH_OK;
+}
+
 const char *wash_last_error(void) { return g_last_error.c_str(); }
 
 uint64_t wash_launch_count(void) { return wash::launch_count(); }

@@ -78,6 +78,8 @@ cudaError_t launch_shuffle(const ShuffleArgs &args, int a_dtype, int b_dtype, in
 cudaError_t launch_reduce(const ReduceArgs &args, int op, int dtype, int out_dtype,
                           const LaunchShape &shape, cudaStream_t stream, bool *supported);
 
+cudaError_t launch_philox_probe(unsigned long long n_blocks, uint64_t seed, uint32_t *checksum, cudaStream_t stream);
+
 // true if a streaming shuffle kernel was compiled for this population size
 bool has_unrolled_kernels(int N);
 
