@@ -224,7 +224,7 @@ def run_ours(args, rank: int, world: int, local_rank: int) -> None:
             from paper_2405_17517_b200 import build as wash_build
             wash_build.build()
     dist = None
-    if world > 1:
+    if world > 1 or os.environ.get("WASH_BENCH_DIST") == "1":   # the second form exercises the multi-rank path on one GPU
         import torch.distributed as dist_mod
         dist = dist_mod
         torch.cuda.set_device(local_rank)
