@@ -11,7 +11,8 @@
 //
 // One group per thread, one trip per thread (the block scheduler refills the SM as
 // blocks retire).  Block image in shared memory:
-//   [N][P]: vector j of thread t at (j*T + t) * vec      (T = threads per block)
+//   [N][P]: vector j of thread t at (j*T + t) * vec      (T = threads per block); fp32 vectors
+//           are copied by their own thread, bf16 rows cooperatively in 16-byte pieces
 //   [P][N]: the block's T*4N elements are contiguous in global memory and are copied
 //           as they lie, vector k*T + t by thread t; thread t's coordinate c of model n
 //           is element (4t + c)*N + n of that image.
@@ -42,7 +43,18 @@ __device__ __forceinline__ void async_fetch(uint32_t image, void *base, const Po
 {
     constexpr int kVec = T::kBytes * 4;
     const uint32_t t = threadIdx.x, T_ = blockDim.x;
-    if (LAYOUT == kLayoutNP) {
+    if (LAYOUT == kLayoutNP && kVec == 8) {
+        // bf16: a row of the image (T groups of 8 bytes) is contiguous in global memory too;
+        // copy it in 16-byte pieces, thread t taking pieces t, t + T, ... of the N rows (the
+        // number of groups in a block is even, so a row is a whole number of pieces)
+        const uint32_t per_row = groups_in_block / 2, pieces = per_row * n_models;
+        const char *row0 = group_vec_ptr<T, LAYOUT>(base, pop, g_block, 0);
+        const size_t row_bytes = static_cast<size_t>(pop.padded_P) * T::kBytes;
+        for (uint32_t k = t; k < pieces; k += T_) {
+            const uint32_t j = k / per_row, piece = k - j * per_row;
+            cp_async<16>(image + j * T_ * kVec + piece * 16, row0 + j * row_bytes + piece * 16);
+        }
+    } else if (LAYOUT == kLayoutNP) {
         if (t < groups_in_block) {
             // model j's vector of this thread's group: one row further in global memory,
             // one row of T vectors further in the image
@@ -131,7 +143,8 @@ __global__ void __launch_bounds__(256, 5) shuffle_async_kernel(const __grid_cons
     // block-wide barrier instead.
     if constexpr (FETCH) {
         cp_async_wait_all();
-        if (LAYOUT == kLayoutPN) __syncthreads_or(sel != 0);
+        constexpr bool kSharedCopies = LAYOUT == kLayoutPN || TA::kBytes == 2 || (kHasB && TB::kBytes == 2);   // a group's bytes were copied by other threads
+        if (kSharedCopies) __syncthreads();
         else __syncwarp();
     }
 
@@ -139,15 +152,15 @@ __global__ void __launch_bounds__(256, 5) shuffle_async_kernel(const __grid_cons
     // lanes 32 at a time: with a few selected coordinates per warp (p around 0.01-0.1)
     // one round serves them all, instead of one divergent pass per coordinate slot.
     const uint32_t lane = threadIdx.x & 31u, warp_base = threadIdx.x & ~31u;
-    const uint32_t mine = __popc(sel);
-    uint32_t upto = mine;   // inclusive prefix sum over the lanes
+    if (__any_sync(0xFFFFFFFFu, sel != 0)) {   // most warps have nothing selected at small p
+        const uint32_t mine = __popc(sel);
+        uint32_t upto = mine;   // inclusive prefix sum over the lanes
 #pragma unroll
-    for (int d = 1; d < 32; d <<= 1) {
-        const uint32_t v = __shfl_up_sync(0xFFFFFFFFu, upto, d);
-        if (lane >= static_cast<uint32_t>(d)) upto += v;
-    }
-    const uint32_t total = __shfl_sync(0xFFFFFFFFu, upto, 31);
-    if (total != 0) {
+        for (int d = 1; d < 32; d <<= 1) {
+            const uint32_t v = __shfl_up_sync(0xFFFFFFFFu, upto, d);
+            if (lane >= static_cast<uint32_t>(d)) upto += v;
+        }
+        const uint32_t total = __shfl_sync(0xFFFFFFFFu, upto, 31);
         uint8_t *list = s_list + (threadIdx.x >> 5) * 128;   // entry = owner lane * 4 + coordinate slot
         uint32_t pos = upto - mine;
 #pragma unroll
