@@ -120,3 +120,55 @@ def test_config5_large_flat_population_on_sampled_ranges(N, logP, p, layout):
     q = oracle.threshold(p) / 2.0 ** 32
     assert abs(sel - P * q) <= 5 * np.sqrt(P * q * (1 - q)) + 1e-9
     pop.close()
+
+
+def test_row_of_more_than_two_to_the_31_coordinates():
+    """Largest rows: one tensor of 2^31 + 24 coordinates per model (N = 2, 17 GB).  Byte
+    offsets exceed 2^32 and coordinate indices 2^31; sampled ranges, among them the last
+    coordinates of the row, must match the oracle."""
+    free, _ = torch.cuda.mem_get_info()
+    P, N = (1 << 31) + 24, 2
+    if free < N * P * 4 + (2 << 30):
+        pytest.skip("not enough free device memory for a 17 GB stack")
+    pop = B.Population(N, [P], B.WASH_LAYOUT_NP, 0)
+    gen = torch.Generator(device="cuda").manual_seed(5)
+    stack = torch.empty(N * pop.padded_P, device="cuda", dtype=torch.float32)
+    for n in range(N):     # fill in pieces: randn of 2^31 elements at once needs a second buffer of that size
+        for lo in range(0, pop.padded_P, 1 << 28):
+            hi = min(pop.padded_P, lo + (1 << 28))
+            stack[n * pop.padded_P + lo:n * pop.padded_P + hi].normal_(0.0, 0.05, generator=gen)
+    pop.bind(B.WASH_STACK_PARAMS, stack)
+    view = stack.view(N, pop.padded_P)
+    rng = np.random.default_rng(3)
+    starts = (rng.integers(0, (P - 4096) // 4, 20) * 4).tolist() + [0, (1 << 31) - 2048, P - 4096, P - 24 - 4072]
+    before = [view[:, s:s + 4096].contiguous().cpu().numpy() for s in starts]
+    stats = torch.zeros(2, dtype=torch.int64, device="cuda")
+    for mode in (B.WASH_MODE_STREAM, B.WASH_MODE_SPARSE):
+        B.wash_set_mode(pop.ctx, mode)
+        B.wash_shuffle(pop.ctx, 1 + mode, 0.01, None, seed=21, stats=stats)
+    torch.cuda.synchronize()
+    B.wash_check(pop.ctx)
+    for s, b in zip(starts, before):
+        width = min(4096, P - s)
+        seg = oracle.Population(N, [width], tensor_id=[0], coord_begin=[s])
+        want = np.ascontiguousarray(b[:, :width])
+        for mode in (B.WASH_MODE_STREAM, B.WASH_MODE_SPARSE):
+            oracle.shuffle(seg, want, 0.01, seed=21, step=1 + mode)
+        got = view[:, s:s + width].contiguous().cpu().numpy()
+        assert (got.view(np.uint32) == want.view(np.uint32)).all(), s
+    q = oracle.threshold(0.01) / 2.0 ** 32
+    assert abs(int(stats[0]) - 2 * P * q) <= 5 * np.sqrt(2 * P * q)
+    pop.close()
+
+
+def test_segment_at_the_top_of_the_coordinate_and_tensor_ranges():
+    """Counters near their limits: a shard holding the last 4096 coordinates of a tensor of
+    2^32 coordinates whose index is 2^32 - 1, at a step just below 2^56."""
+    N = 6
+    c = Case(N, [4096, 100], 0, "f32", "f32", seed=2, tensor_id=[0xFFFFFFFF, 7], coord_begin=[(1 << 32) - 4096, 8])
+    step = (1 << 56) - 1
+    B.wash_shuffle_both(c.gpu.ctx, step, 0.5, None, seed=0xFFFFFFFFFFFFFFFF, stats=c.stats_dev)
+    st = oracle.shuffle(c.ora, c.host, 0.5, seed=0xFFFFFFFFFFFFFFFF, step=step, stack2=c.host_opt)
+    c.assert_equal("top of ranges")
+    assert c.gpu_stats() == st
+    c.close()

@@ -210,3 +210,27 @@ def test_argument_and_state_errors():
     assert (t == 0).all()
     B.wash_check(ctx)
     B.wash_destroy(ctx)
+
+
+def test_resume_from_a_host_copy_continues_bit_identically():
+    """The shuffle is a pure function of (stack bits, seed, step, tensor table, p): 20 steps
+    in one context equal 10 steps, a round trip of the stacks through host memory into a
+    fresh context, and 10 more steps."""
+    N, numel = 5, [3000, 17, 640]
+    a = Case(N, numel, 0, "f32", "f32", seed=31)
+    for step in range(20):
+        B.wash_shuffle_both(a.gpu.ctx, step, 0.05, None, seed=77)
+    b = Case(N, numel, 0, "f32", "f32", seed=31)
+    for step in range(10):
+        B.wash_shuffle_both(b.gpu.ctx, step, 0.05, None, seed=77)
+    torch.cuda.synchronize()
+    saved, saved_opt = b.dev.cpu(), b.dev_opt.cpu()
+    b.close()
+    c = Case(N, numel, 0, "f32", "f32", seed=99)          # different contents, overwritten below
+    c.dev.copy_(saved); c.dev_opt.copy_(saved_opt)
+    for step in range(10, 20):
+        B.wash_shuffle_both(c.gpu.ctx, step, 0.05, None, seed=77)
+    torch.cuda.synchronize()
+    assert torch.equal(a.dev.view(torch.int32), c.dev.view(torch.int32))
+    assert torch.equal(a.dev_opt.view(torch.int32), c.dev_opt.view(torch.int32))
+    a.close(); c.close()
