@@ -197,7 +197,10 @@ enum wash_step_ops { WASH_OP_SHUFFLE = 1, WASH_OP_EMA = 2, WASH_OP_AVERAGE = 4 }
  * the stacks back to the same host buffers and the average (row of padded_P elements
  * of the parameter dtype) to host_avg (may be NULL unless WASH_OP_AVERAGE), and waits
  * for the stream.  host_stats (may be NULL) receives this call's counters.  The
- * device stacks must be bound; they serve as staging and hold the results too. */
+ * device stacks must be bound; they serve as staging and hold the results too.
+ * Populations of 2^20 coordinates per model and more are processed in eight coordinate
+ * ranges on two internal copy streams, so that the copy in of one range, the kernels on
+ * the previous one and the copy out of the one before overlap; the result is the same. */
 int wash_step_host(wash_ctx *ctx, int32_t ops, void *host_params, void *host_opt, void *host_avg,
                    uint64_t step, double p, const double *p_layer, uint64_t seed, float alpha,
                    void *stream, wash_stats *host_stats);

@@ -40,6 +40,7 @@ int cuda_fail(cudaError_t err, const char *what)
 }
 
 constexpr int kSlots = 4;   // pinned staging slots for table uploads
+constexpr int kPipeChunks = 8;   // wash_step_host cuts a large population into this many coordinate ranges
 
 // makes `device` current for the lifetime of the guard
 struct DeviceGuard {
@@ -87,6 +88,8 @@ struct wash_ctx {
     double expected_selected = 0.0;        // sum over tensors of numel * thr / 2^32, for the current thresholds
     void *avg_dev = nullptr;               // for wash_step_host, allocated on first use
     size_t avg_bytes = 0;
+    cudaStream_t copy_in = nullptr, copy_out = nullptr;   // for wash_step_host's pipeline, created on first use
+    cudaEvent_t pipe_event[2 * kPipeChunks + 2] = {};
 
     int mode = WASH_MODE_STREAM;
     wash::LaunchShape shape{0, 0, 148};
@@ -104,6 +107,10 @@ void release(wash_ctx *ctx)
     if (ctx->stats_dev) cudaFree(ctx->stats_dev);
     if (ctx->stat_slots_dev) cudaFree(ctx->stat_slots_dev);
     if (ctx->avg_dev) cudaFree(ctx->avg_dev);
+    if (ctx->copy_in) cudaStreamDestroy(ctx->copy_in);
+    if (ctx->copy_out) cudaStreamDestroy(ctx->copy_out);
+    for (cudaEvent_t e : ctx->pipe_event)
+        if (e) cudaEventDestroy(e);
     for (int s = 0; s < kSlots; ++s) {
         if (ctx->seg_pinned[s]) cudaFreeHost(ctx->seg_pinned[s]);
         if (ctx->slot_event[s]) cudaEventDestroy(ctx->slot_event[s]);
@@ -173,7 +180,7 @@ int ensure_table(wash_ctx *ctx, cudaStream_t stream)
 
 // which: 0 = parameters, 1 = optimizer state, 2 = both
 int shuffle_impl(wash_ctx *ctx, int which, uint64_t step, double p, const double *p_layer, uint64_t seed,
-                 void *stream_v, wash_stats *stats)
+                 void *stream_v, wash_stats *stats, uint32_t group_lo = 0, uint32_t group_hi = 0xFFFFFFFFu)
 {
     if (!ctx) return fail(WASH_ERR_ARG, "ctx is NULL");
     if (step >> 56) return fail(WASH_ERR_ARG, "step must be below 2^56");
@@ -201,6 +208,8 @@ int shuffle_impl(wash_ctx *ctx, int which, uint64_t step, double p, const double
     args.pop = view_of(ctx);
     args.a = a;
     args.b = b;
+    args.group_lo = group_lo;
+    args.group_hi = group_hi < ctx->n_groups ? group_hi : ctx->n_groups;
     args.key0 = static_cast<uint32_t>(seed);
     args.key1 = static_cast<uint32_t>(seed >> 32);
     args.step_lo = static_cast<uint32_t>(step);
@@ -225,7 +234,7 @@ int shuffle_impl(wash_ctx *ctx, int which, uint64_t step, double p, const double
 }
 
 int reduce_impl(wash_ctx *ctx, int op, int stack, void *out, int out_dtype, float alpha, int tensor_lo,
-                int tensor_hi, double *sq_out, void *stream_v)
+                int tensor_hi, double *sq_out, void *stream_v, uint32_t group_lo = 0, uint32_t group_hi = 0xFFFFFFFFu)
 {
     if (!ctx) return fail(WASH_ERR_ARG, "ctx is NULL");
     if (stack != WASH_STACK_PARAMS && stack != WASH_STACK_OPT) return fail(WASH_ERR_ARG, "stack must be 0 or 1");
@@ -243,6 +252,9 @@ int reduce_impl(wash_ctx *ctx, int op, int stack, void *out, int out_dtype, floa
     args.one_minus_alpha = 1.0f - alpha;
     args.group_lo = ctx->seg_host[static_cast<size_t>(tensor_lo)].group_begin;
     args.group_hi = ctx->seg_host[static_cast<size_t>(tensor_hi) - 1].group_end;
+    if (group_lo > args.group_lo) args.group_lo = group_lo;   // optional narrowing to a range of groups
+    if (group_hi < args.group_hi) args.group_hi = group_hi;
+    if (args.group_lo >= args.group_hi) return WASH_OK;
     args.sq_out = sq_out;
     args.status = ctx->status_dev;
     bool supported = false;
@@ -478,6 +490,10 @@ int wash_step_host(wash_ctx *ctx, int32_t ops, void *host_params, void *host_opt
     cudaError_t err;
     if ((ops & WASH_OP_AVERAGE) && ctx->avg_bytes < avg_bytes) {
         if (ctx->avg_dev) cudaFree(ctx->avg_dev);
+    if (ctx->copy_in) cudaStreamDestroy(ctx->copy_in);
+    if (ctx->copy_out) cudaStreamDestroy(ctx->copy_out);
+    for (cudaEvent_t e : ctx->pipe_event)
+        if (e) cudaEventDestroy(e);
         ctx->avg_dev = nullptr;
         ctx->avg_bytes = 0;
         if ((err = cudaMalloc(&ctx->avg_dev, avg_bytes)) != cudaSuccess) {
@@ -486,11 +502,88 @@ int wash_step_host(wash_ctx *ctx, int32_t ops, void *host_params, void *host_opt
         }
         ctx->avg_bytes = avg_bytes;
     }
+    int rc;
+    wash_stats st = {0, 0};
+    // Large populations go through in kPipeChunks coordinate ranges so that the copy of one
+    // range to the device, the kernels on the previous one and the copy of the one before
+    // back to the host overlap (the PCIe link is full duplex, and the draws are keyed by
+    // global coordinates, so a range can be processed on its own).
+    if (ctx->mode != WASH_MODE_STREAM_STAGED && ctx->n_groups >= (1u << 18)) {
+        if (!ctx->copy_in) {
+            if ((err = cudaStreamCreateWithFlags(&ctx->copy_in, cudaStreamNonBlocking)) != cudaSuccess ||
+                (err = cudaStreamCreateWithFlags(&ctx->copy_out, cudaStreamNonBlocking)) != cudaSuccess)
+                return cuda_fail(err, "cudaStreamCreate");
+            for (cudaEvent_t &e : ctx->pipe_event)
+                if ((err = cudaEventCreateWithFlags(&e, cudaEventDisableTiming)) != cudaSuccess) return cuda_fail(err, "cudaEventCreate");
+        }
+        cudaEvent_t *ev_in = ctx->pipe_event, *ev_done = ctx->pipe_event + kPipeChunks;
+        cudaEvent_t ev_start = ctx->pipe_event[2 * kPipeChunks], ev_out = ctx->pipe_event[2 * kPipeChunks + 1];
+        if ((ops & WASH_OP_SHUFFLE) && (err = cudaMemsetAsync(ctx->stats_dev, 0, sizeof(wash_stats), stream)) != cudaSuccess) return cuda_fail(err, "cudaMemsetAsync(stats)");
+        if ((ops & WASH_OP_AVERAGE) && (err = cudaMemsetAsync(ctx->avg_dev, 0, avg_bytes, stream)) != cudaSuccess) return cuda_fail(err, "cudaMemsetAsync(average row)");
+        // the copy streams start after whatever the caller's stream has queued so far
+        if ((err = cudaEventRecord(ev_start, stream)) != cudaSuccess ||
+            (err = cudaStreamWaitEvent(ctx->copy_in, ev_start, 0)) != cudaSuccess ||
+            (err = cudaStreamWaitEvent(ctx->copy_out, ev_start, 0)) != cudaSuccess) return cuda_fail(err, "pipeline set-up");
+        const uint32_t per = ((ctx->n_groups + kPipeChunks - 1) / kPipeChunks + 255u) & ~255u;   // groups per range
+        // moves the elements [e0, e0 + count) of every model between a host and the device stack
+        auto copy_range = [&](void *dst, const void *src, int dtype, size_t e0, size_t count, cudaMemcpyKind kind, cudaStream_t s) {
+            const size_t eb = elem_bytes(dtype);
+            if (ctx->layout == WASH_LAYOUT_NP) {
+                const size_t pitch = static_cast<size_t>(ctx->padded_P) * eb;
+                return cudaMemcpy2DAsync(static_cast<char *>(dst) + e0 * eb, pitch, static_cast<const char *>(src) + e0 * eb, pitch,
+                                         count * eb, static_cast<size_t>(ctx->N), kind, s);
+            }
+            const size_t off = e0 * ctx->N * eb;
+            return cudaMemcpyAsync(static_cast<char *>(dst) + off, static_cast<const char *>(src) + off, count * ctx->N * eb, kind, s);
+        };
+        const int od = ctx->stack_dtype[WASH_STACK_OPT];
+        for (int k = 0; k < kPipeChunks; ++k) {
+            const uint32_t g0 = static_cast<uint32_t>(k) * per;
+            if (g0 >= ctx->n_groups) break;
+            const uint32_t g1 = g0 + per < ctx->n_groups ? g0 + per : ctx->n_groups;
+            const size_t e0 = 4ull * g0, count = 4ull * (g1 - g0);
+            if ((err = copy_range(ctx->stack_ptr[WASH_STACK_PARAMS], host_params, pd, e0, count, cudaMemcpyHostToDevice, ctx->copy_in)) != cudaSuccess)
+                return cuda_fail(err, "copy of a parameter range to the device");
+            if (host_opt && (err = copy_range(ctx->stack_ptr[WASH_STACK_OPT], host_opt, od, e0, count, cudaMemcpyHostToDevice, ctx->copy_in)) != cudaSuccess)
+                return cuda_fail(err, "copy of an optimizer-state range to the device");
+            if ((err = cudaEventRecord(ev_in[k], ctx->copy_in)) != cudaSuccess || (err = cudaStreamWaitEvent(stream, ev_in[k], 0)) != cudaSuccess)
+                return cuda_fail(err, "pipeline event");
+            if (ops & WASH_OP_SHUFFLE) {
+                rc = shuffle_impl(ctx, host_opt ? 2 : 0, step, p, p_layer, seed, stream, ctx->stats_dev, g0, g1);
+                if (rc != WASH_OK) return rc;
+            }
+            if (ops & WASH_OP_EMA) {
+                rc = reduce_impl(ctx, wash::kOpEma, WASH_STACK_PARAMS, nullptr, WASH_F32, alpha, 0, ctx->n_seg, nullptr, stream, g0, g1);
+                if (rc != WASH_OK) return rc;
+            }
+            if (ops & WASH_OP_AVERAGE) {
+                rc = reduce_impl(ctx, wash::kOpAverage, WASH_STACK_PARAMS, ctx->avg_dev, pd, 0.0f, 0, ctx->n_seg, nullptr, stream, g0, g1);
+                if (rc != WASH_OK) return rc;
+            }
+            if ((err = cudaEventRecord(ev_done[k], stream)) != cudaSuccess || (err = cudaStreamWaitEvent(ctx->copy_out, ev_done[k], 0)) != cudaSuccess)
+                return cuda_fail(err, "pipeline event");
+            if ((err = copy_range(host_params, ctx->stack_ptr[WASH_STACK_PARAMS], pd, e0, count, cudaMemcpyDeviceToHost, ctx->copy_out)) != cudaSuccess)
+                return cuda_fail(err, "copy of a parameter range to the host");
+            if (host_opt && (err = copy_range(host_opt, ctx->stack_ptr[WASH_STACK_OPT], od, e0, count, cudaMemcpyDeviceToHost, ctx->copy_out)) != cudaSuccess)
+                return cuda_fail(err, "copy of an optimizer-state range to the host");
+            if ((ops & WASH_OP_AVERAGE) &&
+                (err = cudaMemcpyAsync(static_cast<char *>(host_avg) + e0 * elem_bytes(pd), static_cast<char *>(ctx->avg_dev) + e0 * elem_bytes(pd),
+                                       count * elem_bytes(pd), cudaMemcpyDeviceToHost, ctx->copy_out)) != cudaSuccess)
+                return cuda_fail(err, "copy of an average range to the host");
+        }
+        // the caller's stream continues only when the last range is back on the host
+        if ((err = cudaEventRecord(ev_out, ctx->copy_out)) != cudaSuccess || (err = cudaStreamWaitEvent(stream, ev_out, 0)) != cudaSuccess)
+            return cuda_fail(err, "pipeline event");
+        if ((ops & WASH_OP_SHUFFLE) && (err = cudaMemcpyAsync(&st, ctx->stats_dev, sizeof st, cudaMemcpyDeviceToHost, stream)) != cudaSuccess)
+            return cuda_fail(err, "copy of the counters to the host");
+        if ((err = cudaStreamSynchronize(stream)) != cudaSuccess) return cuda_fail(err, "cudaStreamSynchronize");
+        if (host_stats) *host_stats = st;
+        return WASH_OK;
+    }
     if ((err = cudaMemcpyAsync(ctx->stack_ptr[WASH_STACK_PARAMS], host_params, p_bytes, cudaMemcpyHostToDevice, stream)) != cudaSuccess)
         return cuda_fail(err, "copy of the parameter stack to the device");
     if (host_opt && (err = cudaMemcpyAsync(ctx->stack_ptr[WASH_STACK_OPT], host_opt, o_bytes, cudaMemcpyHostToDevice, stream)) != cudaSuccess)
         return cuda_fail(err, "copy of the optimizer-state stack to the device");
-    int rc;
     if (ops & WASH_OP_SHUFFLE) {
         if ((err = cudaMemsetAsync(ctx->stats_dev, 0, sizeof(wash_stats), stream)) != cudaSuccess) return cuda_fail(err, "cudaMemsetAsync(stats)");
         rc = shuffle_impl(ctx, host_opt ? 2 : 0, step, p, p_layer, seed, stream, ctx->stats_dev);
@@ -513,7 +606,6 @@ int wash_step_host(wash_ctx *ctx, int32_t ops, void *host_params, void *host_opt
         return cuda_fail(err, "copy of the optimizer-state stack to the host");
     if ((ops & WASH_OP_AVERAGE) && (err = cudaMemcpyAsync(host_avg, ctx->avg_dev, avg_bytes, cudaMemcpyDeviceToHost, stream)) != cudaSuccess)
         return cuda_fail(err, "copy of the average to the host");
-    wash_stats st = {0, 0};
     if ((ops & WASH_OP_SHUFFLE) && (err = cudaMemcpyAsync(&st, ctx->stats_dev, sizeof st, cudaMemcpyDeviceToHost, stream)) != cudaSuccess)
         return cuda_fail(err, "copy of the counters to the host");
     if ((err = cudaStreamSynchronize(stream)) != cudaSuccess) return cuda_fail(err, "cudaStreamSynchronize");

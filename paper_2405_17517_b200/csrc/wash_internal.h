@@ -46,6 +46,7 @@ struct ShuffleArgs {
     PopView pop;
     void *a;                      // first stack (device)
     void *b;                      // second stack or nullptr
+    uint32_t group_lo, group_hi;  // groups of a row to process (whole row: 0 .. n_groups)
     uint32_t key0, key1;          // seed
     uint32_t step_lo, step_hi8;   // step & 0xFFFFFFFF, (step >> 32) << 8
     unsigned long long *stats;    // device-accessible {selected, moved} or nullptr

@@ -146,6 +146,8 @@ extern "C" int wash_shuffle_noalloc(int32_t N, int32_t n_tensors, const int64_t 
             args.pop.tile_first = tile_dev;
             args.a = dev_stack;
             args.b = nullptr;
+            args.group_lo = 0;
+            args.group_hi = n_groups;
             args.key0 = static_cast<uint32_t>(seed);
             args.key1 = static_cast<uint32_t>(seed >> 32);
             args.step_lo = static_cast<uint32_t>(step);

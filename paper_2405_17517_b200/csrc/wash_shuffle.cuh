@@ -54,7 +54,7 @@ __global__ void __launch_bounds__(256) shuffle_kernel(const __grid_constant__ Sh
     uint32_t *s_val = smem + n_models * ts + threadIdx.x;       // [n][ts]
     uint32_t selected = 0, moved = 0;
     const uint64_t stride = static_cast<uint64_t>(gridDim.x) * blockDim.x;
-    for (uint64_t g = static_cast<uint64_t>(blockIdx.x) * blockDim.x + threadIdx.x; g < a.pop.n_groups; g += stride) {
+    for (uint64_t g = a.group_lo + static_cast<uint64_t>(blockIdx.x) * blockDim.x + threadIdx.x; g < a.group_hi; g += stride) {
         typename TA::vec va[kRegs];
         typename TB::vec vb[kRegs];
         if constexpr (STREAM) {
@@ -120,8 +120,8 @@ cudaError_t launch_shuffle_typed(const ShuffleArgs &args, const LaunchShape &sha
     // the most warps resident and measured fastest on the ResNet-50 populations
     const GridDefault dflt{128, true};
     if (args.pop.layout == kLayoutNP)
-        return launch_grid_stride(shuffle_kernel<N, TA, TB, kLayoutNP, STREAM>, args, args.pop.n_groups, smem_per_thread, shape, stream, dflt);
-    return launch_grid_stride(shuffle_kernel<N, TA, TB, kLayoutPN, STREAM>, args, args.pop.n_groups, smem_per_thread, shape, stream, dflt);
+        return launch_grid_stride(shuffle_kernel<N, TA, TB, kLayoutNP, STREAM>, args, args.group_hi - args.group_lo, smem_per_thread, shape, stream, dflt);
+    return launch_grid_stride(shuffle_kernel<N, TA, TB, kLayoutPN, STREAM>, args, args.group_hi - args.group_lo, smem_per_thread, shape, stream, dflt);
 }
 
 // dtype dispatch: parameters fp32 or bf16; second stack absent, fp32 or bf16

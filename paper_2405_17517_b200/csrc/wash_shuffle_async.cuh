@@ -116,8 +116,8 @@ __global__ void __launch_bounds__(256, 5) shuffle_async_kernel(const __grid_cons
     uint8_t *s_perm = s_list + 4 * T_ + threadIdx.x;   // column [n][T], used when N > 16
     uint32_t *s_col = reinterpret_cast<uint32_t *>(smem_raw) + threadIdx.x;   // !FETCH: column [n][T]
 
-    const uint64_t g_block = static_cast<uint64_t>(blockIdx.x) * T_;
-    const uint32_t groups_in_block = static_cast<uint32_t>(min(static_cast<uint64_t>(T_), a.pop.n_groups - g_block));
+    const uint64_t g_block = a.group_lo + static_cast<uint64_t>(blockIdx.x) * T_;
+    const uint32_t groups_in_block = static_cast<uint32_t>(min(static_cast<uint64_t>(T_), a.group_hi - g_block));
     if constexpr (FETCH) {
         async_fetch<TA, LAYOUT>(smem_addr(image_a), a.a, a.pop, g_block, groups_in_block, n_models);
         if constexpr (kHasB) async_fetch<TB, LAYOUT>(smem_addr(image_b), a.b, a.pop, g_block, groups_in_block, n_models);
@@ -233,7 +233,7 @@ cudaError_t launch_shuffle_async_typed(const ShuffleArgs &args, const LaunchShap
     cudaError_t err = kernel_fit(reinterpret_cast<const void *>(kernel), threads, smem, &fit);
     if (err != cudaSuccess) return err;
     if (fit.occupancy < 1) return cudaErrorLaunchOutOfResources;
-    const uint64_t grid = (static_cast<uint64_t>(args.pop.n_groups) + threads - 1) / threads;
+    const uint64_t grid = (static_cast<uint64_t>(args.group_hi - args.group_lo) + threads - 1) / threads;
     if (grid == 0) return cudaSuccess;
     if (grid > 0x7FFFFFFFull) return cudaErrorInvalidConfiguration;
     kernel<<<static_cast<unsigned>(grid), threads, smem, stream>>>(args);

@@ -129,3 +129,32 @@ def test_step_over_host_buffers():
     assert (ho.numpy().view(np.uint32) == bits(c.host_opt)).all()
     assert (havg.numpy().view(np.uint32) == want_avg.view(np.uint32)).all()
     c.close()
+
+
+@pytest.mark.parametrize("layout", [0, 1])
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_step_over_host_buffers_pipelined(dtype, layout):
+    """A population large enough for wash_step_host to cut it into coordinate ranges whose
+    copies and kernels overlap: the result must not depend on that."""
+    N, numel = 3, [700001, 9, 400000, 77]
+    c = Case(N, numel, layout, dtype, "f32", seed=14)
+    assert c.P // 4 >= 1 << 18
+    def pinned(a):
+        t = torch.from_numpy(a.reshape(-1).view(np.int16).copy() if a.dtype == np.uint16 else a.reshape(-1).copy())
+        return (t.view(torch.bfloat16) if a.dtype == np.uint16 else t).pin_memory()
+    hp, ho = pinned(c.host), pinned(c.host_opt)
+    havg = torch.zeros(c.P, dtype=hp.dtype).pin_memory()
+    ops = B.WASH_OP_SHUFFLE | B.WASH_OP_EMA | B.WASH_OP_AVERAGE
+    pl = [0.02, 1.0, 0.3, 0.0]
+    for step in (5, 6):
+        st = B.wash_step_host(c.gpu.ctx, ops, hp, ho, havg, step, 0.0, pl, seed=4, alpha=0.99)
+        want_st = oracle.shuffle(c.ora, c.host, pl, seed=4, step=step, stack2=c.host_opt)
+        oracle.papa_ema(c.ora, c.host, 0.99)
+        want_avg = np.zeros(c.P, dtype=c.host.dtype)
+        oracle.population_average(c.ora, c.host, want_avg)
+        assert st == want_st
+        assert (to_host_bits(hp) == bits(c.host)).all()
+        assert (to_host_bits(ho) == bits(c.host_opt)).all()
+        assert (to_host_bits(havg) == bits(want_avg)).all()
+    B.wash_check(c.gpu.ctx)
+    c.close()
