@@ -180,7 +180,7 @@ __global__ void __launch_bounds__(32 * kProducerWarps + 512) shuffle_tma_kernel(
         uint32_t issued = 0;
         for (uint32_t i = 0; i < my_tiles; ++i) {
             const int s = static_cast<int>(i % S);
-            // lane 0 waits for the stage to be free; the verdict is made warp-uniform
+            // lane 0 waits for the stage to be free; the answer is made warp-uniform
             // (the stage's previous tile must have landed, so that the barrier's byte count
             // is settled, and every consumer warp must have let go of it)
             int go = 1;
