@@ -129,6 +129,7 @@ __device__ __forceinline__ uint32_t group_value(const typename T::vec (&v)[CAP],
 __device__ __forceinline__ void publish_block_stats(unsigned long long *stats, StatSlot *slots, uint32_t selected, uint32_t moved)
 {
     if (!stats) return;
+    if (!__syncthreads_or(selected != 0)) return;   // most blocks have nothing to report at small p
     __shared__ uint32_t block_sum[2];
     if (threadIdx.x == 0) block_sum[0] = block_sum[1] = 0;
     __syncthreads();

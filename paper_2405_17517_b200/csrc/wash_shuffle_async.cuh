@@ -61,6 +61,7 @@ __device__ __forceinline__ void async_fetch(uint32_t image, void *base, const Po
             const char *src = group_vec_ptr<T, LAYOUT>(base, pop, g_block + t, 0);
             const size_t row_bytes = static_cast<size_t>(pop.padded_P) * T::kBytes;
             uint32_t dst = image + t * kVec;
+#pragma unroll 4
             for (int j = 0; j < n_models; ++j, src += row_bytes, dst += T_ * kVec) cp_async<kVec>(dst, src);
         }
     } else {
@@ -130,10 +131,14 @@ __global__ void __launch_bounds__(256, 5) shuffle_async_kernel(const __grid_cons
         gi = find_group(a.pop, static_cast<uint32_t>(g), a.status);
         if (gi.thr != 0 && gi.valid != 0) {
             const Philox4 w = philox4x32_10(gi.cgroup, gi.tensor_id, a.step_lo, a.step_hi8, a.key0, a.key1);
-            sel |= (static_cast<uint64_t>(w.x) < gi.thr && gi.valid > 0) ? 1u : 0u;
-            sel |= (static_cast<uint64_t>(w.y) < gi.thr && gi.valid > 1) ? 2u : 0u;
-            sel |= (static_cast<uint64_t>(w.z) < gi.thr && gi.valid > 2) ? 4u : 0u;
-            sel |= (static_cast<uint64_t>(w.w) < gi.thr && gi.valid > 3) ? 8u : 0u;
+            // word < thr with thr in [0, 2^32]: a 32-bit compare, or always when thr is 2^32
+            const uint32_t thr_lo = static_cast<uint32_t>(gi.thr);
+            const bool always = (gi.thr >> 32) != 0;
+            sel |= (w.x < thr_lo || always) ? 1u : 0u;
+            sel |= (w.y < thr_lo || always) ? 2u : 0u;
+            sel |= (w.z < thr_lo || always) ? 4u : 0u;
+            sel |= (w.w < thr_lo || always) ? 8u : 0u;
+            sel &= (1u << gi.valid) - 1u;   // coordinates beyond the tensor's end do not exist
         }
     }
     // Every thread waits for its own copies (none may be in flight when the block ends).
