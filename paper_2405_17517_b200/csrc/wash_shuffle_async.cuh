@@ -188,12 +188,22 @@ __global__ void __launch_bounds__(256, 5) shuffle_async_kernel(const __grid_cons
                 return n_models <= 16 ? static_cast<int>((perm >> (4 * n)) & 15ull) : static_cast<int>(s_perm[n * T_]);
             };
             if constexpr (FETCH) {
-                for (int n = 0; n < n_models; ++n) {
-                    const int src = source_of(n);
-                    if (src == n) continue;
-                    TA::store_elem(a.a, elem_index<LAYOUT>(a.pop, n, e), image_value<TA, LAYOUT>(image_a, n_models, t_owner, src, c));
+                // model n's value of this coordinate sits at out0 + n*out_step in the stack and at
+                // element img0 + n*img_step of the image: no multiplication left inside the loop
+                const long long out_step = LAYOUT == kLayoutNP ? a.pop.padded_P : 1;
+                const long long out0 = LAYOUT == kLayoutNP ? e : e * n_models;
+                const uint32_t img_step = LAYOUT == kLayoutNP ? T_ * 4u : 1u;
+                const uint32_t img0 = LAYOUT == kLayoutNP ? t_owner * 4u + c : (4u * t_owner + c) * n_models;
+                long long out = out0;
+                for (int n = 0; n < n_models; ++n, out += out_step) {
+                    const uint32_t src = static_cast<uint32_t>(source_of(n));
+                    if (src == static_cast<uint32_t>(n)) continue;
+                    const uint32_t from = img0 + src * img_step;
+                    TA::store_elem(a.a, out, TA::kBytes == 4 ? reinterpret_cast<const uint32_t *>(image_a)[from]
+                                                             : reinterpret_cast<const uint16_t *>(image_a)[from]);
                     if constexpr (kHasB)
-                        TB::store_elem(a.b, elem_index<LAYOUT>(a.pop, n, e), image_value<TB, LAYOUT>(image_b, n_models, t_owner, src, c));
+                        TB::store_elem(a.b, out, TB::kBytes == 4 ? reinterpret_cast<const uint32_t *>(image_b)[from]
+                                                                 : reinterpret_cast<const uint16_t *>(image_b)[from]);
                     ++moved;
                 }
             } else {
