@@ -78,6 +78,12 @@ def lib() -> ctypes.CDLL:
         L.wo_papa_all.argtypes = [popp, ctypes.c_void_p, ctypes.c_int32]
         L.wo_consensus_sq.argtypes = [popp, ctypes.c_void_p, ctypes.c_int32, ctypes.c_int32, ctypes.c_int32, f64p]
         L.wo_set_threads.argtypes = [ctypes.c_int]; L.wo_set_threads.restype = None
+        i64p = ctypes.POINTER(ctypes.c_int64)
+        L.wo_exchange_counts.argtypes = [popp, f64p, ctypes.c_uint64, ctypes.c_uint64, i64p, i64p]
+        L.wo_exchange_send.argtypes = [popp, ctypes.c_int32, ctypes.c_void_p, ctypes.c_int32, f64p, ctypes.c_uint64,
+                                       ctypes.c_uint64, ctypes.POINTER(ctypes.c_void_p), ctypes.c_int64, i64p]
+        L.wo_exchange_receive.argtypes = [popp, ctypes.c_int32, ctypes.c_void_p, ctypes.c_int32, f64p, ctypes.c_uint64,
+                                          ctypes.c_uint64, ctypes.c_void_p, ctypes.c_int64, u64p]
         _lib = L
     return _lib
 
@@ -220,3 +226,55 @@ def consensus_sq(pop: Population, stack: np.ndarray, seg_lo: int = 0, seg_hi: in
                              out.ctypes.data_as(ctypes.POINTER(ctypes.c_double))) != 0:
         raise ValueError("wo_consensus_sq: bad argument")
     return out
+
+
+def _p_seg(pop: Population, p_seg) -> np.ndarray:
+    return np.ascontiguousarray(np.broadcast_to(np.asarray(p_seg, dtype=np.float64), (pop.T,)))
+
+
+def exchange_counts(pop: Population, p_seg, seed: int, step: int):
+    """-> (need[N], selected): slots each worker's staging buffer needs in this step."""
+    p = _p_seg(pop, p_seg)
+    need = np.zeros(pop.N, dtype=np.int64)
+    sel = ctypes.c_int64(0)
+    rc = lib().wo_exchange_counts(pop.ref(), p.ctypes.data_as(ctypes.POINTER(ctypes.c_double)), seed, step,
+                                  need.ctypes.data_as(ctypes.POINTER(ctypes.c_int64)), ctypes.byref(sel))
+    if rc != 0:
+        raise ValueError("wo_exchange_counts: bad argument")
+    return need, int(sel.value)
+
+
+def exchange_send(pop: Population, self_rank: int, row: np.ndarray, p_seg, seed: int, step: int, staging) -> np.ndarray:
+    """Worker `self_rank` (holding the model `row`) fills its slots of the other workers'
+    staging buffers (a list of N arrays of the row's dtype). -> slots written per worker."""
+    _check_stack(pop, row, rows=1)
+    p = _p_seg(pop, p_seg)
+    code = _np_dtype_code(row)
+    cap = min(int(b.size) for k, b in enumerate(staging) if k != self_rank)
+    for k, b in enumerate(staging):
+        if k != self_rank and _np_dtype_code(b) != code:
+            raise TypeError("staging buffers must have the row's element type")
+    ptrs = (ctypes.c_void_p * pop.N)(*[b.ctypes.data for b in staging])
+    filled = np.zeros(pop.N, dtype=np.int64)
+    rc = lib().wo_exchange_send(pop.ref(), self_rank, row.ctypes.data, code,
+                                p.ctypes.data_as(ctypes.POINTER(ctypes.c_double)), seed, step, ptrs, cap,
+                                filled.ctypes.data_as(ctypes.POINTER(ctypes.c_int64)))
+    if rc != 0:
+        raise ValueError("wo_exchange_send: bad argument or staging buffer too small")
+    return filled
+
+
+def exchange_receive(pop: Population, self_rank: int, row: np.ndarray, p_seg, seed: int, step: int, staging_self: np.ndarray):
+    """Worker `self_rank` takes its new values out of its own staging buffer.
+    -> (selected_coords, values received)"""
+    _check_stack(pop, row, rows=1)
+    p = _p_seg(pop, p_seg)
+    if _np_dtype_code(staging_self) != _np_dtype_code(row):
+        raise TypeError("staging buffer must have the row's element type")
+    stats = (ctypes.c_uint64 * 2)(0, 0)
+    rc = lib().wo_exchange_receive(pop.ref(), self_rank, row.ctypes.data, _np_dtype_code(row),
+                                   p.ctypes.data_as(ctypes.POINTER(ctypes.c_double)), seed, step,
+                                   staging_self.ctypes.data, int(staging_self.size), stats)
+    if rc != 0:
+        raise ValueError("wo_exchange_receive: bad argument or staging buffer too small")
+    return int(stats[0]), int(stats[1])

@@ -25,6 +25,10 @@
  *   wo_papa_all           PAPA-all / DART step (section "Reducing distance to
  *                         consensus"): every model replaced by the average.
  *   wo_consensus_distance Average distance to the consensus (caption of Fig. 2).
+ *   wo_exchange_send / wo_exchange_receive / wo_exchange_counts
+ *                         The same shuffling step seen from one worker that holds one
+ *                         model (the deployment the Introduction describes: parameters
+ *                         travel peer to peer along the permutation).
  *
  * Readings taken where the paper is silent (each is a convention of this library,
  * not a fact of the paper; parity for them is pinned by the tests, not by the paper):
@@ -44,7 +48,9 @@
  * selected; per-coordinate multiset preserved (Eq. 5); Eq. 4 by Monte Carlo;
  * chi-square uniformity of pi for N = 3, 4, 5; selected fraction against the
  * binomial law; last layer untouched; brute force on tiny stacks; Eq. 2 and a
- * binary64 mean with an a-priori error bound for Eq. 1 and the average.
+ * binary64 mean with an a-priori error bound for Eq. 1 and the average; the worker
+ * form against wo_shuffle on the stacked population, its slot counts against the
+ * permutations drawn one by one, and the expected volume p d (N-1)/N per worker.
  */
 #include <stdint.h>
 #include <stddef.h>
@@ -352,5 +358,127 @@ int wo_consensus_sq(const wo_population *pop, const void *stack, int32_t dtype,
             }
         }
     }
+    return WO_OK;
+}
+
+/* ---- the shuffling step as the workers see it (one model per worker) ----
+ * The paper's deployment keeps model n on worker n; a shuffled parameter travels
+ * peer to peer along the permutation (Introduction: models communicate their
+ * parameters peer-to-peer following the permutation; section "WASH": each model
+ * communicates p x d parameters per step in expectation).  Every worker draws the same
+ * mask and the same pi_i from the shared (seed, step), so only values travel.
+ *
+ * Wire format (a convention of this library, the paper has none): worker n owns a
+ * staging buffer.  Visit the selected coordinates in the order of the shuffling loop
+ * (segment by segment, coordinate by coordinate); each one with pi_i(n) != n takes the
+ * next free slot of worker n's buffer, and the slot is filled by worker pi_i(n) with
+ * its own value of that coordinate.  Fixed points (pi_i(n) == n) do not travel.
+ *
+ * wo_exchange_send    worker `self` fills its slots in every other worker's buffer.
+ *                     row = the worker's own model (padded_P elements, `offset`s as in
+ *                     the population; N and layout of `pop` describe the population, the
+ *                     row itself is one model).  staging[n] = worker n's buffer
+ *                     (staging[self] is not touched); capacity in elements, a slot
+ *                     beyond it is an error.  filled[n] (may be NULL) = slots of worker
+ *                     n written by this call.
+ * wo_exchange_receive worker `self` replaces its value of every selected coordinate with
+ *                     pi_i(self) != self by the next slot of its own buffer.
+ *                     stats[0] += selected coordinates, stats[1] += values received.
+ * wo_exchange_counts  need[n] = slots worker n's buffer needs in this step.
+ * A send by every worker followed by a receive by every worker is the shuffling step
+ * of wo_shuffle on the stacked population: that identity is the definition, and the
+ * tests pin these functions to it. */
+static int wo_check_exchange(const wo_population *pop, const double *p_seg, uint64_t step)
+{
+    if (wo_check_pop(pop) != WO_OK || !p_seg || pop->N < 2) return WO_ERR_ARG;
+    if (step >> 56) return WO_ERR_ARG;
+    for (int s = 0; s < pop->T; ++s)
+        if (!(p_seg[s] >= 0.0 && p_seg[s] <= 1.0)) return WO_ERR_ARG;
+    return WO_OK;
+}
+
+int wo_exchange_counts(const wo_population *pop, const double *p_seg, uint64_t seed, uint64_t step,
+                       int64_t *need, int64_t *selected)
+{
+    if (wo_check_exchange(pop, p_seg, step) != WO_OK || !need) return WO_ERR_ARG;
+    for (int n = 0; n < pop->N; ++n) need[n] = 0;
+    int64_t sel = 0;
+    for (int s = 0; s < pop->T; ++s) {
+        const uint32_t t = pop->tensor_id ? pop->tensor_id[s] : (uint32_t)s;
+        const int64_t i0 = pop->coord_begin ? pop->coord_begin[s] : 0;
+        const uint64_t thr = wo_threshold(p_seg[s]);
+        for (int64_t c = 0; c < pop->numel[s]; ++c) {
+            const uint64_t i = (uint64_t)(i0 + c);
+            if ((uint64_t)wo_mask_word(seed, step, t, i) >= thr) continue;
+            int32_t perm[1024];
+            wo_draw_permutation(seed, step, t, i, pop->N, perm);
+            sel += 1;
+            for (int n = 0; n < pop->N; ++n) need[n] += (perm[n] != n);
+        }
+    }
+    if (selected) *selected = sel;
+    return WO_OK;
+}
+
+int wo_exchange_send(const wo_population *pop, int32_t self, const void *row, int32_t dtype,
+                     const double *p_seg, uint64_t seed, uint64_t step,
+                     void *const *staging, int64_t capacity, int64_t *filled)
+{
+    if (wo_check_exchange(pop, p_seg, step) != WO_OK || !row || !staging) return WO_ERR_ARG;
+    if (self < 0 || self >= pop->N) return WO_ERR_ARG;
+    int64_t next[1024];                                  /* next free slot of every worker's buffer */
+    for (int n = 0; n < pop->N; ++n) next[n] = 0;
+    if (filled) for (int n = 0; n < pop->N; ++n) filled[n] = 0;
+    for (int s = 0; s < pop->T; ++s) {
+        const uint32_t t = pop->tensor_id ? pop->tensor_id[s] : (uint32_t)s;
+        const int64_t i0 = pop->coord_begin ? pop->coord_begin[s] : 0;
+        const uint64_t thr = wo_threshold(p_seg[s]);
+        for (int64_t c = 0; c < pop->numel[s]; ++c) {
+            const uint64_t i = (uint64_t)(i0 + c);
+            if ((uint64_t)wo_mask_word(seed, step, t, i) >= thr) continue;
+            int32_t perm[1024];
+            wo_draw_permutation(seed, step, t, i, pop->N, perm);
+            const int64_t elem = pop->offset[s] + c;
+            for (int n = 0; n < pop->N; ++n) {
+                if (perm[n] == n) continue;              /* worker n keeps its own value     */
+                const int64_t slot = next[n]++;
+                if (perm[n] != self) continue;           /* another worker fills this slot   */
+                if (slot >= capacity) return WO_ERR_ARG;
+                if (dtype == WO_F32) ((uint32_t *)staging[n])[slot] = ((const uint32_t *)row)[elem];
+                else ((uint16_t *)staging[n])[slot] = ((const uint16_t *)row)[elem];
+                if (filled) filled[n] += 1;
+            }
+        }
+    }
+    return WO_OK;
+}
+
+int wo_exchange_receive(const wo_population *pop, int32_t self, void *row, int32_t dtype,
+                        const double *p_seg, uint64_t seed, uint64_t step,
+                        const void *staging_self, int64_t capacity, uint64_t *stats)
+{
+    if (wo_check_exchange(pop, p_seg, step) != WO_OK || !row || !staging_self) return WO_ERR_ARG;
+    if (self < 0 || self >= pop->N) return WO_ERR_ARG;
+    int64_t next = 0;
+    uint64_t selected = 0;
+    for (int s = 0; s < pop->T; ++s) {
+        const uint32_t t = pop->tensor_id ? pop->tensor_id[s] : (uint32_t)s;
+        const int64_t i0 = pop->coord_begin ? pop->coord_begin[s] : 0;
+        const uint64_t thr = wo_threshold(p_seg[s]);
+        for (int64_t c = 0; c < pop->numel[s]; ++c) {
+            const uint64_t i = (uint64_t)(i0 + c);
+            if ((uint64_t)wo_mask_word(seed, step, t, i) >= thr) continue;
+            int32_t perm[1024];
+            wo_draw_permutation(seed, step, t, i, pop->N, perm);
+            selected += 1;
+            if (perm[self] == self) continue;
+            if (next >= capacity) return WO_ERR_ARG;
+            const int64_t elem = pop->offset[s] + c;
+            if (dtype == WO_F32) ((uint32_t *)row)[elem] = ((const uint32_t *)staging_self)[next];
+            else ((uint16_t *)row)[elem] = ((const uint16_t *)staging_self)[next];
+            next += 1;
+        }
+    }
+    if (stats) { stats[0] += selected; stats[1] += (uint64_t)next; }
     return WO_OK;
 }

@@ -490,10 +490,6 @@ int wash_step_host(wash_ctx *ctx, int32_t ops, void *host_params, void *host_opt
     cudaError_t err;
     if ((ops & WASH_OP_AVERAGE) && ctx->avg_bytes < avg_bytes) {
         if (ctx->avg_dev) cudaFree(ctx->avg_dev);
-    if (ctx->copy_in) cudaStreamDestroy(ctx->copy_in);
-    if (ctx->copy_out) cudaStreamDestroy(ctx->copy_out);
-    for (cudaEvent_t e : ctx->pipe_event)
-        if (e) cudaEventDestroy(e);
         ctx->avg_dev = nullptr;
         ctx->avg_bytes = 0;
         if ((err = cudaMalloc(&ctx->avg_dev, avg_bytes)) != cudaSuccess) {

@@ -158,3 +158,23 @@ def test_step_over_host_buffers_pipelined(dtype, layout):
         assert (to_host_bits(havg) == bits(want_avg)).all()
     B.wash_check(c.gpu.ctx)
     c.close()
+
+
+def test_host_step_average_requested_on_a_later_call():
+    """The pipeline's copy streams are set up by the first call; a later call that asks for
+    the average for the first time must leave them usable."""
+    N, numel = 2, [1 << 20, 12]
+    c = Case(N, numel, 0, "f32", None, seed=15)
+    hp = torch.from_numpy(c.host.reshape(-1).copy()).pin_memory()
+    havg = torch.zeros(c.P, dtype=torch.float32).pin_memory()
+    st = B.wash_step_host(c.gpu.ctx, B.WASH_OP_SHUFFLE, hp, None, None, 0, 0.01, None, seed=9, alpha=0.5)
+    assert st == oracle.shuffle(c.ora, c.host, 0.01, seed=9, step=0)
+    for step in (1, 2):
+        st = B.wash_step_host(c.gpu.ctx, B.WASH_OP_SHUFFLE | B.WASH_OP_AVERAGE, hp, None, havg, step, 0.01, None, seed=9, alpha=0.5)
+        assert st == oracle.shuffle(c.ora, c.host, 0.01, seed=9, step=step)
+        want_avg = np.zeros(c.P, dtype=np.float32)
+        oracle.population_average(c.ora, c.host, want_avg)
+        assert (hp.numpy().view(np.uint32) == bits(c.host)).all()
+        assert (havg.numpy().view(np.uint32) == want_avg.view(np.uint32)).all()
+    B.wash_check(c.gpu.ctx)
+    c.close()

@@ -28,6 +28,12 @@ MUTATIONS = {
     "sum from the last model down": ("for (int n = 1; n < pop->N; ++n) {\n        float x = wo_load(stack, dtype, wo_index(pop, n, elem));",
                                        "for (int n = pop->N - 1; n >= 1; --n) {\n        float x = wo_load(stack, dtype, wo_index(pop, n, elem));", "test_oracle_ema_avg.py"),
     "bf16 truncates": ("u += 0x7FFFu + lsb;", "", "test_oracle_ema_avg.py"),
+    "worker sends along the inverse permutation": ("if (perm[n] != self) continue;", "if (perm[self] != n) continue;", "test_oracle_exchange.py"),
+    "fixed points take a slot": ("if (perm[n] == n) continue;              /* worker n keeps its own value     */", "", "test_oracle_exchange.py"),
+    "receiver takes a slot for a fixed point": ("if (perm[self] == self) continue;", "", "test_oracle_exchange.py"),
+    "slot counts include fixed points": ("need[n] += (perm[n] != n);", "need[n] += 1;", "test_oracle_exchange.py"),
+    "slots numbered per sender": ("const int64_t slot = next[n]++;\n                if (perm[n] != self) continue;           /* another worker fills this slot   */",
+                                  "if (perm[n] != self) continue;\n                const int64_t slot = next[n]++;", "test_oracle_exchange.py"),
     "last layer still shuffled": ("(double)l / (double)(L - 1);", "(double)l / (double)(L);", "test_oracle_ema_avg.py"),
 }
 
@@ -52,7 +58,7 @@ def test_unmodified_copy_passes_the_pins(tmp_path):
         text = f.read()
     lib = str(tmp_path / "liboracle_copy.so")
     _build(text, lib)
-    for test_file in ("test_oracle_philox.py", "test_oracle_shuffle.py", "test_oracle_ema_avg.py"):
+    for test_file in ("test_oracle_philox.py", "test_oracle_shuffle.py", "test_oracle_ema_avg.py", "test_oracle_exchange.py"):
         ok, tail = _pins_pass(lib, test_file)
         assert ok, tail
 
