@@ -205,6 +205,71 @@ int wash_step_host(wash_ctx *ctx, int32_t ops, void *host_params, void *host_opt
                    uint64_t step, double p, const double *p_layer, uint64_t seed, float alpha,
                    void *stream, wash_stats *host_stats);
 
+/* ---- one model per device ----------------------------------------------------------
+ *
+ * The deployment the paper describes (Introduction: a permutation is drawn and models
+ * communicate their parameters peer to peer following it; section "WASH": each model
+ * communicates p*d parameters per step in expectation): worker n holds model n only.
+ * Every worker derives the same mask and the same permutations from the shared
+ * (seed, step), so nothing but values crosses the link, and in a fixed order that needs
+ * no indices:
+ *
+ *   worker n owns a STAGING buffer.  The selected coordinates with pi_i(n) != n, taken
+ *   in the order of Algorithm 1's shuffling loop (tensor by tensor, coordinate by
+ *   coordinate), occupy its slots 0, 1, 2, ...; the slot of coordinate i is filled by
+ *   worker pi_i(n) with its own value of i (Eq. 3 read as a gather).  Fixed points of
+ *   pi_i do not travel.
+ *
+ * A step is  wash_exchange_plan  ->  wash_exchange_send  ->  (all workers have sent)  ->
+ * wash_exchange_receive  on every worker; the result equals wash_shuffle (or
+ * wash_shuffle_both when both rows are bound) on the stacked population, bit for bit.
+ * The library performs no inter-device synchronisation: between send and receive the
+ * caller orders the workers (a barrier of the process group enqueued on the same
+ * stream, or stream/event order when one process drives several workers).
+ * Two staging sets (parity 0 and 1) may be registered; a step uses set (step & 1) if it
+ * is registered, else set 0.  With both registered one barrier per step suffices (a
+ * worker can start sending step s+1 while a slower peer still reads step s's set).
+ *
+ * The context is created with wash_create / wash_create_segments as usual (N = size of
+ * the population, the tensor table of ONE model; layout is ignored).  Rows of 2^32 and
+ * more elements are not supported in this form (WASH_ERR_UNSUPPORTED). */
+
+/* Declares this context worker `self` (0 <= self < N) and borrows the worker's model:
+ * dev_row is a DEVICE row of padded_P elements (n_elems must say so) of `dtype`, 16-byte
+ * aligned, for `stack` (WASH_STACK_PARAMS, or WASH_STACK_OPT for the optimizer state,
+ * which then follows the same mask and permutations).  NULL unbinds.  The first call
+ * allocates the plan's tables (padded_P/4 bytes + 4 (N+1) padded_P/1024 bytes). */
+int wash_exchange_bind(wash_ctx *ctx, int32_t self, int32_t stack, int32_t dtype, void *dev_row, int64_t n_elems);
+
+/* Registers staging set `parity` (0 or 1) of `stack`: buffers is a HOST array of N
+ * pointers, entry n = worker n's staging buffer for this stack, each holding
+ * capacity_elems elements of the stack's dtype, 4-byte aligned, and accessible from this
+ * device (entry `self` is this worker's own buffer; the others are peer mappings, or
+ * plain device buffers when one process emulates all workers).  The pointers are copied;
+ * the buffers stay the caller's.  A step that needs more slots than capacity_elems writes
+ * and reads nothing beyond the buffers and makes wash_check fail. */
+int wash_exchange_staging(wash_ctx *ctx, int32_t stack, int32_t parity, void *const *buffers, int64_t capacity_elems);
+
+/* Draws the step: mask, permutations, and the slot offsets of every worker's buffer.
+ * Reads no model data.  step, p, p_layer, seed as for wash_shuffle; every worker must
+ * pass the same values. */
+int wash_exchange_plan(wash_ctx *ctx, uint64_t step, double p, const double *p_layer, uint64_t seed, void *stream);
+
+/* Stores this worker's values into the other workers' staging buffers, for every bound
+ * stack, according to the last plan. */
+int wash_exchange_send(wash_ctx *ctx, void *stream);
+
+/* Copies this worker's slots from its own staging buffer into its model, for every bound
+ * stack.  stats (DEVICE-accessible, may be NULL): selected_coords += coordinates selected
+ * in the step (the same on every worker), moved_values += values this worker received
+ * (summed over workers: wash_shuffle's moved_values). */
+int wash_exchange_receive(wash_ctx *ctx, void *stream, wash_stats *stats);
+
+/* Waits for `stream` and reports the last plan: host_need[n] (HOST array of N, may be
+ * NULL) = slots worker n's buffer needs, *host_selected (may be NULL) = selected
+ * coordinates. */
+int wash_exchange_counts(wash_ctx *ctx, uint64_t *host_need, uint64_t *host_selected, void *stream);
+
 /* ---- for callers that must not allocate ------------------------------------------- */
 
 #define WASH_NOALLOC_MAX_TENSORS 1024                 /* most tensors per model            */

@@ -73,6 +73,12 @@ def load() -> ctypes.CDLL:
     L.wash_launch_count.restype = ctypes.c_uint64
     L.wash_shuffle_noalloc.argtypes = [i32, i32, i64p, i32, i32, vp, i64, u64, dbl, dblp, u64, i32, vp, vp]
     L.wash_noalloc_last_error.restype = ctypes.c_char_p
+    L.wash_exchange_bind.argtypes = [vp, i32, i32, i32, vp, i64]
+    L.wash_exchange_staging.argtypes = [vp, i32, i32, ctypes.POINTER(vp), i64]
+    L.wash_exchange_plan.argtypes = [vp, u64, dbl, dblp, u64, vp]
+    L.wash_exchange_send.argtypes = [vp, vp]
+    L.wash_exchange_receive.argtypes = [vp, vp, vp]
+    L.wash_exchange_counts.argtypes = [vp, ctypes.POINTER(u64), ctypes.POINTER(u64), vp]
     _lib = L
     return L
 
@@ -223,6 +229,37 @@ def wash_shuffle_noalloc(N: int, numel, layout: int, dtype: int, dev_stack, n_el
 
 def wash_noalloc_last_error() -> str:
     return load().wash_noalloc_last_error().decode()
+
+
+def wash_exchange_bind(ctx, self_rank: int, stack: int, dtype: int, dev_row, n_elems: int) -> None:
+    _check(load().wash_exchange_bind(ctx, self_rank, stack, dtype, _ptr(dev_row), n_elems))
+
+
+def wash_exchange_staging(ctx, stack: int, parity: int, buffers, capacity_elems: int) -> None:
+    """buffers: one tensor / address per worker (worker n's staging buffer)"""
+    ptrs = (ctypes.c_void_p * len(buffers))(*[_ptr(b) for b in buffers])
+    _check(load().wash_exchange_staging(ctx, stack, parity, ptrs, capacity_elems))
+
+
+def wash_exchange_plan(ctx, step: int, p: float, p_layer=None, seed: int = 0, stream=None) -> None:
+    keep, pl = _dbl_or_null(p_layer)
+    _check(load().wash_exchange_plan(ctx, step, float(p), pl, seed, _stream(stream)))
+
+
+def wash_exchange_send(ctx, stream=None) -> None:
+    _check(load().wash_exchange_send(ctx, _stream(stream)))
+
+
+def wash_exchange_receive(ctx, stream=None, stats=None) -> None:
+    _check(load().wash_exchange_receive(ctx, _stream(stream), _ptr(stats)))
+
+
+def wash_exchange_counts(ctx, N: int, stream=None):
+    """-> (need[N], selected) of the last plan; waits for the stream"""
+    need = (ctypes.c_uint64 * N)()
+    sel = ctypes.c_uint64(0)
+    _check(load().wash_exchange_counts(ctx, need, ctypes.byref(sel), _stream(stream)))
+    return [int(x) for x in need], int(sel.value)
 
 
 def wash_philox_probe(n_blocks: int, seed: int = 0, dev_checksum=None, device: int = 0, stream=None) -> None:

@@ -93,6 +93,19 @@ struct wash_ctx {
 
     int mode = WASH_MODE_STREAM;
     wash::LaunchShape shape{0, 0, 148};
+
+    // one model per device (wash_exchange_*)
+    int x_self = -1;
+    void *x_row[2] = {nullptr, nullptr};
+    int x_dtype[2] = {0, 0};
+    uint8_t *x_mask = nullptr;             // a byte per group
+    uint32_t *x_count = nullptr;           // [N + 1][x_tiles]
+    uint32_t *x_total = nullptr;           // [N + 1]
+    uint32_t x_tiles = 0;
+    void **x_staging[2][2] = {{nullptr, nullptr}, {nullptr, nullptr}};   // [parity][stack]: device array of N pointers
+    int64_t x_capacity[2][2] = {{0, 0}, {0, 0}};
+    bool x_planned = false;
+    uint64_t x_step = 0, x_seed = 0;
 };
 
 namespace {
@@ -107,6 +120,12 @@ void release(wash_ctx *ctx)
     if (ctx->stats_dev) cudaFree(ctx->stats_dev);
     if (ctx->stat_slots_dev) cudaFree(ctx->stat_slots_dev);
     if (ctx->avg_dev) cudaFree(ctx->avg_dev);
+    if (ctx->x_mask) cudaFree(ctx->x_mask);
+    if (ctx->x_count) cudaFree(ctx->x_count);
+    if (ctx->x_total) cudaFree(ctx->x_total);
+    for (auto &set : ctx->x_staging)
+        for (void **ptrs : set)
+            if (ptrs) cudaFree(ptrs);
     if (ctx->copy_in) cudaStreamDestroy(ctx->copy_in);
     if (ctx->copy_out) cudaStreamDestroy(ctx->copy_out);
     for (cudaEvent_t e : ctx->pipe_event)
@@ -609,6 +628,178 @@ int wash_step_host(wash_ctx *ctx, int32_t ops, void *host_params, void *host_opt
     return WASH_OK;
 }
 
+// ---- one model per device ------------------------------------------------------------
+
+}  // extern "C"
+
+namespace {
+
+// kernel arguments of the planned step; `need_rows`: at least one row must be bound
+int exchange_args(wash_ctx *ctx, wash::ExchangeArgs *out)
+{
+    if (!ctx) return fail(WASH_ERR_ARG, "ctx is NULL");
+    if (ctx->x_self < 0) return fail(WASH_ERR_STATE, "wash_exchange_bind has not been called");
+    wash::ExchangeArgs &a = *out;
+    a.pop = view_of(ctx);
+    a.self = ctx->x_self;
+    a.n_tiles = ctx->x_tiles;
+    a.key0 = static_cast<uint32_t>(ctx->x_seed);
+    a.key1 = static_cast<uint32_t>(ctx->x_seed >> 32);
+    a.step_lo = static_cast<uint32_t>(ctx->x_step);
+    a.step_hi8 = static_cast<uint32_t>(ctx->x_step >> 32) << 8;
+    a.mask = ctx->x_mask;
+    a.tile_count = ctx->x_count;
+    a.total = ctx->x_total;
+    const int parity = static_cast<int>(ctx->x_step & 1u);
+    for (int k = 0; k < 2; ++k) {
+        a.row[k] = ctx->x_row[k];
+        a.dtype[k] = ctx->x_dtype[k];
+        const int set = ctx->x_staging[parity][k] ? parity : 0;
+        a.staging[k] = ctx->x_staging[set][k];
+        a.capacity[k] = ctx->x_capacity[set][k];
+    }
+    a.stats = nullptr;
+    a.status = ctx->status_dev;
+    return WASH_OK;
+}
+
+int exchange_ready(const wash_ctx *ctx, const wash::ExchangeArgs &a)
+{
+    if (!ctx->x_planned) return fail(WASH_ERR_STATE, "no step has been planned (wash_exchange_plan)");
+    if (!a.row[0] && !a.row[1]) return fail(WASH_ERR_STATE, "no model row is bound");
+    for (int k = 0; k < 2; ++k)
+        if (a.row[k] && !a.staging[k]) return fail(WASH_ERR_STATE, "stack %d has no staging buffers (wash_exchange_staging)", k);
+    return WASH_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int wash_exchange_bind(wash_ctx *ctx, int32_t self, int32_t stack, int32_t dtype, void *dev_row, int64_t n_elems)
+{
+    if (!ctx) return fail(WASH_ERR_ARG, "ctx is NULL");
+    if (self < 0 || self >= ctx->N) return fail(WASH_ERR_ARG, "self = %d, must be in [0, %d)", self, ctx->N);
+    if (stack != WASH_STACK_PARAMS && stack != WASH_STACK_OPT) return fail(WASH_ERR_ARG, "stack must be 0 or 1");
+    if (ctx->padded_P >= (int64_t(1) << 32)) return fail(WASH_ERR_UNSUPPORTED, "rows of 2^32 elements and more cannot be exchanged");
+    if (ctx->x_self >= 0 && ctx->x_self != self) return fail(WASH_ERR_STATE, "context already is worker %d", ctx->x_self);
+    if (dev_row) {
+        if (dtype != WASH_F32 && dtype != WASH_BF16) return fail(WASH_ERR_ARG, "unknown dtype %d", dtype);
+        if (n_elems != ctx->padded_P) return fail(WASH_ERR_ARG, "row has %lld elements, a model needs padded_P = %lld", (long long)n_elems, (long long)ctx->padded_P);
+        if (reinterpret_cast<uintptr_t>(dev_row) & 15) return fail(WASH_ERR_ARG, "row pointer must be 16-byte aligned");
+    }
+    if (!ctx->x_mask) {
+        DeviceGuard guard(ctx->device);
+        if (guard.err != cudaSuccess) return cuda_fail(guard.err, "cudaSetDevice");
+        const uint32_t tiles = (ctx->n_groups + wash::kExchangeTileGroups - 1) / wash::kExchangeTileGroups;
+        const size_t columns = static_cast<size_t>(ctx->N) + 1;
+        cudaError_t err;
+        if ((err = cudaMalloc(&ctx->x_mask, ctx->n_groups)) != cudaSuccess ||
+            (err = cudaMalloc(&ctx->x_count, sizeof(uint32_t) * columns * tiles)) != cudaSuccess ||
+            (err = cudaMalloc(&ctx->x_total, sizeof(uint32_t) * columns)) != cudaSuccess) {
+            cudaGetLastError();
+            if (ctx->x_mask) cudaFree(ctx->x_mask);
+            if (ctx->x_count) cudaFree(ctx->x_count);
+            ctx->x_mask = nullptr;
+            ctx->x_count = nullptr;
+            return fail(WASH_ERR_ALLOC, "device allocation of the exchange tables failed: %s", cudaGetErrorString(err));
+        }
+        ctx->x_tiles = tiles;
+    }
+    ctx->x_self = self;
+    ctx->x_row[stack] = dev_row;
+    ctx->x_dtype[stack] = dtype;
+    return WASH_OK;
+}
+
+int wash_exchange_staging(wash_ctx *ctx, int32_t stack, int32_t parity, void *const *buffers, int64_t capacity_elems)
+{
+    if (!ctx) return fail(WASH_ERR_ARG, "ctx is NULL");
+    if (stack != WASH_STACK_PARAMS && stack != WASH_STACK_OPT) return fail(WASH_ERR_ARG, "stack must be 0 or 1");
+    if (parity != 0 && parity != 1) return fail(WASH_ERR_ARG, "parity must be 0 or 1");
+    if (!buffers) return fail(WASH_ERR_ARG, "buffers is NULL");
+    if (capacity_elems < 0) return fail(WASH_ERR_ARG, "capacity_elems = %lld", (long long)capacity_elems);
+    for (int n = 0; n < ctx->N; ++n)
+        if (!buffers[n] || (reinterpret_cast<uintptr_t>(buffers[n]) & 3)) return fail(WASH_ERR_ARG, "buffers[%d] must be a 4-byte aligned device-accessible pointer", n);
+    DeviceGuard guard(ctx->device);
+    if (guard.err != cudaSuccess) return cuda_fail(guard.err, "cudaSetDevice");
+    cudaError_t err;
+    if (!ctx->x_staging[parity][stack] &&
+        (err = cudaMalloc(reinterpret_cast<void **>(&ctx->x_staging[parity][stack]), sizeof(void *) * static_cast<size_t>(ctx->N))) != cudaSuccess) {
+        cudaGetLastError();
+        return fail(WASH_ERR_ALLOC, "device allocation of the pointer table failed: %s", cudaGetErrorString(err));
+    }
+    // synchronous: earlier steps that read the table are complete when it is replaced
+    if ((err = cudaDeviceSynchronize()) != cudaSuccess) return cuda_fail(err, "cudaDeviceSynchronize");
+    if ((err = cudaMemcpy(ctx->x_staging[parity][stack], buffers, sizeof(void *) * static_cast<size_t>(ctx->N), cudaMemcpyHostToDevice)) != cudaSuccess)
+        return cuda_fail(err, "upload of the staging pointers");
+    ctx->x_capacity[parity][stack] = capacity_elems;
+    return WASH_OK;
+}
+
+int wash_exchange_plan(wash_ctx *ctx, uint64_t step, double p, const double *p_layer, uint64_t seed, void *stream_v)
+{
+    if (!ctx) return fail(WASH_ERR_ARG, "ctx is NULL");
+    if (ctx->x_self < 0) return fail(WASH_ERR_STATE, "wash_exchange_bind has not been called");
+    if (step >> 56) return fail(WASH_ERR_ARG, "step must be below 2^56");
+    if (!p_layer && !(p >= 0.0 && p <= 1.0)) return fail(WASH_ERR_ARG, "p is %g, not in [0,1]", p);
+    DeviceGuard guard(ctx->device);
+    if (guard.err != cudaSuccess) return cuda_fail(guard.err, "cudaSetDevice");
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
+    int rc = sync_table(ctx, p, p_layer, stream);
+    if (rc != WASH_OK) return rc;
+    ctx->x_step = step;
+    ctx->x_seed = seed;
+    wash::ExchangeArgs args;
+    if ((rc = exchange_args(ctx, &args)) != WASH_OK) return rc;
+    cudaError_t err = wash::launch_exchange_plan(args, stream);
+    if (err != cudaSuccess) return cuda_fail(err, "exchange plan launch");
+    ctx->x_planned = true;
+    return WASH_OK;
+}
+
+int wash_exchange_send(wash_ctx *ctx, void *stream_v)
+{
+    wash::ExchangeArgs args;
+    int rc = exchange_args(ctx, &args);
+    if (rc != WASH_OK || (rc = exchange_ready(ctx, args)) != WASH_OK) return rc;
+    DeviceGuard guard(ctx->device);
+    if (guard.err != cudaSuccess) return cuda_fail(guard.err, "cudaSetDevice");
+    cudaError_t err = wash::launch_exchange_send(args, static_cast<cudaStream_t>(stream_v));
+    if (err != cudaSuccess) return cuda_fail(err, "exchange send launch");
+    return WASH_OK;
+}
+
+int wash_exchange_receive(wash_ctx *ctx, void *stream_v, wash_stats *stats)
+{
+    wash::ExchangeArgs args;
+    int rc = exchange_args(ctx, &args);
+    if (rc != WASH_OK || (rc = exchange_ready(ctx, args)) != WASH_OK) return rc;
+    args.stats = reinterpret_cast<unsigned long long *>(stats);
+    DeviceGuard guard(ctx->device);
+    if (guard.err != cudaSuccess) return cuda_fail(guard.err, "cudaSetDevice");
+    cudaError_t err = wash::launch_exchange_receive(args, static_cast<cudaStream_t>(stream_v));
+    if (err != cudaSuccess) return cuda_fail(err, "exchange receive launch");
+    return WASH_OK;
+}
+
+int wash_exchange_counts(wash_ctx *ctx, uint64_t *host_need, uint64_t *host_selected, void *stream_v)
+{
+    if (!ctx) return fail(WASH_ERR_ARG, "ctx is NULL");
+    if (!ctx->x_planned) return fail(WASH_ERR_STATE, "no step has been planned (wash_exchange_plan)");
+    DeviceGuard guard(ctx->device);
+    if (guard.err != cudaSuccess) return cuda_fail(guard.err, "cudaSetDevice");
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
+    std::vector<uint32_t> total(static_cast<size_t>(ctx->N) + 1);
+    cudaError_t err = cudaMemcpyAsync(total.data(), ctx->x_total, sizeof(uint32_t) * total.size(), cudaMemcpyDeviceToHost, stream);
+    if (err == cudaSuccess) err = cudaStreamSynchronize(stream);
+    if (err != cudaSuccess) return cuda_fail(err, "reading the plan's totals");
+    if (host_need)
+        for (int n = 0; n < ctx->N; ++n) host_need[n] = total[static_cast<size_t>(n)];
+    if (host_selected) *host_selected = total[static_cast<size_t>(ctx->N)];
+    return WASH_OK;
+}
+
 int wash_check(wash_ctx *ctx, void *stream_v)
 {
     if (!ctx) return fail(WASH_ERR_ARG, "ctx is NULL");
@@ -621,7 +812,10 @@ int wash_check(wash_ctx *ctx, void *stream_v)
     if (err != cudaSuccess) return cuda_fail(err, "reading the status word");
     if (status) {
         cudaMemsetAsync(ctx->status_dev, 0, sizeof(uint32_t), stream);
-        return fail(WASH_ERR_DEVICE_CHECK, "a kernel found a group outside its segment table (status 0x%x)", status);
+        return fail(WASH_ERR_DEVICE_CHECK, "device status 0x%x:%s%s%s", status,
+                    (status & 1u) ? " a group outside its segment table;" : "",
+                    (status & 2u) ? " a bounded wait of the staged shuffle ran out;" : "",
+                    (status & 4u) ? " an exchange step needed more slots than the staging buffers hold;" : "");
     }
     return WASH_OK;
 }

@@ -64,6 +64,29 @@ struct ReduceArgs {
     uint32_t *status;
 };
 
+// One model per device (wash_exchange_*): the row is one model of a population of pop.N.
+constexpr int kExchangeTileGroups = 256;   // a tile = one block = 256 groups = 1024 coordinates
+struct ExchangeArgs {
+    PopView pop;
+    int self;                     // this worker's index in the population
+    uint32_t n_tiles;             // ceil(n_groups / kExchangeTileGroups)
+    uint32_t key0, key1;
+    uint32_t step_lo, step_hi8;
+    uint8_t *mask;                // [n_groups] low nibble: selected coordinates; high nibble: those this worker receives
+    uint32_t *tile_count;         // [N + 1][n_tiles]: column n = slots of worker n's buffer per tile (after the scan:
+                                  // slots before the tile); column N = selected coordinates
+    uint32_t *total;              // [N + 1] column totals
+    void *row[2];                 // this worker's model: parameters, optimizer state (nullptr: absent)
+    int dtype[2];
+    void *const *staging[2];      // per stack: device array of N pointers, entry n = worker n's staging buffer
+    long long capacity[2];        // elements per staging buffer
+    unsigned long long *stats;    // {selected, received} or nullptr
+    uint32_t *status;
+};
+cudaError_t launch_exchange_plan(const ExchangeArgs &args, cudaStream_t stream);
+cudaError_t launch_exchange_send(const ExchangeArgs &args, cudaStream_t stream);
+cudaError_t launch_exchange_receive(const ExchangeArgs &args, cudaStream_t stream);
+
 enum ReduceOp { kOpEma = 0, kOpAverage = 1, kOpPapaAll = 2, kOpConsensus = 3 };
 
 struct LaunchShape {
