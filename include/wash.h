@@ -250,6 +250,20 @@ int wash_exchange_bind(wash_ctx *ctx, int32_t self, int32_t stack, int32_t dtype
  * and reads nothing beyond the buffers and makes wash_check fail. */
 int wash_exchange_staging(wash_ctx *ctx, int32_t stack, int32_t parity, void *const *buffers, int64_t capacity_elems);
 
+/* The same registration for workers that live in different processes (one per GPU).
+ * wash_exchange_staging_create allocates this worker's buffer of set `parity` for `stack`
+ * (the row must be bound; capacity_elems elements of its dtype; owned and freed by the
+ * context) and writes its inter-process handle, WASH_IPC_HANDLE_BYTES bytes, to the HOST
+ * buffer handle_out.  The processes exchange the handles (any host channel) and every
+ * worker passes all N of them, in worker order, to wash_exchange_staging_open, which maps
+ * the peers' buffers into this process (entry `self` is ignored; peer access over NVLink
+ * is enabled as needed) and registers the set.  All workers must use one capacity.
+ * The mappings are closed by wash_destroy: destroy every context of the group only after
+ * all workers have finished their last step. */
+#define WASH_IPC_HANDLE_BYTES 64
+int wash_exchange_staging_create(wash_ctx *ctx, int32_t stack, int32_t parity, int64_t capacity_elems, void *handle_out);
+int wash_exchange_staging_open(wash_ctx *ctx, int32_t stack, int32_t parity, const void *handles);
+
 /* Draws the step: mask, permutations, and the slot offsets of every worker's buffer.
  * Reads no model data.  step, p, p_layer, seed as for wash_shuffle; every worker must
  * pass the same values. */

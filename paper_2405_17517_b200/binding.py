@@ -75,6 +75,8 @@ def load() -> ctypes.CDLL:
     L.wash_noalloc_last_error.restype = ctypes.c_char_p
     L.wash_exchange_bind.argtypes = [vp, i32, i32, i32, vp, i64]
     L.wash_exchange_staging.argtypes = [vp, i32, i32, ctypes.POINTER(vp), i64]
+    L.wash_exchange_staging_create.argtypes = [vp, i32, i32, i64, vp]
+    L.wash_exchange_staging_open.argtypes = [vp, i32, i32, vp]
     L.wash_exchange_plan.argtypes = [vp, u64, dbl, dblp, u64, vp]
     L.wash_exchange_send.argtypes = [vp, vp]
     L.wash_exchange_receive.argtypes = [vp, vp, vp]
@@ -239,6 +241,22 @@ def wash_exchange_staging(ctx, stack: int, parity: int, buffers, capacity_elems:
     """buffers: one tensor / address per worker (worker n's staging buffer)"""
     ptrs = (ctypes.c_void_p * len(buffers))(*[_ptr(b) for b in buffers])
     _check(load().wash_exchange_staging(ctx, stack, parity, ptrs, capacity_elems))
+
+
+WASH_IPC_HANDLE_BYTES = 64
+
+
+def wash_exchange_staging_create(ctx, stack: int, parity: int, capacity_elems: int) -> bytes:
+    """-> this worker's inter-process handle (bytes) for the buffer it just allocated"""
+    out = ctypes.create_string_buffer(WASH_IPC_HANDLE_BYTES)
+    _check(load().wash_exchange_staging_create(ctx, stack, parity, capacity_elems, out))
+    return out.raw
+
+
+def wash_exchange_staging_open(ctx, stack: int, parity: int, handles) -> None:
+    """handles: the N workers' handles in worker order (bytes each)"""
+    blob = b"".join(bytes(h) for h in handles)
+    _check(load().wash_exchange_staging_open(ctx, stack, parity, blob))
 
 
 def wash_exchange_plan(ctx, step: int, p: float, p_layer=None, seed: int = 0, stream=None) -> None:

@@ -104,6 +104,8 @@ struct wash_ctx {
     uint32_t x_tiles = 0;
     void **x_staging[2][2] = {{nullptr, nullptr}, {nullptr, nullptr}};   // [parity][stack]: device array of N pointers
     int64_t x_capacity[2][2] = {{0, 0}, {0, 0}};
+    void *x_own[2][2] = {{nullptr, nullptr}, {nullptr, nullptr}};        // staging buffers this library allocated
+    std::vector<void *> x_opened;          // peers' buffers mapped by wash_exchange_staging_open
     bool x_planned = false;
     uint64_t x_step = 0, x_seed = 0;
 };
@@ -126,6 +128,10 @@ void release(wash_ctx *ctx)
     for (auto &set : ctx->x_staging)
         for (void **ptrs : set)
             if (ptrs) cudaFree(ptrs);
+    for (void *peer : ctx->x_opened) cudaIpcCloseMemHandle(peer);
+    for (auto &set : ctx->x_own)
+        for (void *own : set)
+            if (own) cudaFree(own);
     if (ctx->copy_in) cudaStreamDestroy(ctx->copy_in);
     if (ctx->copy_out) cudaStreamDestroy(ctx->copy_out);
     for (cudaEvent_t e : ctx->pipe_event)
@@ -735,6 +741,56 @@ int wash_exchange_staging(wash_ctx *ctx, int32_t stack, int32_t parity, void *co
         return cuda_fail(err, "upload of the staging pointers");
     ctx->x_capacity[parity][stack] = capacity_elems;
     return WASH_OK;
+}
+
+int wash_exchange_staging_create(wash_ctx *ctx, int32_t stack, int32_t parity, int64_t capacity_elems, void *handle_out)
+{
+    if (!ctx) return fail(WASH_ERR_ARG, "ctx is NULL");
+    if (stack != WASH_STACK_PARAMS && stack != WASH_STACK_OPT) return fail(WASH_ERR_ARG, "stack must be 0 or 1");
+    if (parity != 0 && parity != 1) return fail(WASH_ERR_ARG, "parity must be 0 or 1");
+    if (capacity_elems < 1) return fail(WASH_ERR_ARG, "capacity_elems = %lld", (long long)capacity_elems);
+    if (!handle_out) return fail(WASH_ERR_ARG, "handle_out is NULL");
+    if (ctx->x_self < 0 || !ctx->x_row[stack]) return fail(WASH_ERR_STATE, "bind the row of stack %d first (wash_exchange_bind)", stack);
+    if (ctx->x_own[parity][stack]) return fail(WASH_ERR_STATE, "staging set %d of stack %d already exists", parity, stack);
+    DeviceGuard guard(ctx->device);
+    if (guard.err != cudaSuccess) return cuda_fail(guard.err, "cudaSetDevice");
+    void *buf = nullptr;
+    cudaError_t err = cudaMalloc(&buf, static_cast<size_t>(capacity_elems) * elem_bytes(ctx->x_dtype[stack]));
+    if (err != cudaSuccess) {
+        cudaGetLastError();
+        return fail(WASH_ERR_ALLOC, "device allocation of the staging buffer failed: %s", cudaGetErrorString(err));
+    }
+    cudaIpcMemHandle_t handle;
+    if ((err = cudaIpcGetMemHandle(&handle, buf)) != cudaSuccess) {
+        cudaFree(buf);
+        return cuda_fail(err, "cudaIpcGetMemHandle");
+    }
+    static_assert(sizeof handle == WASH_IPC_HANDLE_BYTES, "handle size");
+    std::memcpy(handle_out, &handle, sizeof handle);
+    ctx->x_own[parity][stack] = buf;
+    ctx->x_capacity[parity][stack] = capacity_elems;
+    return WASH_OK;
+}
+
+int wash_exchange_staging_open(wash_ctx *ctx, int32_t stack, int32_t parity, const void *handles)
+{
+    if (!ctx) return fail(WASH_ERR_ARG, "ctx is NULL");
+    if (stack != WASH_STACK_PARAMS && stack != WASH_STACK_OPT) return fail(WASH_ERR_ARG, "stack must be 0 or 1");
+    if (parity != 0 && parity != 1) return fail(WASH_ERR_ARG, "parity must be 0 or 1");
+    if (!handles) return fail(WASH_ERR_ARG, "handles is NULL");
+    if (!ctx->x_own[parity][stack]) return fail(WASH_ERR_STATE, "create this worker's buffer first (wash_exchange_staging_create)");
+    DeviceGuard guard(ctx->device);
+    if (guard.err != cudaSuccess) return cuda_fail(guard.err, "cudaSetDevice");
+    std::vector<void *> buffers(static_cast<size_t>(ctx->N), nullptr);
+    for (int n = 0; n < ctx->N; ++n) {
+        if (n == ctx->x_self) { buffers[n] = ctx->x_own[parity][stack]; continue; }
+        cudaIpcMemHandle_t handle;
+        std::memcpy(&handle, static_cast<const char *>(handles) + static_cast<size_t>(n) * WASH_IPC_HANDLE_BYTES, sizeof handle);
+        cudaError_t err = cudaIpcOpenMemHandle(&buffers[n], handle, cudaIpcMemLazyEnablePeerAccess);
+        if (err != cudaSuccess) return cuda_fail(err, "cudaIpcOpenMemHandle (is worker's buffer in another process on a device this one can reach?)");
+        ctx->x_opened.push_back(buffers[n]);
+    }
+    return wash_exchange_staging(ctx, stack, parity, buffers.data(), ctx->x_capacity[parity][stack]);
 }
 
 int wash_exchange_plan(wash_ctx *ctx, uint64_t step, double p, const double *p_layer, uint64_t seed, void *stream_v)

@@ -199,3 +199,54 @@ def test_state_errors_are_reported_before_any_launch():
         B.wash_exchange_bind(ctx, 2, 0, B.WASH_F32, row, 64)   # already worker 1
     torch.cuda.synchronize()
     B.wash_destroy(ctx)
+
+
+# ---- workers in separate processes: buffers mapped through inter-process handles ----------
+# Two processes share the one GPU; they are ordered on the host (gloo), no kernel waits for
+# another process's kernel.
+
+def _process_worker(rank, world, port, out_dir):
+    import os
+    import torch.distributed as dist
+    from paper_2405_17517_b200.exchange import ExchangeWorker
+    os.environ["MASTER_ADDR"] = "127.0.0.1"
+    os.environ["MASTER_PORT"] = str(port)
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    try:
+        torch.cuda.set_device(0)
+        numel = [70001, 9, 4000]
+        off, P = W.padded_offsets(numel)
+        stack = W.to_stack(W.flat_population(world, sum(numel), seed=41), numel, off, P, 0)
+        mom = W.to_stack(W.flat_population(world, sum(numel), seed=42, std=1e-3), numel, off, P, 0)
+        row = to_device(stack.reshape(world, P)[rank])
+        opt = to_device(mom.reshape(world, P)[rank])
+        stats = torch.zeros(2, dtype=torch.int64, device="cuda")
+        worker = ExchangeWorker(numel, row, opt, capacity=P // 2)
+        pop = oracle.Population(world, numel, off, P, 0)
+        pl = [0.05, 1.0, 0.2]
+        ok = True
+        for step in range(3):
+            worker.step(step, 0.0, pl, seed=17, stats=stats)
+            torch.cuda.synchronize()
+            worker.check()
+            rows = [None] * world
+            dist.all_gather_object(rows, (to_host_bits(row), to_host_bits(opt), int(stats[1].item())))
+            sel, moved = oracle.shuffle(pop, stack, pl, seed=17, step=step, stack2=mom)
+            ok = ok and (np.concatenate([r[0] for r in rows]) == bits(stack)).all()
+            ok = ok and (np.concatenate([r[1] for r in rows]) == bits(mom)).all()
+        worker.close()
+        if rank == 0:
+            with open(os.path.join(out_dir, "result.txt"), "w") as f:
+                f.write("ok" if ok else "mismatch")
+    finally:
+        dist.destroy_process_group()
+
+
+def test_workers_in_two_processes_exchange_through_mapped_buffers(tmp_path):
+    import socket
+    import torch.multiprocessing as mp
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        port = s.getsockname()[1]
+    mp.spawn(_process_worker, args=(2, port, str(tmp_path)), nprocs=2, join=True)
+    assert (tmp_path / "result.txt").read_text() == "ok"
