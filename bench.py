@@ -494,6 +494,69 @@ def run_sweep(args) -> None:
                 torch.cuda.empty_cache()
 
 
+def run_exchange(args) -> None:
+    """One worker of the one-model-per-device form, timed alone on this GPU: plan (mask,
+    permutations, slot offsets), send (stores into the peers' staging buffers, here plain
+    buffers on the same device) and receive, per workload.  One JSON line each (not the
+    driver's bench line)."""
+    import torch
+    from paper_2405_17517_b200 import binding as B
+
+    torch.cuda.set_device(0)
+    B.load()
+    stream = torch.cuda.current_stream()
+    names = [args.workload] if args.workload_given else ["cfg2_resnet18_n5", "cfg3_resnet50_n10", "cfg4_resnet50_bf16_n8"]
+    for name in names:
+        wl = Workload(name)
+        ctx = B.wash_create_segments(wl.N, wl.numel, None, None, 0, 0)
+        P = B.wash_stack_elems(ctx, wl.T)[0]
+        p_layer = B.wash_layer_probs(wl.T, wl.p, 0) if wl.schedule == "decreasing" else None
+        gen = torch.Generator(device="cuda").manual_seed(SEED)
+        row = (torch.randn(P, generator=gen, device="cuda") * 0.05).to(torch.bfloat16 if wl.bf16 else torch.float32)
+        rows = [row]
+        B.wash_exchange_bind(ctx, 0, 0, B.WASH_BF16 if wl.bf16 else B.WASH_F32, row, P)
+        if wl.opt:
+            rows.append(torch.randn(P, generator=gen, device="cuda") * 1e-3)
+            B.wash_exchange_bind(ctx, 0, 1, B.WASH_F32, rows[1], P)
+        cap = max(1 << 16, int(4 * wl.p * wl.P))
+        keep = []
+        for k, r in enumerate(rows):
+            for parity in (0, 1):
+                bufs = [torch.zeros(cap, dtype=r.dtype, device="cuda") for _ in range(wl.N)]
+                keep.append(bufs)
+                B.wash_exchange_staging(ctx, k, parity, bufs, cap)
+        stats = torch.zeros(2, dtype=torch.int64, device="cuda")
+        flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")   # larger than L2
+        reps = 30
+        ev = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(reps)]
+        for i in range(3 + reps):
+            flush.zero_()
+            e = ev[max(i - 3, 0)]
+            e[0].record(stream)
+            B.wash_exchange_plan(ctx, i, wl.p, p_layer, SEED, stream)
+            e[1].record(stream)
+            B.wash_exchange_send(ctx, stream)
+            e[2].record(stream)
+            B.wash_exchange_receive(ctx, stream, stats if i >= 3 else None)
+            e[3].record(stream)
+        torch.cuda.synchronize()
+        B.wash_check(ctx)
+        med = lambda a, b: float(np.median([e[a].elapsed_time(e[b]) for e in ev])) * 1e3
+        sel, recv = int(stats[0]) / reps, int(stats[1]) / reps
+        elem = (wl.E + wl.E_opt)
+        print(json.dumps({
+            "workload": name, "worker": 0, "N": wl.N, "coordinates": wl.P,
+            "plan_us": med(0, 1), "send_us": med(1, 2), "receive_us": med(2, 3), "step_us": med(0, 3),
+            "selected_per_step": sel, "values_received_per_step": recv,
+            "link_bytes_in_per_step": recv * elem, "model_bytes": wl.P * elem,
+            "mask_coordinates_per_s": wl.P / (med(0, 1) * 1e-6),
+            "note": "L2 flushed before every step; peers' buffers are on the same device",
+        }), flush=True)
+        B.wash_destroy(ctx)
+        del keep, rows, row, flush
+        torch.cuda.empty_cache()
+
+
 def main() -> None:
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -513,7 +576,9 @@ def main() -> None:
     ap.add_argument("--sweep-logP", default="", help="comma list; default 20,24,27")
     ap.add_argument("--sweep-p", default="", help="comma list; default 1e-4..1")
     ap.add_argument("--sweep-layout", default="", choices=["", "np", "pn"])
+    ap.add_argument("--exchange", action="store_true", help="time one worker of the one-model-per-device form (JSON line per workload)")
     args = ap.parse_args()
+    args.workload_given = any(a == "--workload" or a.startswith("--workload=") for a in sys.argv[1:])
     if args.warmup < 3 and args.impl == "ours":
         args.warmup = 3
     rank = int(os.environ.get("RANK", "0"))
@@ -521,6 +586,9 @@ def main() -> None:
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
     if args.sweep:
         run_sweep(args)
+        return
+    if args.exchange:
+        run_exchange(args)
         return
     if args.impl == "reference":
         run_reference(args, rank, world)

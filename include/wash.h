@@ -238,7 +238,7 @@ int wash_step_host(wash_ctx *ctx, int32_t ops, void *host_params, void *host_opt
  * dev_row is a DEVICE row of padded_P elements (n_elems must say so) of `dtype`, 16-byte
  * aligned, for `stack` (WASH_STACK_PARAMS, or WASH_STACK_OPT for the optimizer state,
  * which then follows the same mask and permutations).  NULL unbinds.  The first call
- * allocates the plan's tables (padded_P/4 bytes + 4 (N+1) padded_P/1024 bytes). */
+ * allocates the plan's tables (about padded_P/4 bytes + 4 (N+1) padded_P/4096 bytes). */
 int wash_exchange_bind(wash_ctx *ctx, int32_t self, int32_t stack, int32_t dtype, void *dev_row, int64_t n_elems);
 
 /* Registers staging set `parity` (0 or 1) of `stack`: buffers is a HOST array of N

@@ -98,7 +98,7 @@ struct wash_ctx {
     int x_self = -1;
     void *x_row[2] = {nullptr, nullptr};
     int x_dtype[2] = {0, 0};
-    uint8_t *x_mask = nullptr;             // a byte per group
+    uint8_t *x_mask = nullptr;             // a byte per group, whole tiles
     uint32_t *x_count = nullptr;           // [N + 1][x_tiles]
     uint32_t *x_total = nullptr;           // [N + 1]
     uint32_t x_tiles = 0;
@@ -700,7 +700,7 @@ int wash_exchange_bind(wash_ctx *ctx, int32_t self, int32_t stack, int32_t dtype
         const uint32_t tiles = (ctx->n_groups + wash::kExchangeTileGroups - 1) / wash::kExchangeTileGroups;
         const size_t columns = static_cast<size_t>(ctx->N) + 1;
         cudaError_t err;
-        if ((err = cudaMalloc(&ctx->x_mask, ctx->n_groups)) != cudaSuccess ||
+        if ((err = cudaMalloc(&ctx->x_mask, static_cast<size_t>(tiles) * wash::kExchangeTileGroups)) != cudaSuccess ||
             (err = cudaMalloc(&ctx->x_count, sizeof(uint32_t) * columns * tiles)) != cudaSuccess ||
             (err = cudaMalloc(&ctx->x_total, sizeof(uint32_t) * columns)) != cudaSuccess) {
             cudaGetLastError();

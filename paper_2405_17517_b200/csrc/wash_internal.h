@@ -65,14 +65,14 @@ struct ReduceArgs {
 };
 
 // One model per device (wash_exchange_*): the row is one model of a population of pop.N.
-constexpr int kExchangeTileGroups = 256;   // a tile = one block = 256 groups = 1024 coordinates
+constexpr int kExchangeTileGroups = 1024;   // a tile = one block = 1024 groups = 4096 coordinates
 struct ExchangeArgs {
     PopView pop;
     int self;                     // this worker's index in the population
     uint32_t n_tiles;             // ceil(n_groups / kExchangeTileGroups)
     uint32_t key0, key1;
     uint32_t step_lo, step_hi8;
-    uint8_t *mask;                // [n_groups] low nibble: selected coordinates; high nibble: those this worker receives
+    uint8_t *mask;                // [n_tiles * kExchangeTileGroups] low nibble: selected coordinates; high nibble: those this worker receives
     uint32_t *tile_count;         // [N + 1][n_tiles]: column n = slots of worker n's buffer per tile (after the scan:
                                   // slots before the tile); column N = selected coordinates
     uint32_t *total;              // [N + 1] column totals

@@ -115,6 +115,22 @@ def test_workers_reproduce_the_population_shuffle(N, dtype, opt_dtype):
     w.close()
 
 
+@pytest.mark.parametrize("p", [1.0, 0.6])
+@pytest.mark.parametrize("N", [3, 20])
+def test_dense_selection_needs_several_passes_over_a_tile(N, p):
+    """More selected coordinates in a tile than the send kernel lists at once."""
+    w = Workers(N, [9000, 5, 4099], "f32", "f32", seed=50 + N)
+    for step in (0, 3):
+        w.step(step, p, None, seed=6)
+        oracle.shuffle(w.ora, w.host[0], p, seed=6, step=step, stack2=w.host[1])
+    w.check()
+    for k in range(2):
+        assert (to_host_bits(w.dev[k]) == bits(w.host[k])).all()
+    need, sel = oracle.exchange_counts(w.ora, p, seed=6, step=3)
+    assert B.wash_exchange_counts(w.ctx[1], N) == (need.tolist(), sel)
+    w.close()
+
+
 def test_resnet_rows_with_the_layer_schedule():
     """ResNet-18 tensor table, N = 5, the default layer-wise schedule, parameters and momentum."""
     numel = W.numels(W.resnet18_table(100))
