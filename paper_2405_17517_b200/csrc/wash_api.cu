@@ -98,10 +98,10 @@ struct wash_ctx {
     int x_self = -1;
     void *x_row[2] = {nullptr, nullptr};
     int x_dtype[2] = {0, 0};
-    uint8_t *x_mask = nullptr;             // a byte per group, whole tiles
-    uint32_t *x_count = nullptr;           // [N + 1][x_tiles]
-    uint32_t *x_total = nullptr;           // [N + 1]
-    uint32_t x_tiles = 0;
+    uint32_t *x_mask = nullptr;            // a byte per group, whole warp tiles
+    uint32_t *x_warp_total = nullptr;      // [x_blocks * kExchangeWarps][N + 1]
+    uint32_t *x_block_total = nullptr;     // [x_blocks][N + 1]
+    uint32_t x_wtiles = 0, x_blocks = 0, x_tiles_per_warp = 0;
     void **x_staging[2][2] = {{nullptr, nullptr}, {nullptr, nullptr}};   // [parity][stack]: device array of N pointers
     int64_t x_capacity[2][2] = {{0, 0}, {0, 0}};
     void *x_own[2][2] = {{nullptr, nullptr}, {nullptr, nullptr}};        // staging buffers this library allocated
@@ -123,8 +123,8 @@ void release(wash_ctx *ctx)
     if (ctx->stat_slots_dev) cudaFree(ctx->stat_slots_dev);
     if (ctx->avg_dev) cudaFree(ctx->avg_dev);
     if (ctx->x_mask) cudaFree(ctx->x_mask);
-    if (ctx->x_count) cudaFree(ctx->x_count);
-    if (ctx->x_total) cudaFree(ctx->x_total);
+    if (ctx->x_warp_total) cudaFree(ctx->x_warp_total);
+    if (ctx->x_block_total) cudaFree(ctx->x_block_total);
     for (auto &set : ctx->x_staging)
         for (void **ptrs : set)
             if (ptrs) cudaFree(ptrs);
@@ -648,14 +648,16 @@ int exchange_args(wash_ctx *ctx, wash::ExchangeArgs *out)
     wash::ExchangeArgs &a = *out;
     a.pop = view_of(ctx);
     a.self = ctx->x_self;
-    a.n_tiles = ctx->x_tiles;
+    a.n_wtiles = ctx->x_wtiles;
+    a.tiles_per_warp = ctx->x_tiles_per_warp;
+    a.n_blocks = ctx->x_blocks;
     a.key0 = static_cast<uint32_t>(ctx->x_seed);
     a.key1 = static_cast<uint32_t>(ctx->x_seed >> 32);
     a.step_lo = static_cast<uint32_t>(ctx->x_step);
     a.step_hi8 = static_cast<uint32_t>(ctx->x_step >> 32) << 8;
     a.mask = ctx->x_mask;
-    a.tile_count = ctx->x_count;
-    a.total = ctx->x_total;
+    a.warp_total = ctx->x_warp_total;
+    a.block_total = ctx->x_block_total;
     const int parity = static_cast<int>(ctx->x_step & 1u);
     for (int k = 0; k < 2; ++k) {
         a.row[k] = ctx->x_row[k];
@@ -697,20 +699,26 @@ int wash_exchange_bind(wash_ctx *ctx, int32_t self, int32_t stack, int32_t dtype
     if (!ctx->x_mask) {
         DeviceGuard guard(ctx->device);
         if (guard.err != cudaSuccess) return cuda_fail(guard.err, "cudaSetDevice");
-        const uint32_t tiles = (ctx->n_groups + wash::kExchangeTileGroups - 1) / wash::kExchangeTileGroups;
+        // a warp visits tiles_per_warp consecutive warp tiles; the grid is at most four blocks per SM (what the plan kernel fits)
+        const uint32_t wtiles = (ctx->n_groups + wash::kExchangeTileGroups - 1) / wash::kExchangeTileGroups;
+        const uint32_t max_warps = static_cast<uint32_t>(ctx->shape.sm_count > 0 ? ctx->shape.sm_count : 148) * 4u * wash::kExchangeWarps;
+        const uint32_t per_warp = (wtiles + max_warps - 1) / max_warps;
+        const uint32_t blocks = (wtiles + per_warp * wash::kExchangeWarps - 1) / (per_warp * wash::kExchangeWarps);
         const size_t columns = static_cast<size_t>(ctx->N) + 1;
         cudaError_t err;
-        if ((err = cudaMalloc(&ctx->x_mask, static_cast<size_t>(tiles) * wash::kExchangeTileGroups)) != cudaSuccess ||
-            (err = cudaMalloc(&ctx->x_count, sizeof(uint32_t) * columns * tiles)) != cudaSuccess ||
-            (err = cudaMalloc(&ctx->x_total, sizeof(uint32_t) * columns)) != cudaSuccess) {
+        if ((err = cudaMalloc(&ctx->x_mask, sizeof(uint32_t) * 32u * static_cast<size_t>(wtiles))) != cudaSuccess ||
+            (err = cudaMalloc(&ctx->x_warp_total, sizeof(uint32_t) * columns * blocks * wash::kExchangeWarps)) != cudaSuccess ||
+            (err = cudaMalloc(&ctx->x_block_total, sizeof(uint32_t) * columns * blocks)) != cudaSuccess) {
             cudaGetLastError();
             if (ctx->x_mask) cudaFree(ctx->x_mask);
-            if (ctx->x_count) cudaFree(ctx->x_count);
+            if (ctx->x_warp_total) cudaFree(ctx->x_warp_total);
             ctx->x_mask = nullptr;
-            ctx->x_count = nullptr;
+            ctx->x_warp_total = nullptr;
             return fail(WASH_ERR_ALLOC, "device allocation of the exchange tables failed: %s", cudaGetErrorString(err));
         }
-        ctx->x_tiles = tiles;
+        ctx->x_wtiles = wtiles;
+        ctx->x_tiles_per_warp = per_warp;
+        ctx->x_blocks = blocks;
     }
     ctx->x_self = self;
     ctx->x_row[stack] = dev_row;
@@ -846,10 +854,14 @@ int wash_exchange_counts(wash_ctx *ctx, uint64_t *host_need, uint64_t *host_sele
     DeviceGuard guard(ctx->device);
     if (guard.err != cudaSuccess) return cuda_fail(guard.err, "cudaSetDevice");
     cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
-    std::vector<uint32_t> total(static_cast<size_t>(ctx->N) + 1);
-    cudaError_t err = cudaMemcpyAsync(total.data(), ctx->x_total, sizeof(uint32_t) * total.size(), cudaMemcpyDeviceToHost, stream);
+    const size_t columns = static_cast<size_t>(ctx->N) + 1;
+    std::vector<uint32_t> per_block(columns * ctx->x_blocks);
+    cudaError_t err = cudaMemcpyAsync(per_block.data(), ctx->x_block_total, sizeof(uint32_t) * per_block.size(), cudaMemcpyDeviceToHost, stream);
     if (err == cudaSuccess) err = cudaStreamSynchronize(stream);
     if (err != cudaSuccess) return cuda_fail(err, "reading the plan's totals");
+    std::vector<uint64_t> total(columns, 0);
+    for (size_t b = 0; b < ctx->x_blocks; ++b)
+        for (size_t col = 0; col < columns; ++col) total[col] += per_block[b * columns + col];
     if (host_need)
         for (int n = 0; n < ctx->N; ++n) host_need[n] = total[static_cast<size_t>(n)];
     if (host_selected) *host_selected = total[static_cast<size_t>(ctx->N)];

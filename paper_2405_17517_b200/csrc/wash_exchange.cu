@@ -6,18 +6,22 @@
 // value of the coordinate straight into the slot (a peer store when the buffer lives on
 // another device).  After all workers have sent, each one copies its slots into its model.
 //
-// Three kernels and a small scan, all on tiles of 1024 groups (4096 coordinates; a block of
-// 256 threads, four consecutive groups per thread so that the four Philox draws overlap):
-//   plan     draws the mask (one Philox block per group) and, for selected coordinates, the
-//            permutation; writes one byte per group (low nibble: selected coordinates, high
-//            nibble: those whose new value comes from another worker) and, per tile, how many
-//            slots of every worker's buffer the tile takes (+ the selected count)
-//   scan     turns each worker's column of tile counts into slot offsets (one block per column)
-//   send     lists the tile's selected coordinates in order, redraws their permutations, and
-//            lets thread n walk the list for worker n: it counts worker n's slots and stores
-//            this worker's value where pi_i(n) is this worker
-//   receive  reads the bytes, numbers its own slots with a block scan and copies them in
+// Work is cut into warp tiles of 128 groups (512 coordinates: a lane owns four consecutive
+// groups, so its four Philox draws overlap and its four mask bytes move as one word).  A
+// warp owns a contiguous range of warp tiles and visits them in order, which turns "the
+// slot of a coordinate" into a running count: no per-tile offsets are stored, only one
+// total per warp and per block, and the kernels need no block-wide barrier inside the loop.
+//   plan     draws the mask and, for selected coordinates, the permutation; writes a byte per
+//            group (low nibble: selected coordinates, high nibble: those whose new value comes
+//            from another worker) and, per warp and per block, how many slots of every
+//            worker's buffer its range takes (+ the selected count)
+//   send     adds up the totals of the blocks and warps before it (its first slots), then
+//            replays its range: redraws the permutations of the selected coordinates, numbers
+//            every worker's slots with warp votes and stores this worker's value where
+//            pi_i(n) is this worker
+//   receive  the same replay for its own buffer only, from the high nibbles: no draw at all
 // The plan reads no model data; send and receive touch only selected coordinates.
+// All three kernels must be launched with the same grid (n_blocks) and tiles_per_warp.
 #include "wash_device.cuh"
 #include "wash_launch.cuh"
 #include "wash_shuffle_tma.cuh"     // draw_permutation_u8
@@ -25,157 +29,184 @@
 
 namespace wash {
 
-constexpr int kXThreads = 256;
-constexpr int kXPerThread = kExchangeTileGroups / kXThreads;   // consecutive groups per thread
-static_assert(kXPerThread == 4, "a thread's mask bytes are moved as one 32-bit word");
-constexpr int kXList = 1024;   // selected coordinates listed per pass of the send kernel
+constexpr int kXThreads = 32 * kExchangeWarps;
+constexpr uint32_t kFull = 0xFFFFFFFFu;
+constexpr uint32_t kNoDestination = 0xFFu;
 
-// exclusive prefix sum of `mine` over the block's threads (in thread order); *total = block sum
-__device__ __forceinline__ uint32_t block_exclusive_scan(uint32_t mine, uint32_t *s_warp, uint32_t *total)
+// What a lane knows about its four consecutive groups g0 .. g0+3.
+struct LaneGroups {
+    bool one_tensor;   // all four lie in one tensor (the usual case): described by the fields below
+    uint32_t cgroup0, tensor;
+    uint64_t thr;
+    long long left;    // coordinates of the tensor from the first group on
+};
+
+__device__ __forceinline__ LaneGroups describe_groups(const ExchangeArgs &a, uint32_t g0, uint32_t &cursor)
 {
-    const uint32_t lane = threadIdx.x & 31u, warp = threadIdx.x >> 5;
-    uint32_t upto = mine;
-#pragma unroll
-    for (int d = 1; d < 32; d <<= 1) {
-        const uint32_t v = __shfl_up_sync(0xFFFFFFFFu, upto, d);
-        if (lane >= static_cast<uint32_t>(d)) upto += v;
-    }
-    if (lane == 31) s_warp[warp] = upto;
-    __syncthreads();
-    uint32_t before = 0, sum = 0;
-#pragma unroll
-    for (int w = 0; w < kXThreads / 32; ++w) {
-        const uint32_t v = s_warp[w];
-        if (static_cast<uint32_t>(w) < warp) before += v;
-        sum += v;
-    }
-    *total = sum;
-    return before + upto - mine;
+    LaneGroups lg{true, 0, 0, 0, 0};
+    if (g0 >= a.pop.n_groups) return lg;   // thr == 0: nothing to draw
+    const GroupInfo gi = find_group_forward(a.pop.seg, a.pop.n_seg, cursor, g0, a.status);
+    const SegEntry &seg = a.pop.seg[cursor];
+    lg.one_tensor = g0 + 4 <= seg.group_end;
+    lg.cgroup0 = gi.cgroup;
+    lg.tensor = gi.tensor_id;
+    lg.thr = gi.thr;
+    lg.left = static_cast<long long>(seg.numel) - 4ll * (gi.cgroup - seg.cgroup_begin);
+    return lg;
 }
 
-// source model pi(n) out of either representation of the permutation
-__device__ __forceinline__ int perm_source(int n_models, uint64_t packed, const uint8_t *s_perm, int n)
+// group q of the lane
+__device__ __forceinline__ GroupInfo lane_group(const ExchangeArgs &a, const LaneGroups &lg, uint32_t g0, int q)
 {
-    return n_models <= 16 ? static_cast<int>((packed >> (4 * n)) & 15ull) : static_cast<int>(s_perm[n * kXThreads]);
+    if (lg.one_tensor) {
+        const long long l = lg.left - 4 * q;
+        return GroupInfo{lg.tensor, lg.cgroup0 + q, l >= 4 ? 4 : (l > 0 ? static_cast<int>(l) : 0), lg.thr};
+    }
+    if (g0 + q >= a.pop.n_groups) return GroupInfo{0, 0, 0, 0};
+    return find_group(a.pop, g0 + q, a.status);
 }
-
-// the four groups of this thread: g0 .. g0+3
-__device__ __forceinline__ uint32_t first_group() { return (blockIdx.x * kXThreads + threadIdx.x) * kXPerThread; }
 
 // the mask of one group: bit c set iff coordinate c is selected
-__device__ __forceinline__ uint32_t draw_mask(uint32_t cgroup, uint32_t tensor, uint64_t thr, int valid, const ExchangeArgs &a)
+__device__ __forceinline__ uint32_t draw_mask(const GroupInfo &gi, const ExchangeArgs &a)
 {
-    const Philox4 w = philox4x32_10(cgroup, tensor, a.step_lo, a.step_hi8, a.key0, a.key1);
-    const uint32_t thr_lo = static_cast<uint32_t>(thr);
-    const bool always = (thr >> 32) != 0;
+    if (gi.thr == 0 || gi.valid == 0) return 0;
+    const Philox4 w = philox4x32_10(gi.cgroup, gi.tensor_id, a.step_lo, a.step_hi8, a.key0, a.key1);
+    const uint32_t thr_lo = static_cast<uint32_t>(gi.thr);
+    const bool always = (gi.thr >> 32) != 0;
     uint32_t m = 0;
     m |= (w.x < thr_lo || always) ? 1u : 0u;
     m |= (w.y < thr_lo || always) ? 2u : 0u;
     m |= (w.z < thr_lo || always) ? 4u : 0u;
     m |= (w.w < thr_lo || always) ? 8u : 0u;
-    return m & ((1u << valid) - 1u);
+    return m & ((1u << gi.valid) - 1u);
 }
 
-// Permutations of a group's selected coordinates: counts every worker's slots in s_count and
-// returns the group's byte (low nibble sel, high nibble the coordinates this worker receives).
-__device__ __forceinline__ uint32_t plan_selected(uint32_t sel, uint32_t cgroup, uint32_t tensor, uint8_t *s_perm,
-                                                  uint32_t *s_count, const ExchangeArgs &a)
+__device__ __forceinline__ uint32_t warp_exclusive_scan(uint32_t mine, uint32_t *total)
+{
+    const uint32_t lane = threadIdx.x & 31u;
+    uint32_t upto = mine;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+        const uint32_t v = __shfl_up_sync(kFull, upto, d);
+        if (lane >= static_cast<uint32_t>(d)) upto += v;
+    }
+    *total = __shfl_sync(kFull, upto, 31);
+    return upto - mine;
+}
+
+// The selected coordinates of a warp's range are few and scattered: serving each where it is
+// found would leave 31 lanes idle.  Instead the warp queues them, in coordinate order, as
+// row elements in a ring in shared memory and serves them 32 at a time, one per lane.
+constexpr uint32_t kXRing = 1024;   // entries; a warp tile adds at most 512, a round removes 32
+
+// appends the lane's selected coordinates of warp tile t (sel4: a nibble per byte, one byte per group)
+__device__ __forceinline__ uint32_t ring_append(uint32_t *ring, uint32_t tail, uint32_t sel4, uint32_t t)
+{
+    const uint32_t lane = threadIdx.x & 31u;
+    uint32_t total = 0;
+    uint32_t pos = tail + warp_exclusive_scan(__popc(sel4), &total);
+    const uint32_t elem0 = 4u * (t * kExchangeTileGroups + 4u * lane);   // rows are shorter than 2^32 elements
+    for (uint32_t left = sel4; left; left &= left - 1u, ++pos) {
+        const uint32_t bit = static_cast<uint32_t>(__ffs(left) - 1);   // byte q = bit / 8, coordinate c = bit % 8
+        ring[pos % kXRing] = elem0 + 4u * (bit >> 3) + (bit & 7u);
+    }
+    __syncwarp();
+    return tail + total;
+}
+
+// pi of the coordinate stored at row element `elem`, as {need: bit n set iff pi(n) != n,
+// dest: the n != self with pi(n) == self, if any}
+__device__ __forceinline__ void routes_of(const ExchangeArgs &a, uint32_t elem, uint8_t *s_perm,
+                                          unsigned long long *need, uint32_t *dest)
 {
     const int n_models = a.pop.N;
-    uint32_t byte = sel;
-    for (uint32_t left = sel; left; left &= left - 1u) {
-        const int c = __ffs(left) - 1;
-        uint64_t packed = 0;
-        if (n_models <= 16) packed = draw_permutation_packed(n_models, 4u * cgroup + c, tensor, a.step_lo, a.step_hi8, a.key0, a.key1);
-        else draw_permutation_u8(s_perm, kXThreads, n_models, 4u * cgroup + c, tensor, a.step_lo, a.step_hi8, a.key0, a.key1);
-        for (int n = 0; n < n_models; ++n)
-            if (perm_source(n_models, packed, s_perm, n) != n) {
-                atomicAdd(&s_count[n], 1u);
-                if (n == a.self) byte |= 16u << c;
-            }
-        atomicAdd(&s_count[n_models], 1u);
+    const GroupInfo gi = find_group(a.pop, elem >> 2, a.status);
+    const uint32_t coord = 4u * gi.cgroup + (elem & 3u);
+    uint64_t packed = 0;
+    if (n_models <= 16) packed = draw_permutation_packed(n_models, coord, gi.tensor_id, a.step_lo, a.step_hi8, a.key0, a.key1);
+    else draw_permutation_u8(s_perm, kXThreads, n_models, coord, gi.tensor_id, a.step_lo, a.step_hi8, a.key0, a.key1);
+    unsigned long long nd = 0;
+    uint32_t d = kNoDestination;
+    for (int n = 0; n < n_models; ++n) {
+        const int src = n_models <= 16 ? static_cast<int>((packed >> (4 * n)) & 15ull) : static_cast<int>(s_perm[n * kXThreads]);
+        if (src == n) continue;
+        nd |= 1ull << n;
+        if (src == a.self) d = static_cast<uint32_t>(n);
     }
-    return byte;
+    *need = nd;
+    *dest = d;
 }
 
-__global__ void __launch_bounds__(kXThreads, 5) exchange_plan_kernel(const __grid_constant__ ExchangeArgs a)
+// first and one-past-last warp tile of this warp, and the cursor into the segment table for the first
+__device__ __forceinline__ void warp_range(const ExchangeArgs &a, uint32_t *t0, uint32_t *t1, uint32_t *cursor)
+{
+    const uint32_t range = blockIdx.x * kExchangeWarps + (threadIdx.x >> 5);
+    const uint64_t lo = static_cast<uint64_t>(range) * a.tiles_per_warp;
+    *t0 = static_cast<uint32_t>(min(lo, static_cast<uint64_t>(a.n_wtiles)));
+    *t1 = static_cast<uint32_t>(min(lo + a.tiles_per_warp, static_cast<uint64_t>(a.n_wtiles)));
+    const uint32_t g = *t0 * kExchangeTileGroups;
+    *cursor = (*t0 < *t1 && g < a.pop.n_groups) ? __ldg(a.pop.tile_first + (g >> kTileShift)) : 0u;
+}
+
+__global__ void __launch_bounds__(kXThreads, 4) exchange_plan_kernel(const __grid_constant__ ExchangeArgs a)
 {
     extern __shared__ uint8_t s_perm_all[];   // column per thread (kMaxN * kXThreads bytes) when N > 16, else nothing
-    __shared__ uint32_t s_count[kMaxN + 1];
-    uint8_t *s_perm = s_perm_all + threadIdx.x;
-    const int n_models = a.pop.N;
-    if (threadIdx.x <= static_cast<uint32_t>(n_models)) s_count[threadIdx.x] = 0;
-    __syncthreads();
-    const uint32_t g0 = first_group();
-    uint32_t bytes = 0;
-    if (g0 < a.pop.n_groups) {
-        uint32_t cursor = __ldg(a.pop.tile_first + (g0 >> kTileShift));
-        const GroupInfo gi0 = find_group_forward(a.pop.seg, a.pop.n_seg, cursor, g0, a.status);
-        const uint32_t seg_end = a.pop.seg[cursor].group_end;
-        if (g0 + kXPerThread <= seg_end) {
-            // the usual case: the thread's four groups lie in one tensor -- one table lookup,
-            // four independent Philox draws
-            if (gi0.thr != 0 && gi0.valid != 0) {
-                const long long left = static_cast<long long>(a.pop.seg[cursor].numel) - 4ll * (gi0.cgroup - a.pop.seg[cursor].cgroup_begin);
-                uint32_t sel[kXPerThread];
+    __shared__ uint32_t s_count[kExchangeWarps][kMaxN + 1];
+    __shared__ uint32_t s_ring[kExchangeWarps][kXRing];
+    const uint32_t lane = threadIdx.x & 31u, warp = threadIdx.x >> 5;
+    const int n_models = a.pop.N, columns = n_models + 1;
+    for (int col = lane; col < columns; col += 32) s_count[warp][col] = 0;
+    __syncwarp();
+    uint32_t t0, t1, cursor;
+    warp_range(a, &t0, &t1, &cursor);
+    uint32_t head = 0, tail = 0;   // ring positions served / queued so far
+    // one round: lane j takes entry head + j; counts every worker's slots and marks the
+    // coordinates this worker receives in the (already written) mask words
+    auto serve = [&](uint32_t count) {
+        if (lane < count) {
+            const uint32_t elem = s_ring[warp][(head + lane) % kXRing];
+            unsigned long long need;
+            uint32_t dest;
+            routes_of(a, elem, s_perm_all + threadIdx.x, &need, &dest);
+            for (unsigned long long left = need; left; left &= left - 1ull) atomicAdd(&s_count[warp][__ffsll(static_cast<long long>(left)) - 1], 1u);
+            atomicAdd(&s_count[warp][n_models], 1u);
+            if ((need >> a.self) & 1ull) {
+                const uint32_t g = elem >> 2;   // byte g % 4 of word g / 4, bit 4 + c
+                atomicOr(&a.mask[g >> 2], 16u << ((elem & 3u) + 8u * (g & 3u)));
+            }
+        }
+        __syncwarp();
+        head += count;
+    };
+    for (uint32_t t = t0; t < t1; ++t) {
+        const uint32_t g0 = t * kExchangeTileGroups + 4u * lane;
+        const LaneGroups lg = describe_groups(a, g0, cursor);
+        uint32_t sel4 = 0;
+        if (lg.one_tensor) {
+            if (lg.thr != 0) {
 #pragma unroll
-                for (int q = 0; q < kXPerThread; ++q) {
-                    const long long l = left - 4 * q;
-                    const int valid = l >= 4 ? 4 : (l > 0 ? static_cast<int>(l) : 0);
-                    sel[q] = draw_mask(gi0.cgroup + q, gi0.tensor_id, gi0.thr, valid, a);
-                }
-#pragma unroll
-                for (int q = 0; q < kXPerThread; ++q)
-                    if (sel[q]) bytes |= plan_selected(sel[q], gi0.cgroup + q, gi0.tensor_id, s_perm, s_count, a) << (8 * q);
+                for (int q = 0; q < 4; ++q) sel4 |= draw_mask(lane_group(a, lg, g0, q), a) << (8 * q);
             }
         } else {
 #pragma unroll 1
-            for (int q = 0; q < kXPerThread; ++q) {
-                if (g0 + q >= a.pop.n_groups) break;
-                const GroupInfo gi = find_group_forward(a.pop.seg, a.pop.n_seg, cursor, g0 + q, a.status);
-                if (gi.thr == 0 || gi.valid == 0) continue;
-                const uint32_t sel = draw_mask(gi.cgroup, gi.tensor_id, gi.thr, gi.valid, a);
-                if (sel) bytes |= plan_selected(sel, gi.cgroup, gi.tensor_id, s_perm, s_count, a) << (8 * q);
-            }
+            for (int q = 0; q < 4; ++q) sel4 |= draw_mask(lane_group(a, lg, g0, q), a) << (8 * q);
+        }
+        a.mask[static_cast<size_t>(t) * 32u + lane] = sel4;
+        if (__any_sync(kFull, sel4 != 0)) {
+            tail = ring_append(s_ring[warp], tail, sel4, t);   // orders the mask stores before the rounds' atomics, too
+            while (tail - head >= 32u) serve(32u);
         }
     }
-    reinterpret_cast<uint32_t *>(a.mask)[g0 / kXPerThread] = bytes;   // the array covers whole tiles
+    if (tail != head) serve(tail - head);
+    const uint32_t range = blockIdx.x * kExchangeWarps + warp;
+    for (int col = lane; col < columns; col += 32) a.warp_total[static_cast<size_t>(range) * columns + col] = s_count[warp][col];
     __syncthreads();
-    if (threadIdx.x <= static_cast<uint32_t>(n_models))
-        a.tile_count[static_cast<size_t>(threadIdx.x) * a.n_tiles + blockIdx.x] = s_count[threadIdx.x];
-}
-
-// One block per column: counts -> exclusive prefix sums in place, column total to a.total.
-__global__ void __launch_bounds__(1024) exchange_scan_kernel(const __grid_constant__ ExchangeArgs a)
-{
-    __shared__ uint32_t s_warp[32];
-    uint32_t *col = a.tile_count + static_cast<size_t>(blockIdx.x) * a.n_tiles;
-    const uint32_t chunk = (a.n_tiles + 1023u) / 1024u;
-    const uint32_t lo = min(threadIdx.x * chunk, a.n_tiles), hi = min(lo + chunk, a.n_tiles);
-    uint32_t sum = 0;
-    for (uint32_t t = lo; t < hi; ++t) sum += col[t];
-    const uint32_t lane = threadIdx.x & 31u, warp = threadIdx.x >> 5;
-    uint32_t upto = sum;
+    if (threadIdx.x < static_cast<uint32_t>(columns)) {
+        uint32_t sum = 0;
 #pragma unroll
-    for (int d = 1; d < 32; d <<= 1) {
-        const uint32_t v = __shfl_up_sync(0xFFFFFFFFu, upto, d);
-        if (lane >= static_cast<uint32_t>(d)) upto += v;
+        for (int w = 0; w < kExchangeWarps; ++w) sum += s_count[w][threadIdx.x];
+        a.block_total[static_cast<size_t>(blockIdx.x) * columns + threadIdx.x] = sum;
     }
-    if (lane == 31) s_warp[warp] = upto;
-    __syncthreads();
-    uint32_t before = 0, total = 0;
-    for (uint32_t w = 0; w < 32; ++w) {
-        const uint32_t v = s_warp[w];
-        if (w < warp) before += v;
-        total += v;
-    }
-    uint32_t run = before + upto - sum;
-    for (uint32_t t = lo; t < hi; ++t) {
-        const uint32_t v = col[t];
-        col[t] = run;
-        run += v;
-    }
-    if (threadIdx.x == 0) a.total[blockIdx.x] = total;
 }
 
 __device__ __forceinline__ void copy_element(void *dst, long long dst_idx, const void *src, long long src_idx, int dtype)
@@ -184,148 +215,163 @@ __device__ __forceinline__ void copy_element(void *dst, long long dst_idx, const
     else static_cast<uint16_t *>(dst)[dst_idx] = static_cast<const uint16_t *>(src)[src_idx];
 }
 
-// A selected coordinate's value of this worker goes to at most one other worker: the n with
-// pi(n) = self (pi is a permutation), unless pi(self) = self and it stays.
-constexpr uint8_t kNoDestination = 0xFF;
+// Sum over the blocks before this one of column `col` of block_total, by one warp.
+__device__ __forceinline__ uint32_t blocks_before(const ExchangeArgs &a, int col)
+{
+    const uint32_t lane = threadIdx.x & 31u;
+    const int columns = a.pop.N + 1;
+    uint32_t sum = 0;
+    for (uint32_t b = lane; b < blockIdx.x; b += 32) sum += a.block_total[static_cast<size_t>(b) * columns + col];
+    return __reduce_add_sync(kFull, sum);
+}
 
 __global__ void __launch_bounds__(kXThreads) exchange_send_kernel(const __grid_constant__ ExchangeArgs a)
 {
-    extern __shared__ uint8_t s_perm_all[];         // kMaxN * kXThreads bytes when N > 16, else nothing
-    __shared__ unsigned long long s_need[kXList];   // bit n: the coordinate takes a slot of worker n
-    __shared__ uint32_t s_slot[kXList];             // slot of the destination's buffer this worker fills
-    __shared__ uint16_t s_offset[kXList];           // coordinate within the tile
-    __shared__ uint8_t s_dest[kXList];              // the worker that receives this worker's value
-    __shared__ uint32_t s_warp[kXThreads / 32];
-    uint8_t *s_perm = s_perm_all + threadIdx.x;
-    const int n_models = a.pop.N;
-    const uint32_t g0 = first_group();
-    const uint32_t bytes = reinterpret_cast<const uint32_t *>(a.mask)[g0 / kXPerThread];
-    const uint32_t sel4 = bytes & 0x0F0F0F0Fu;
-    if (!__syncthreads_or(sel4 != 0)) return;
-    uint32_t listed = 0;
-    const uint32_t first = block_exclusive_scan(__popc(sel4), s_warp, &listed);   // position of this thread's first entry
-    // thread n numbers worker n's slots
-    const int n = static_cast<int>(threadIdx.x);
-    const bool walker = n < n_models && n != a.self;
-    uint32_t slot = walker ? a.tile_count[static_cast<size_t>(n) * a.n_tiles + blockIdx.x] : 0u;
-    const long long tile_elem = 4ll * kExchangeTileGroups * static_cast<long long>(blockIdx.x);
-    uint32_t cursor = sel4 ? __ldg(a.pop.tile_first + (g0 >> kTileShift)) : 0u;
-    // the list is served kXList entries at a time (one pass unless p is large)
-    for (uint32_t base = 0; base < listed; base += kXList) {
-        if (sel4) {
-            uint32_t pos = first;
-#pragma unroll 1
-            for (int q = 0; q < kXPerThread; ++q) {
-                const uint32_t sel = (sel4 >> (8 * q)) & 15u;
-                if (!sel) continue;
-                if (pos + 4 <= base || pos >= base + kXList) { pos += __popc(sel); continue; }   // not in this pass
-                const GroupInfo gi = find_group_forward(a.pop.seg, a.pop.n_seg, cursor, g0 + q, a.status);
-#pragma unroll 1
-                for (int c = 0; c < 4; ++c) {
-                    if (!((sel >> c) & 1u)) continue;
-                    if (pos >= base && pos < base + kXList) {
-                        uint64_t packed = 0;
-                        if (n_models <= 16) packed = draw_permutation_packed(n_models, 4u * gi.cgroup + c, gi.tensor_id, a.step_lo, a.step_hi8, a.key0, a.key1);
-                        else draw_permutation_u8(s_perm, kXThreads, n_models, 4u * gi.cgroup + c, gi.tensor_id, a.step_lo, a.step_hi8, a.key0, a.key1);
-                        unsigned long long need = 0;
-                        uint8_t dest = kNoDestination;
-                        for (int m = 0; m < n_models; ++m) {
-                            const int src = perm_source(n_models, packed, s_perm, m);
-                            if (src == m) continue;
-                            need |= 1ull << m;
-                            if (src == a.self) dest = static_cast<uint8_t>(m);
-                        }
-                        s_need[pos - base] = need;
-                        s_dest[pos - base] = dest;
-                        s_offset[pos - base] = static_cast<uint16_t>(4u * (kXPerThread * threadIdx.x + q) + c);
-                    }
-                    ++pos;
-                }
+    extern __shared__ uint8_t s_perm_all[];
+    __shared__ uint32_t s_base[kMaxN];
+    __shared__ uint32_t s_ring[kExchangeWarps][kXRing];
+    const uint32_t lane = threadIdx.x & 31u, warp = threadIdx.x >> 5;
+    const int n_models = a.pop.N, columns = n_models + 1;
+    // slots of every worker's buffer taken before this block, then before this warp
+    for (int col = warp; col < n_models; col += kExchangeWarps) {
+        const uint32_t sum = blocks_before(a, col);
+        if (lane == 0) s_base[col] = sum;
+    }
+    __syncthreads();
+    uint32_t run[2] = {0, 0};   // next slot of worker lane (run[0]) and worker lane + 32 (run[1])
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+        const int col = static_cast<int>(lane) + 32 * h;
+        if (col >= n_models) continue;
+        uint32_t sum = s_base[col];
+        for (uint32_t w = 0; w < warp; ++w) sum += a.warp_total[static_cast<size_t>(blockIdx.x * kExchangeWarps + w) * columns + col];
+        run[h] = sum;
+    }
+    uint32_t t0, t1, cursor;
+    warp_range(a, &t0, &t1, &cursor);
+    uint32_t head = 0, tail = 0;
+    // one round: lane j takes entry head + j (coordinate order along the lanes); the warp votes
+    // worker by worker to number the slots, then every lane with a destination copies its value
+    auto serve = [&](uint32_t count) {
+        unsigned long long need = 0;
+        uint32_t dest = kNoDestination, elem = 0;
+        if (lane < count) {
+            elem = s_ring[warp][(head + lane) % kXRing];
+            routes_of(a, elem, s_perm_all + threadIdx.x, &need, &dest);
+        }
+        uint32_t slot = 0;
+        for (int n = 0; n < n_models; ++n) {
+            const uint32_t votes = __ballot_sync(kFull, (need >> n) & 1ull);
+            const uint32_t next = __shfl_sync(kFull, n < 32 ? run[0] : run[1], n & 31);
+            if (dest == static_cast<uint32_t>(n)) slot = next + __popc(votes & ((1u << lane) - 1u));
+            if (lane == static_cast<uint32_t>(n & 31)) {
+                if (n < 32) run[0] += __popc(votes);
+                else run[1] += __popc(votes);
             }
         }
-        __syncthreads();
-        const uint32_t count = min(listed - base, static_cast<uint32_t>(kXList));
-        if (walker) {   // shared memory only: no load from the model sits in this serial loop
-            for (uint32_t e = 0; e < count; ++e) {
-                if (!((s_need[e] >> n) & 1ull)) continue;
-                if (s_dest[e] == n) s_slot[e] = slot;
-                ++slot;
-            }
-        }
-        __syncthreads();
-        // the copies, one entry per thread: all loads of the pass are in flight together
-        for (uint32_t e = threadIdx.x; e < count; e += kXThreads) {
-            const uint32_t dest = s_dest[e];
-            if (dest == kNoDestination) continue;
-            const long long to = s_slot[e];
+        if (dest != kNoDestination) {
 #pragma unroll
             for (int k = 0; k < 2; ++k) {
                 if (!a.row[k]) continue;
-                if (to < a.capacity[k]) copy_element(a.staging[k][dest], to, a.row[k], tile_elem + s_offset[e], a.dtype[k]);
+                if (static_cast<long long>(slot) < a.capacity[k]) copy_element(a.staging[k][dest], slot, a.row[k], elem, a.dtype[k]);
                 else atomicOr(a.status, 4u);   // staging buffer too small: nothing is written beyond it
             }
         }
-        __syncthreads();   // the list is rewritten by the next pass
+        __syncwarp();
+        head += count;
+    };
+    for (uint32_t t = t0; t < t1; ++t) {
+        const uint32_t sel4 = a.mask[static_cast<size_t>(t) * 32u + lane] & 0x0F0F0F0Fu;
+        if (!__any_sync(kFull, sel4 != 0)) continue;
+        tail = ring_append(s_ring[warp], tail, sel4, t);
+        while (tail - head >= 32u) serve(32u);
     }
+    if (tail != head) serve(tail - head);
 }
 
 __global__ void __launch_bounds__(kXThreads) exchange_receive_kernel(const __grid_constant__ ExchangeArgs a)
 {
-    __shared__ uint32_t s_warp[kXThreads / 32];
-    if (a.stats && blockIdx.x == 0 && threadIdx.x == 0) {
-        atomicAdd(a.stats, static_cast<unsigned long long>(a.total[a.pop.N]));
-        atomicAdd(a.stats + 1, static_cast<unsigned long long>(a.total[a.self]));
+    __shared__ uint32_t s_part[kExchangeWarps];
+    const uint32_t lane = threadIdx.x & 31u, warp = threadIdx.x >> 5;
+    const int columns = a.pop.N + 1;
+    if (a.stats && blockIdx.x == 0 && warp < 2) {   // the step's totals: selected coordinates, values this worker receives
+        const int col = warp == 0 ? a.pop.N : a.self;
+        uint32_t sum = 0;
+        for (uint32_t b = lane; b < a.n_blocks; b += 32) sum += a.block_total[static_cast<size_t>(b) * columns + col];
+        sum = __reduce_add_sync(kFull, sum);
+        if (lane == 0) atomicAdd(a.stats + warp, static_cast<unsigned long long>(sum));
     }
-    const uint32_t g0 = first_group();
-    const uint32_t take4 = (reinterpret_cast<const uint32_t *>(a.mask)[g0 / kXPerThread] >> 4) & 0x0F0F0F0Fu;
-    if (!__syncthreads_or(take4 != 0)) return;
-    uint32_t total = 0;
-    uint32_t slot = a.tile_count[static_cast<size_t>(a.self) * a.n_tiles + blockIdx.x] + block_exclusive_scan(__popc(take4), s_warp, &total);
-    if (!take4) return;
-    const void *src[2] = {a.row[0] ? a.staging[0][a.self] : nullptr, a.row[1] ? a.staging[1][a.self] : nullptr};
-#pragma unroll 1
-    for (int q = 0; q < kXPerThread; ++q) {
-        const uint32_t take = (take4 >> (8 * q)) & 15u;
+    // slots of this worker's buffer taken before this block (all warps share the sum), then before this warp
+    {
+        uint32_t sum = 0;
+        for (uint32_t b = threadIdx.x; b < blockIdx.x; b += kXThreads) sum += a.block_total[static_cast<size_t>(b) * columns + a.self];
+        sum = __reduce_add_sync(kFull, sum);
+        if (lane == 0) s_part[warp] = sum;
+    }
+    __syncthreads();
+    uint32_t run = 0;
 #pragma unroll
-        for (int c = 0; c < 4; ++c) {
-            if (!((take >> c) & 1u)) continue;
+    for (int w = 0; w < kExchangeWarps; ++w) run += s_part[w];
+    for (uint32_t w = 0; w < warp; ++w) run += a.warp_total[static_cast<size_t>(blockIdx.x * kExchangeWarps + w) * columns + a.self];
+    uint32_t t0, t1, cursor;
+    warp_range(a, &t0, &t1, &cursor);
+    const void *src[2] = {a.row[0] ? a.staging[0][a.self] : nullptr, a.row[1] ? a.staging[1][a.self] : nullptr};
+    for (uint32_t t = t0; t < t1; ++t) {
+        const uint32_t take4 = (a.mask[static_cast<size_t>(t) * 32u + lane] >> 4) & 0x0F0F0F0Fu;
+        if (!__any_sync(kFull, take4 != 0)) continue;
+        uint32_t total = 0;
+        uint32_t slot = run + warp_exclusive_scan(__popc(take4), &total);
+        run += total;
+        const long long lane_elem = 4ll * (static_cast<long long>(t) * kExchangeTileGroups + 4u * lane);
+        for (uint32_t left = take4; left; left &= left - 1u, ++slot) {
+            const int bit = __ffs(left) - 1;   // byte q = bit / 8, coordinate c = bit % 8
+            const long long elem = lane_elem + 4 * (bit >> 3) + (bit & 7);
 #pragma unroll
             for (int k = 0; k < 2; ++k) {
                 if (!a.row[k]) continue;
-                if (static_cast<long long>(slot) < a.capacity[k]) copy_element(a.row[k], 4ll * (g0 + q) + c, src[k], slot, a.dtype[k]);
+                if (static_cast<long long>(slot) < a.capacity[k]) copy_element(a.row[k], elem, src[k], slot, a.dtype[k]);
                 else atomicOr(a.status, 4u);
             }
-            ++slot;
         }
     }
 }
 
+// Populations above 16 models keep their permutations in a column of bytes per thread: with
+// the kernels' static shared memory that is more than the default 48 KiB per block, so the
+// kernel's limit is raised first.
+static cudaError_t perm_smem(const ExchangeArgs &args, const void *kernel, size_t *bytes)
+{
+    *bytes = args.pop.N > 16 ? static_cast<size_t>(kMaxN) * kXThreads : 0;
+    if (*bytes == 0) return cudaSuccess;
+    return cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(*bytes));
+}
+
 cudaError_t launch_exchange_plan(const ExchangeArgs &args, cudaStream_t stream)
 {
-    if (args.n_tiles == 0) return cudaSuccess;
-    const size_t smem = args.pop.N > 16 ? static_cast<size_t>(kMaxN) * kXThreads : 0;
-    exchange_plan_kernel<<<args.n_tiles, kXThreads, smem, stream>>>(args);
-    count_launch();
-    cudaError_t err = cudaGetLastError();
+    if (args.n_blocks == 0) return cudaSuccess;
+    size_t smem = 0;
+    cudaError_t err = perm_smem(args, reinterpret_cast<const void *>(exchange_plan_kernel), &smem);
     if (err != cudaSuccess) return err;
-    exchange_scan_kernel<<<args.pop.N + 1, 1024, 0, stream>>>(args);
+    exchange_plan_kernel<<<args.n_blocks, kXThreads, smem, stream>>>(args);
     count_launch();
     return cudaGetLastError();
 }
 
 cudaError_t launch_exchange_send(const ExchangeArgs &args, cudaStream_t stream)
 {
-    if (args.n_tiles == 0) return cudaSuccess;
-    const size_t smem = args.pop.N > 16 ? static_cast<size_t>(kMaxN) * kXThreads : 0;
-    exchange_send_kernel<<<args.n_tiles, kXThreads, smem, stream>>>(args);
+    if (args.n_blocks == 0) return cudaSuccess;
+    size_t smem = 0;
+    cudaError_t err = perm_smem(args, reinterpret_cast<const void *>(exchange_send_kernel), &smem);
+    if (err != cudaSuccess) return err;
+    exchange_send_kernel<<<args.n_blocks, kXThreads, smem, stream>>>(args);
     count_launch();
     return cudaGetLastError();
 }
 
 cudaError_t launch_exchange_receive(const ExchangeArgs &args, cudaStream_t stream)
 {
-    if (args.n_tiles == 0) return cudaSuccess;
-    exchange_receive_kernel<<<args.n_tiles, kXThreads, 0, stream>>>(args);
+    if (args.n_blocks == 0) return cudaSuccess;
+    exchange_receive_kernel<<<args.n_blocks, kXThreads, 0, stream>>>(args);
     count_launch();
     return cudaGetLastError();
 }

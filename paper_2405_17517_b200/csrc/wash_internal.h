@@ -65,17 +65,21 @@ struct ReduceArgs {
 };
 
 // One model per device (wash_exchange_*): the row is one model of a population of pop.N.
-constexpr int kExchangeTileGroups = 1024;   // a tile = one block = 1024 groups = 4096 coordinates
+constexpr int kExchangeTileGroups = 128;   // a warp tile: 32 lanes x 4 groups = 512 coordinates
+constexpr int kExchangeWarps = 8;          // warps per block of the exchange kernels
 struct ExchangeArgs {
     PopView pop;
     int self;                     // this worker's index in the population
-    uint32_t n_tiles;             // ceil(n_groups / kExchangeTileGroups)
+    uint32_t n_wtiles;            // ceil(n_groups / kExchangeTileGroups)
+    uint32_t tiles_per_warp;      // consecutive warp tiles a warp visits
+    uint32_t n_blocks;            // grid of all three kernels: n_blocks * kExchangeWarps * tiles_per_warp >= n_wtiles
     uint32_t key0, key1;
     uint32_t step_lo, step_hi8;
-    uint8_t *mask;                // [n_tiles * kExchangeTileGroups] low nibble: selected coordinates; high nibble: those this worker receives
-    uint32_t *tile_count;         // [N + 1][n_tiles]: column n = slots of worker n's buffer per tile (after the scan:
-                                  // slots before the tile); column N = selected coordinates
-    uint32_t *total;              // [N + 1] column totals
+    uint32_t *mask;               // [n_wtiles * 32] a word per lane = its four groups' bytes; low nibble of a byte:
+                                  // selected coordinates, high nibble: those this worker receives
+    uint32_t *warp_total;         // [n_blocks * kExchangeWarps][N + 1]: column n = slots of worker n's buffer the
+                                  // warp's range takes; column N = selected coordinates
+    uint32_t *block_total;        // [n_blocks][N + 1] the same per block
     void *row[2];                 // this worker's model: parameters, optimizer state (nullptr: absent)
     int dtype[2];
     void *const *staging[2];      // per stack: device array of N pointers, entry n = worker n's staging buffer
