@@ -530,7 +530,8 @@ def run_exchange(args) -> None:
         reps = 30
         ev = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(reps)]
         for i in range(3 + reps):
-            flush.zero_()
+            if not args.exchange_warm:
+                flush.zero_()
             e = ev[max(i - 3, 0)]
             e[0].record(stream)
             B.wash_exchange_plan(ctx, i, wl.p, p_layer, SEED, stream)
@@ -550,7 +551,8 @@ def run_exchange(args) -> None:
             "selected_per_step": sel, "values_received_per_step": recv,
             "link_bytes_in_per_step": recv * elem, "model_bytes": wl.P * elem,
             "mask_coordinates_per_s": wl.P / (med(0, 1) * 1e-6),
-            "note": "L2 flushed before every step; peers' buffers are on the same device",
+            "note": ("steps back to back (row and tables may stay in L2)" if args.exchange_warm else "L2 flushed before every step")
+                    + "; peers' buffers are on the same device",
         }), flush=True)
         B.wash_destroy(ctx)
         del keep, rows, row, flush
@@ -576,6 +578,7 @@ def main() -> None:
     ap.add_argument("--sweep-logP", default="", help="comma list; default 20,24,27")
     ap.add_argument("--sweep-p", default="", help="comma list; default 1e-4..1")
     ap.add_argument("--sweep-layout", default="", choices=["", "np", "pn"])
+    ap.add_argument("--exchange-warm", action="store_true", help="with --exchange: no L2 flush between steps")
     ap.add_argument("--exchange", action="store_true", help="time one worker of the one-model-per-device form (JSON line per workload)")
     args = ap.parse_args()
     args.workload_given = any(a == "--workload" or a.startswith("--workload=") for a in sys.argv[1:])

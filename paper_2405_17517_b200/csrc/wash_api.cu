@@ -101,7 +101,7 @@ struct wash_ctx {
     uint32_t *x_mask = nullptr;            // a byte per group, whole warp tiles
     uint32_t *x_warp_total = nullptr;      // [x_blocks * kExchangeWarps][N + 1]
     uint32_t *x_block_total = nullptr;     // [x_blocks][N + 1]
-    uint32_t x_wtiles = 0, x_blocks = 0, x_tiles_per_warp = 0;
+    uint32_t x_wtiles = 0, x_blocks = 0;
     void **x_staging[2][2] = {{nullptr, nullptr}, {nullptr, nullptr}};   // [parity][stack]: device array of N pointers
     int64_t x_capacity[2][2] = {{0, 0}, {0, 0}};
     void *x_own[2][2] = {{nullptr, nullptr}, {nullptr, nullptr}};        // staging buffers this library allocated
@@ -649,7 +649,6 @@ int exchange_args(wash_ctx *ctx, wash::ExchangeArgs *out)
     a.pop = view_of(ctx);
     a.self = ctx->x_self;
     a.n_wtiles = ctx->x_wtiles;
-    a.tiles_per_warp = ctx->x_tiles_per_warp;
     a.n_blocks = ctx->x_blocks;
     a.key0 = static_cast<uint32_t>(ctx->x_seed);
     a.key1 = static_cast<uint32_t>(ctx->x_seed >> 32);
@@ -699,11 +698,12 @@ int wash_exchange_bind(wash_ctx *ctx, int32_t self, int32_t stack, int32_t dtype
     if (!ctx->x_mask) {
         DeviceGuard guard(ctx->device);
         if (guard.err != cudaSuccess) return cuda_fail(guard.err, "cudaSetDevice");
-        // a warp visits tiles_per_warp consecutive warp tiles; the grid is at most four blocks per SM (what the plan kernel fits)
+        // the grid: four blocks per SM (what the plan kernel fits), fewer for short rows; its
+        // warps share the warp tiles evenly
         const uint32_t wtiles = (ctx->n_groups + wash::kExchangeTileGroups - 1) / wash::kExchangeTileGroups;
-        const uint32_t max_warps = static_cast<uint32_t>(ctx->shape.sm_count > 0 ? ctx->shape.sm_count : 148) * 4u * wash::kExchangeWarps;
-        const uint32_t per_warp = (wtiles + max_warps - 1) / max_warps;
-        const uint32_t blocks = (wtiles + per_warp * wash::kExchangeWarps - 1) / (per_warp * wash::kExchangeWarps);
+        const uint32_t max_blocks = static_cast<uint32_t>(ctx->shape.sm_count > 0 ? ctx->shape.sm_count : 148) * 4u;
+        const uint32_t want = (wtiles + wash::kExchangeWarps - 1) / wash::kExchangeWarps;
+        const uint32_t blocks = want < max_blocks ? want : max_blocks;
         const size_t columns = static_cast<size_t>(ctx->N) + 1;
         cudaError_t err;
         if ((err = cudaMalloc(&ctx->x_mask, sizeof(uint32_t) * 32u * static_cast<size_t>(wtiles))) != cudaSuccess ||
@@ -717,7 +717,6 @@ int wash_exchange_bind(wash_ctx *ctx, int32_t self, int32_t stack, int32_t dtype
             return fail(WASH_ERR_ALLOC, "device allocation of the exchange tables failed: %s", cudaGetErrorString(err));
         }
         ctx->x_wtiles = wtiles;
-        ctx->x_tiles_per_warp = per_warp;
         ctx->x_blocks = blocks;
     }
     ctx->x_self = self;

@@ -21,7 +21,7 @@
 //            pi_i(n) is this worker
 //   receive  the same replay for its own buffer only, from the high nibbles: no draw at all
 // The plan reads no model data; send and receive touch only selected coordinates.
-// All three kernels must be launched with the same grid (n_blocks) and tiles_per_warp.
+// All three kernels must be launched with the same grid (n_blocks).
 #include "wash_device.cuh"
 #include "wash_launch.cuh"
 #include "wash_shuffle_tma.cuh"     // draw_permutation_u8
@@ -137,13 +137,14 @@ __device__ __forceinline__ void routes_of(const ExchangeArgs &a, uint32_t elem, 
     *dest = d;
 }
 
-// first and one-past-last warp tile of this warp, and the cursor into the segment table for the first
+// first and one-past-last warp tile of this warp (the n_wtiles tiles are dealt out evenly,
+// in order, to the grid's warps), and the cursor into the segment table for the first
 __device__ __forceinline__ void warp_range(const ExchangeArgs &a, uint32_t *t0, uint32_t *t1, uint32_t *cursor)
 {
-    const uint32_t range = blockIdx.x * kExchangeWarps + (threadIdx.x >> 5);
-    const uint64_t lo = static_cast<uint64_t>(range) * a.tiles_per_warp;
-    *t0 = static_cast<uint32_t>(min(lo, static_cast<uint64_t>(a.n_wtiles)));
-    *t1 = static_cast<uint32_t>(min(lo + a.tiles_per_warp, static_cast<uint64_t>(a.n_wtiles)));
+    const uint64_t range = blockIdx.x * kExchangeWarps + (threadIdx.x >> 5);
+    const uint64_t ranges = static_cast<uint64_t>(a.n_blocks) * kExchangeWarps;
+    *t0 = static_cast<uint32_t>(range * a.n_wtiles / ranges);
+    *t1 = static_cast<uint32_t>((range + 1) * a.n_wtiles / ranges);
     const uint32_t g = *t0 * kExchangeTileGroups;
     *cursor = (*t0 < *t1 && g < a.pop.n_groups) ? __ldg(a.pop.tile_first + (g >> kTileShift)) : 0u;
 }

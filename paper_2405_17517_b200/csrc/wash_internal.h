@@ -71,8 +71,7 @@ struct ExchangeArgs {
     PopView pop;
     int self;                     // this worker's index in the population
     uint32_t n_wtiles;            // ceil(n_groups / kExchangeTileGroups)
-    uint32_t tiles_per_warp;      // consecutive warp tiles a warp visits
-    uint32_t n_blocks;            // grid of all three kernels: n_blocks * kExchangeWarps * tiles_per_warp >= n_wtiles
+    uint32_t n_blocks;            // grid of all three kernels; its warps share the warp tiles evenly, in order
     uint32_t key0, key1;
     uint32_t step_lo, step_hi8;
     uint32_t *mask;               // [n_wtiles * 32] a word per lane = its four groups' bytes; low nibble of a byte:
