@@ -461,6 +461,8 @@ def run_sweep(args) -> None:
                 gen = torch.Generator(device="cuda").manual_seed(N * 100 + logP)
                 stack = torch.randn(N * pop.padded_P, generator=gen, device="cuda", dtype=torch.float32) * 0.05
                 pop.bind(B.WASH_STACK_PARAMS, stack)
+                if args.threads or args.blocks_per_sm:
+                    B.wash_set_launch(pop.ctx, args.threads, args.blocks_per_sm)
                 stats = torch.zeros(2, dtype=torch.int64, device="cuda")
                 for p in pick(args.sweep_p, [1e-4, 1e-3, 1e-2, 1e-1, 1.0], float):
                     for mode in args.sweep_modes.split(","):

@@ -123,6 +123,8 @@ int wash_set_mode(wash_ctx *ctx, int32_t mode);
  * 0 = each kernel's default) and grid style: blocks_per_sm == 0 each kernel's default,
  * > 0 a persistent grid of SM count x min(blocks_per_sm, resident blocks per SM) blocks
  * that stride over the groups, < 0 one group of 4 coordinates per thread.  For
+ * WASH_MODE_STREAM blocks_per_sm = 1 or 2 fixes the number of groups a thread takes
+ * (default: 2 when a group of all models is at most 64 bytes, else 1).  For
  * WASH_MODE_STREAM_STAGED `threads` is the tile size in groups (32, 64, 128 or 256)
  * and blocks_per_sm the number of consumer teams per block. */
 int wash_set_launch(wash_ctx *ctx, int32_t threads, int32_t blocks_per_sm);

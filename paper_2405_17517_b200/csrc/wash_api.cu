@@ -698,10 +698,10 @@ int wash_exchange_bind(wash_ctx *ctx, int32_t self, int32_t stack, int32_t dtype
     if (!ctx->x_mask) {
         DeviceGuard guard(ctx->device);
         if (guard.err != cudaSuccess) return cuda_fail(guard.err, "cudaSetDevice");
-        // the grid: four blocks per SM (what the plan kernel fits), fewer for short rows; its
+        // the grid: kExchangeBlocksPerSm blocks per SM, fewer for short rows; its
         // warps share the warp tiles evenly
         const uint32_t wtiles = (ctx->n_groups + wash::kExchangeTileGroups - 1) / wash::kExchangeTileGroups;
-        const uint32_t max_blocks = static_cast<uint32_t>(ctx->shape.sm_count > 0 ? ctx->shape.sm_count : 148) * 4u;
+        const uint32_t max_blocks = static_cast<uint32_t>(ctx->shape.sm_count > 0 ? ctx->shape.sm_count : 148) * static_cast<uint32_t>(wash::kExchangeBlocksPerSm);
         const uint32_t want = (wtiles + wash::kExchangeWarps - 1) / wash::kExchangeWarps;
         const uint32_t blocks = want < max_blocks ? want : max_blocks;
         const size_t columns = static_cast<size_t>(ctx->N) + 1;

@@ -149,7 +149,7 @@ __device__ __forceinline__ void warp_range(const ExchangeArgs &a, uint32_t *t0, 
     *cursor = (*t0 < *t1 && g < a.pop.n_groups) ? __ldg(a.pop.tile_first + (g >> kTileShift)) : 0u;
 }
 
-__global__ void __launch_bounds__(kXThreads, 4) exchange_plan_kernel(const __grid_constant__ ExchangeArgs a)
+__global__ void __launch_bounds__(kXThreads, kExchangeBlocksPerSm) exchange_plan_kernel(const __grid_constant__ ExchangeArgs a)
 {
     extern __shared__ uint8_t s_perm_all[];   // column per thread (kMaxN * kXThreads bytes) when N > 16, else nothing
     __shared__ uint32_t s_count[kExchangeWarps][kMaxN + 1];

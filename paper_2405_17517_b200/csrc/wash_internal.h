@@ -67,6 +67,10 @@ struct ReduceArgs {
 // One model per device (wash_exchange_*): the row is one model of a population of pop.N.
 constexpr int kExchangeTileGroups = 128;   // a warp tile: 32 lanes x 4 groups = 512 coordinates
 constexpr int kExchangeWarps = 8;          // warps per block of the exchange kernels
+#ifndef WASH_EXCHANGE_BLOCKS_PER_SM
+#define WASH_EXCHANGE_BLOCKS_PER_SM 4
+#endif
+constexpr int kExchangeBlocksPerSm = WASH_EXCHANGE_BLOCKS_PER_SM;   // grid of the exchange kernels = this many blocks per SM (what the plan kernel fits)
 struct ExchangeArgs {
     PopView pop;
     int self;                     // this worker's index in the population
