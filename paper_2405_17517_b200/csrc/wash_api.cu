@@ -249,6 +249,7 @@ int shuffle_impl(wash_ctx *ctx, int which, uint64_t step, double p, const double
         const double kernel_ns = bytes / 6000.0 + 2000.0;
         const double reporting_blocks = std::fmin(ctx->expected_selected, static_cast<double>(ctx->n_groups) / 64.0);
         args.stat_slots = (2.0 * reporting_blocks / kernel_ns > 0.35) ? ctx->stat_slots_dev : nullptr;
+        if (ctx->mode == WASH_MODE_SPARSE) args.stat_slots = nullptr;   // one wave of large blocks: a few hundred atomics at most
     }
     args.status = ctx->status_dev;
     bool supported = false;

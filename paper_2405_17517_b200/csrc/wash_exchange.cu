@@ -24,95 +24,15 @@
 // All three kernels must be launched with the same grid (n_blocks).
 #include "wash_device.cuh"
 #include "wash_launch.cuh"
+#include "wash_warp_tiles.cuh"
 #include "wash_shuffle_tma.cuh"     // draw_permutation_u8
 #include "wash_shuffle_async.cuh"   // draw_permutation_packed
 
 namespace wash {
 
 constexpr int kXThreads = 32 * kExchangeWarps;
-constexpr uint32_t kFull = 0xFFFFFFFFu;
+static_assert(kExchangeTileGroups == kWarpTileGroups, "the exchange works on warp tiles");
 constexpr uint32_t kNoDestination = 0xFFu;
-
-// What a lane knows about its four consecutive groups g0 .. g0+3.
-struct LaneGroups {
-    bool one_tensor;   // all four lie in one tensor (the usual case): described by the fields below
-    uint32_t cgroup0, tensor;
-    uint64_t thr;
-    long long left;    // coordinates of the tensor from the first group on
-};
-
-__device__ __forceinline__ LaneGroups describe_groups(const ExchangeArgs &a, uint32_t g0, uint32_t &cursor)
-{
-    LaneGroups lg{true, 0, 0, 0, 0};
-    if (g0 >= a.pop.n_groups) return lg;   // thr == 0: nothing to draw
-    const GroupInfo gi = find_group_forward(a.pop.seg, a.pop.n_seg, cursor, g0, a.status);
-    const SegEntry &seg = a.pop.seg[cursor];
-    lg.one_tensor = g0 + 4 <= seg.group_end;
-    lg.cgroup0 = gi.cgroup;
-    lg.tensor = gi.tensor_id;
-    lg.thr = gi.thr;
-    lg.left = static_cast<long long>(seg.numel) - 4ll * (gi.cgroup - seg.cgroup_begin);
-    return lg;
-}
-
-// group q of the lane
-__device__ __forceinline__ GroupInfo lane_group(const ExchangeArgs &a, const LaneGroups &lg, uint32_t g0, int q)
-{
-    if (lg.one_tensor) {
-        const long long l = lg.left - 4 * q;
-        return GroupInfo{lg.tensor, lg.cgroup0 + q, l >= 4 ? 4 : (l > 0 ? static_cast<int>(l) : 0), lg.thr};
-    }
-    if (g0 + q >= a.pop.n_groups) return GroupInfo{0, 0, 0, 0};
-    return find_group(a.pop, g0 + q, a.status);
-}
-
-// the mask of one group: bit c set iff coordinate c is selected
-__device__ __forceinline__ uint32_t draw_mask(const GroupInfo &gi, const ExchangeArgs &a)
-{
-    if (gi.thr == 0 || gi.valid == 0) return 0;
-    const Philox4 w = philox4x32_10(gi.cgroup, gi.tensor_id, a.step_lo, a.step_hi8, a.key0, a.key1);
-    const uint32_t thr_lo = static_cast<uint32_t>(gi.thr);
-    const bool always = (gi.thr >> 32) != 0;
-    uint32_t m = 0;
-    m |= (w.x < thr_lo || always) ? 1u : 0u;
-    m |= (w.y < thr_lo || always) ? 2u : 0u;
-    m |= (w.z < thr_lo || always) ? 4u : 0u;
-    m |= (w.w < thr_lo || always) ? 8u : 0u;
-    return m & ((1u << gi.valid) - 1u);
-}
-
-__device__ __forceinline__ uint32_t warp_exclusive_scan(uint32_t mine, uint32_t *total)
-{
-    const uint32_t lane = threadIdx.x & 31u;
-    uint32_t upto = mine;
-#pragma unroll
-    for (int d = 1; d < 32; d <<= 1) {
-        const uint32_t v = __shfl_up_sync(kFull, upto, d);
-        if (lane >= static_cast<uint32_t>(d)) upto += v;
-    }
-    *total = __shfl_sync(kFull, upto, 31);
-    return upto - mine;
-}
-
-// The selected coordinates of a warp's range are few and scattered: serving each where it is
-// found would leave 31 lanes idle.  Instead the warp queues them, in coordinate order, as
-// row elements in a ring in shared memory and serves them 32 at a time, one per lane.
-constexpr uint32_t kXRing = 1024;   // entries; a warp tile adds at most 512, a round removes 32
-
-// appends the lane's selected coordinates of warp tile t (sel4: a nibble per byte, one byte per group)
-__device__ __forceinline__ uint32_t ring_append(uint32_t *ring, uint32_t tail, uint32_t sel4, uint32_t t)
-{
-    const uint32_t lane = threadIdx.x & 31u;
-    uint32_t total = 0;
-    uint32_t pos = tail + warp_exclusive_scan(__popc(sel4), &total);
-    const uint32_t elem0 = 4u * (t * kExchangeTileGroups + 4u * lane);   // rows are shorter than 2^32 elements
-    for (uint32_t left = sel4; left; left &= left - 1u, ++pos) {
-        const uint32_t bit = static_cast<uint32_t>(__ffs(left) - 1);   // byte q = bit / 8, coordinate c = bit % 8
-        ring[pos % kXRing] = elem0 + 4u * (bit >> 3) + (bit & 7u);
-    }
-    __syncwarp();
-    return tail + total;
-}
 
 // pi of the coordinate stored at row element `elem`, as {need: bit n set iff pi(n) != n,
 // dest: the n != self with pi(n) == self, if any}
@@ -161,11 +81,12 @@ __global__ void __launch_bounds__(kXThreads, kExchangeBlocksPerSm) exchange_plan
     uint32_t t0, t1, cursor;
     warp_range(a, &t0, &t1, &cursor);
     uint32_t head = 0, tail = 0;   // ring positions served / queued so far
+    const uint32_t range_elem = 4u * kExchangeTileGroups * t0;   // first row element of the warp's range (rows are shorter than 2^32)
     // one round: lane j takes entry head + j; counts every worker's slots and marks the
     // coordinates this worker receives in the (already written) mask words
     auto serve = [&](uint32_t count) {
         if (lane < count) {
-            const uint32_t elem = s_ring[warp][(head + lane) % kXRing];
+            const uint32_t elem = range_elem + s_ring[warp][(head + lane) % kXRing];
             unsigned long long need;
             uint32_t dest;
             routes_of(a, elem, s_perm_all + threadIdx.x, &need, &dest);
@@ -194,7 +115,7 @@ __global__ void __launch_bounds__(kXThreads, kExchangeBlocksPerSm) exchange_plan
         }
         a.mask[static_cast<size_t>(t) * 32u + lane] = sel4;
         if (__any_sync(kFull, sel4 != 0)) {
-            tail = ring_append(s_ring[warp], tail, sel4, t);   // orders the mask stores before the rounds' atomics, too
+            tail = ring_append(s_ring[warp], tail, sel4, t - t0);   // orders the mask stores before the rounds' atomics, too
             while (tail - head >= 32u) serve(32u);
         }
     }
@@ -251,13 +172,14 @@ __global__ void __launch_bounds__(kXThreads) exchange_send_kernel(const __grid_c
     uint32_t t0, t1, cursor;
     warp_range(a, &t0, &t1, &cursor);
     uint32_t head = 0, tail = 0;
+    const uint32_t range_elem = 4u * kExchangeTileGroups * t0;
     // one round: lane j takes entry head + j (coordinate order along the lanes); the warp votes
     // worker by worker to number the slots, then every lane with a destination copies its value
     auto serve = [&](uint32_t count) {
         unsigned long long need = 0;
         uint32_t dest = kNoDestination, elem = 0;
         if (lane < count) {
-            elem = s_ring[warp][(head + lane) % kXRing];
+            elem = range_elem + s_ring[warp][(head + lane) % kXRing];
             routes_of(a, elem, s_perm_all + threadIdx.x, &need, &dest);
         }
         uint32_t slot = 0;
@@ -284,7 +206,7 @@ __global__ void __launch_bounds__(kXThreads) exchange_send_kernel(const __grid_c
     for (uint32_t t = t0; t < t1; ++t) {
         const uint32_t sel4 = a.mask[static_cast<size_t>(t) * 32u + lane] & 0x0F0F0F0Fu;
         if (!__any_sync(kFull, sel4 != 0)) continue;
-        tail = ring_append(s_ring[warp], tail, sel4, t);
+        tail = ring_append(s_ring[warp], tail, sel4, t - t0);
         while (tail - head >= 32u) serve(32u);
     }
     if (tail != head) serve(tail - head);

@@ -65,7 +65,7 @@ struct ReduceArgs {
 };
 
 // One model per device (wash_exchange_*): the row is one model of a population of pop.N.
-constexpr int kExchangeTileGroups = 128;   // a warp tile: 32 lanes x 4 groups = 512 coordinates
+constexpr int kExchangeTileGroups = 128;   // a warp tile (wash_warp_tiles.cuh): 32 lanes x 4 groups = 512 coordinates
 constexpr int kExchangeWarps = 8;          // warps per block of the exchange kernels
 #ifndef WASH_EXCHANGE_BLOCKS_PER_SM
 #define WASH_EXCHANGE_BLOCKS_PER_SM 4

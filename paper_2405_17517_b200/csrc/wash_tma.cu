@@ -1,6 +1,7 @@
-// Translation unit of the shared-memory-staged streaming shuffles (bulk copies; cp.async).
+// Translation unit of the shared-memory-staged streaming shuffles (bulk copies; cp.async) and of the sparse shuffle.
 #include "wash_shuffle_tma.cuh"
 #include "wash_shuffle_async.cuh"
+#include "wash_shuffle_sparse.cuh"
 
 namespace wash {
 
@@ -16,11 +17,11 @@ cudaError_t launch_shuffle_async_staged(const ShuffleArgs &args, int a_dtype, in
     return launch_shuffle_async<true>(args, a_dtype, b_dtype, shape, stream, supported);
 }
 
-// sparse mode: the same kernel without the up-front copies
+// sparse mode: mask first, only selected coordinates touched (wash_shuffle_sparse.cuh)
 cudaError_t launch_shuffle_sparse(const ShuffleArgs &args, int a_dtype, int b_dtype, const LaunchShape &shape,
                                   cudaStream_t stream, bool *supported)
 {
-    return launch_shuffle_async<false>(args, a_dtype, b_dtype, shape, stream, supported);
+    return launch_shuffle_sparse_tiles(args, a_dtype, b_dtype, shape, stream, supported);
 }
 
 }  // namespace wash
