@@ -394,7 +394,7 @@ def run_ours(args, rank: int, world: int, local_rank: int) -> None:
 # DRAM bytes per shuffle launch from the ncu capture summarised under profiles/ (None
 # until a capture of the current kernel exists).
 TRAFFIC = {
-    # shuffle_async_kernel<F32, F32, [N][P], FETCH, 1>: 448.9 MB read + 6.0 MB written per launch
+    # shuffle_async_kernel<F32, F32, [N][P], 1>: 448.9 MB read + 6.0 MB written per launch
     "cfg2_resnet18_n5": {"dram_bytes": 448.9e6 + 6.0e6,
                          "source": "profiles/shuffle_async_kernel_cfg2_resnet18_n5.md"},
 }

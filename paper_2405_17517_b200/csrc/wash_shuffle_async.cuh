@@ -104,9 +104,9 @@ __device__ __forceinline__ uint64_t draw_permutation_packed(int n_models, uint32
 // selected coordinates are listed in shared memory and dealt out to the lanes 32 at a time:
 // with a few selected coordinates per warp (p around 0.01-0.1) one round serves them all,
 // instead of one divergent pass per coordinate slot.  Called by all threads of the block.
-template <class TA, class TB, int LAYOUT, bool FETCH>
+template <class TA, class TB, int LAYOUT>
 __device__ __forceinline__ void serve_tile(const ShuffleArgs &a, const unsigned char *image_a, const unsigned char *image_b,
-                                           uint8_t *s_list, uint8_t *s_perm, uint32_t *s_col, uint64_t g_block,
+                                           uint8_t *s_list, uint8_t *s_perm, uint64_t g_block,
                                            uint32_t sel, const GroupInfo &gi, uint32_t &selected, uint32_t &moved)
 {
     constexpr bool kHasB = TB::kCode != kDtypeNone;
@@ -143,67 +143,44 @@ __device__ __forceinline__ void serve_tile(const ShuffleArgs &a, const unsigned 
         auto source_of = [&](int n) -> int {
             return n_models <= 16 ? static_cast<int>((perm >> (4 * n)) & 15ull) : static_cast<int>(s_perm[n * T_]);
         };
-        if constexpr (FETCH) {
-            // model n's value of this coordinate sits at out0 + n*out_step in the stack and at
-            // element img0 + n*img_step of the image: no multiplication left inside the loop
-            const long long out_step = LAYOUT == kLayoutNP ? a.pop.padded_P : 1;
-            const long long out0 = LAYOUT == kLayoutNP ? e : e * n_models;
-            const uint32_t img_step = LAYOUT == kLayoutNP ? T_ * 4u : 1u;
-            const uint32_t img0 = LAYOUT == kLayoutNP ? t_owner * 4u + c : (4u * t_owner + c) * n_models;
-            long long out = out0;
-            for (int n = 0; n < n_models; ++n, out += out_step) {
-                const uint32_t src = static_cast<uint32_t>(source_of(n));
-                if (src == static_cast<uint32_t>(n)) continue;
-                const uint32_t from = img0 + src * img_step;
-                TA::store_elem(a.a, out, TA::kBytes == 4 ? reinterpret_cast<const uint32_t *>(image_a)[from]
-                                                         : reinterpret_cast<const uint16_t *>(image_a)[from]);
-                if constexpr (kHasB)
-                    TB::store_elem(a.b, out, TB::kBytes == 4 ? reinterpret_cast<const uint32_t *>(image_b)[from]
-                                                             : reinterpret_cast<const uint16_t *>(image_b)[from]);
-                ++moved;
-            }
-        } else {
-            // all N old values first (the exchange is in place), then the moved ones back
-            for (int n = 0; n < n_models; ++n) s_col[n * T_] = TA::load_elem(a.a, elem_index<LAYOUT>(a.pop, n, e));
-            for (int n = 0; n < n_models; ++n) {
-                const int src = source_of(n);
-                if (src == n) continue;
-                TA::store_elem(a.a, elem_index<LAYOUT>(a.pop, n, e), s_col[src * T_]);
-                ++moved;
-            }
-            if constexpr (kHasB) {
-                for (int n = 0; n < n_models; ++n) s_col[n * T_] = TB::load_elem(a.b, elem_index<LAYOUT>(a.pop, n, e));
-                for (int n = 0; n < n_models; ++n) {
-                    const int src = source_of(n);
-                    if (src != n) TB::store_elem(a.b, elem_index<LAYOUT>(a.pop, n, e), s_col[src * T_]);
-                }
-            }
+        // model n's value of this coordinate sits at out0 + n*out_step in the stack and at
+        // element img0 + n*img_step of the image: no multiplication left inside the loop
+        const long long out_step = LAYOUT == kLayoutNP ? a.pop.padded_P : 1;
+        const long long out0 = LAYOUT == kLayoutNP ? e : e * n_models;
+        const uint32_t img_step = LAYOUT == kLayoutNP ? T_ * 4u : 1u;
+        const uint32_t img0 = LAYOUT == kLayoutNP ? t_owner * 4u + c : (4u * t_owner + c) * n_models;
+        long long out = out0;
+        for (int n = 0; n < n_models; ++n, out += out_step) {
+            const uint32_t src = static_cast<uint32_t>(source_of(n));
+            if (src == static_cast<uint32_t>(n)) continue;
+            const uint32_t from = img0 + src * img_step;
+            TA::store_elem(a.a, out, TA::kBytes == 4 ? reinterpret_cast<const uint32_t *>(image_a)[from]
+                                                     : reinterpret_cast<const uint16_t *>(image_a)[from]);
+            if constexpr (kHasB)
+                TB::store_elem(a.b, out, TB::kBytes == 4 ? reinterpret_cast<const uint32_t *>(image_b)[from]
+                                                         : reinterpret_cast<const uint16_t *>(image_b)[from]);
+            ++moved;
         }
         ++selected;
     }
     __syncwarp();   // the warp's list is rewritten by the next tile
 }
 
-// FETCH = true: the streaming kernel described above.  FETCH = false: the sparse mode --
-// nothing is copied up front; the mask is drawn first and a selected coordinate's N values
-// are loaded from global memory into a private shared-memory column when it is served.
 // G = tiles per block (one group per thread and tile).  Small populations move few bytes per
 // group (N * 16 for fp32), so a thread takes G = 2 groups, T apart, to keep more bytes in
 // flight per SM; the two Philox draws overlap as well.
-template <class TA, class TB, int LAYOUT, bool FETCH, int G>
+template <class TA, class TB, int LAYOUT, int G>
 __global__ void __launch_bounds__(256, 5) shuffle_async_kernel(const __grid_constant__ ShuffleArgs a)
 {
     extern __shared__ __align__(128) unsigned char smem_raw[];
     constexpr bool kHasB = TB::kCode != kDtypeNone;
-    static_assert(FETCH || G == 1, "the sparse mode takes one tile per block");
     const int n_models = a.pop.N;
     const uint32_t T_ = blockDim.x;
-    // FETCH: G pairs of images of the two stacks.  !FETCH: one column of N words per thread.
-    const size_t a_bytes = static_cast<size_t>(n_models) * T_ * (FETCH ? TA::kBytes * 4 : 4);
-    const size_t b_bytes = FETCH && kHasB ? static_cast<size_t>(n_models) * T_ * TB::kBytes * 4 : 0;
+    // G pairs of images of the two stacks, then the warps' lists, then the permutation columns
+    const size_t a_bytes = static_cast<size_t>(n_models) * T_ * TA::kBytes * 4;
+    const size_t b_bytes = kHasB ? static_cast<size_t>(n_models) * T_ * TB::kBytes * 4 : 0;
     uint8_t *s_list = smem_raw + G * (a_bytes + b_bytes);   // 128 bytes per warp
     uint8_t *s_perm = s_list + 4 * T_ + threadIdx.x;        // column [n][T], used when N > 16
-    uint32_t *s_col = reinterpret_cast<uint32_t *>(smem_raw) + threadIdx.x;   // !FETCH: column [n][T]
 
     const uint64_t g_first = a.group_lo + static_cast<uint64_t>(blockIdx.x) * (T_ * G);
     uint32_t in_tile[G];   // groups of tile i that exist
@@ -211,12 +188,10 @@ __global__ void __launch_bounds__(256, 5) shuffle_async_kernel(const __grid_cons
     for (int i = 0; i < G; ++i) {
         const uint64_t g_block = g_first + static_cast<uint64_t>(i) * T_;
         in_tile[i] = g_block < a.group_hi ? static_cast<uint32_t>(min(static_cast<uint64_t>(T_), a.group_hi - g_block)) : 0u;
-        if constexpr (FETCH) {
-            if (in_tile[i] == 0) continue;
-            unsigned char *image_a = smem_raw + i * (a_bytes + b_bytes);
-            async_fetch<TA, LAYOUT>(smem_addr(image_a), a.a, a.pop, g_block, in_tile[i], n_models);
-            if constexpr (kHasB) async_fetch<TB, LAYOUT>(smem_addr(image_a + a_bytes), a.b, a.pop, g_block, in_tile[i], n_models);
-        }
+        if (in_tile[i] == 0) continue;
+        unsigned char *image_a = smem_raw + i * (a_bytes + b_bytes);
+        async_fetch<TA, LAYOUT>(smem_addr(image_a), a.a, a.pop, g_block, in_tile[i], n_models);
+        if constexpr (kHasB) async_fetch<TB, LAYOUT>(smem_addr(image_a + a_bytes), a.b, a.pop, g_block, in_tile[i], n_models);
     }
 
     uint32_t selected = 0, moved = 0;
@@ -247,37 +222,34 @@ __global__ void __launch_bounds__(256, 5) shuffle_async_kernel(const __grid_cons
     // must see each other's copies; in the [P][N] image a group's values were copied by
     // threads of other warps, so a block with a selected coordinate needs a block-wide
     // barrier instead.
-    if constexpr (FETCH) {
-        cp_async_wait_all();
-        constexpr bool kSharedCopies = LAYOUT == kLayoutPN || TA::kBytes == 2 || (kHasB && TB::kBytes == 2);   // a group's bytes were copied by other threads
-        if (kSharedCopies) __syncthreads();
-        else __syncwarp();
-    }
+    cp_async_wait_all();
+    constexpr bool kSharedCopies = LAYOUT == kLayoutPN || TA::kBytes == 2 || (kHasB && TB::kBytes == 2);   // a group's bytes were copied by other threads
+    if (kSharedCopies) __syncthreads();
+    else __syncwarp();
 #pragma unroll
     for (int i = 0; i < G; ++i) {
-        const unsigned char *image_a = smem_raw + (FETCH ? i * (a_bytes + b_bytes) : 0);
-        serve_tile<TA, TB, LAYOUT, FETCH>(a, image_a, image_a + a_bytes, s_list, s_perm, s_col,
-                                          g_first + static_cast<uint64_t>(i) * T_, sel[i], gi[i], selected, moved);
+        const unsigned char *image_a = smem_raw + i * (a_bytes + b_bytes);
+        serve_tile<TA, TB, LAYOUT>(a, image_a, image_a + a_bytes, s_list, s_perm,
+                                   g_first + static_cast<uint64_t>(i) * T_, sel[i], gi[i], selected, moved);
     }
     publish_block_stats(a.stats, a.stat_slots, selected, moved);
 }
 
-template <class TA, class TB, bool FETCH, int G>
+template <class TA, class TB, int G>
 cudaError_t launch_shuffle_async_tiles(const ShuffleArgs &args, const LaunchShape &shape, cudaStream_t stream)
 {
     constexpr bool kHasB = TB::kCode != kDtypeNone;
-    // G images of both stacks (or one column of words), 4 bytes of the warp's list, a byte
-    // per model for the permutation
-    const size_t image = static_cast<size_t>(args.pop.N) * (FETCH ? TA::kBytes * 4 + (kHasB ? TB::kBytes * 4 : 0) : 4);
+    // G images of both stacks, 4 bytes of the warp's list, a byte per model for the permutation
+    const size_t image = static_cast<size_t>(args.pop.N) * (TA::kBytes * 4 + (kHasB ? TB::kBytes * 4 : 0));
     const size_t per_thread = image * G + args.pop.N + 4;
     // block size: as many threads as keep a block's image near 44 KiB, so that five blocks
     // (about 200 KiB in flight) share an SM
-    int threads = shape.threads > 0 ? shape.threads : (FETCH ? 64 : 128);   // measured: 64 beats 128 and 256 when streaming (a block holds its shared memory until its slowest thread is done)
+    int threads = shape.threads > 0 ? shape.threads : 64;   // measured: 64 beats 128 and 256 (a block holds its shared memory until its slowest thread is done)
     if (threads > 256) threads = 256;
     if (shape.threads <= 0)
         while (threads > 32 && per_thread * threads > 44 * 1024) threads >>= 1;
     const size_t smem = (per_thread * threads + 15) & ~static_cast<size_t>(15);
-    auto kernel = args.pop.layout == kLayoutNP ? shuffle_async_kernel<TA, TB, kLayoutNP, FETCH, G> : shuffle_async_kernel<TA, TB, kLayoutPN, FETCH, G>;
+    auto kernel = args.pop.layout == kLayoutNP ? shuffle_async_kernel<TA, TB, kLayoutNP, G> : shuffle_async_kernel<TA, TB, kLayoutPN, G>;
     KernelFit fit;
     cudaError_t err = kernel_fit(reinterpret_cast<const void *>(kernel), threads, smem, &fit);
     if (err != cudaSuccess) return err;
@@ -291,34 +263,31 @@ cudaError_t launch_shuffle_async_tiles(const ShuffleArgs &args, const LaunchShap
     return cudaGetLastError();
 }
 
-template <class TA, class TB, bool FETCH>
+template <class TA, class TB>
 cudaError_t launch_shuffle_async_typed(const ShuffleArgs &args, const LaunchShape &shape, cudaStream_t stream)
 {
-    if constexpr (FETCH) {
-        // bytes a thread has in flight for one group: up to 64 (N = 2 .. 4 in fp32, one stack) it
-        // takes two groups (measured on 2^27 coordinates, p = 1e-3: N = 4 0.84 -> 0.95 of the copy
-        // bandwidth, N = 2 0.48 -> 0.56; four groups were slower than two for every N).
-        // blocks_per_sm of wash_set_launch, when 1 or 2, overrides.
-        constexpr bool kHasB = TB::kCode != kDtypeNone;
-        const size_t per_group = static_cast<size_t>(args.pop.N) * (TA::kBytes * 4 + (kHasB ? TB::kBytes * 4 : 0));
-        int tiles = per_group <= 64 ? 2 : 1;
-        if (shape.blocks_per_sm == 1 || shape.blocks_per_sm == 2) tiles = shape.blocks_per_sm;
-        if (tiles == 2) return launch_shuffle_async_tiles<TA, TB, FETCH, 2>(args, shape, stream);
-    }
-    return launch_shuffle_async_tiles<TA, TB, FETCH, 1>(args, shape, stream);
+    // bytes a thread has in flight for one group: up to 64 (N = 2 .. 4 in fp32, one stack) it
+    // takes two groups (measured on 2^27 coordinates, p = 1e-3: N = 4 0.84 -> 0.95 of the copy
+    // bandwidth, N = 2 0.48 -> 0.56; four groups were slower than two for every N).
+    // blocks_per_sm of wash_set_launch, when 1 or 2, overrides.
+    constexpr bool kHasB = TB::kCode != kDtypeNone;
+    const size_t per_group = static_cast<size_t>(args.pop.N) * (TA::kBytes * 4 + (kHasB ? TB::kBytes * 4 : 0));
+    int tiles = per_group <= 64 ? 2 : 1;
+    if (shape.blocks_per_sm == 1 || shape.blocks_per_sm == 2) tiles = shape.blocks_per_sm;
+    if (tiles == 2) return launch_shuffle_async_tiles<TA, TB, 2>(args, shape, stream);
+    return launch_shuffle_async_tiles<TA, TB, 1>(args, shape, stream);
 }
 
-template <bool FETCH>
-cudaError_t launch_shuffle_async(const ShuffleArgs &args, int a_dtype, int b_dtype, const LaunchShape &shape,
-                                 cudaStream_t stream, bool *supported)
+inline cudaError_t launch_shuffle_async(const ShuffleArgs &args, int a_dtype, int b_dtype, const LaunchShape &shape,
+                                        cudaStream_t stream, bool *supported)
 {
     *supported = true;
-    if (a_dtype == kDtypeF32 && b_dtype == kDtypeNone) return launch_shuffle_async_typed<F32, NoStack, FETCH>(args, shape, stream);
-    if (a_dtype == kDtypeBF16 && b_dtype == kDtypeNone) return launch_shuffle_async_typed<BF16, NoStack, FETCH>(args, shape, stream);
-    if (a_dtype == kDtypeF32 && b_dtype == kDtypeF32) return launch_shuffle_async_typed<F32, F32, FETCH>(args, shape, stream);
-    if (a_dtype == kDtypeBF16 && b_dtype == kDtypeF32) return launch_shuffle_async_typed<BF16, F32, FETCH>(args, shape, stream);
-    if (a_dtype == kDtypeBF16 && b_dtype == kDtypeBF16) return launch_shuffle_async_typed<BF16, BF16, FETCH>(args, shape, stream);
-    if (a_dtype == kDtypeF32 && b_dtype == kDtypeBF16) return launch_shuffle_async_typed<F32, BF16, FETCH>(args, shape, stream);
+    if (a_dtype == kDtypeF32 && b_dtype == kDtypeNone) return launch_shuffle_async_typed<F32, NoStack>(args, shape, stream);
+    if (a_dtype == kDtypeBF16 && b_dtype == kDtypeNone) return launch_shuffle_async_typed<BF16, NoStack>(args, shape, stream);
+    if (a_dtype == kDtypeF32 && b_dtype == kDtypeF32) return launch_shuffle_async_typed<F32, F32>(args, shape, stream);
+    if (a_dtype == kDtypeBF16 && b_dtype == kDtypeF32) return launch_shuffle_async_typed<BF16, F32>(args, shape, stream);
+    if (a_dtype == kDtypeBF16 && b_dtype == kDtypeBF16) return launch_shuffle_async_typed<BF16, BF16>(args, shape, stream);
+    if (a_dtype == kDtypeF32 && b_dtype == kDtypeBF16) return launch_shuffle_async_typed<F32, BF16>(args, shape, stream);
     *supported = false;
     return cudaSuccess;
 }

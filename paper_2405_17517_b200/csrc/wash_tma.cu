@@ -14,7 +14,7 @@ cudaError_t launch_shuffle_staged(const ShuffleArgs &args, int a_dtype, int b_dt
 cudaError_t launch_shuffle_async_staged(const ShuffleArgs &args, int a_dtype, int b_dtype, const LaunchShape &shape,
                                         cudaStream_t stream, bool *supported)
 {
-    return launch_shuffle_async<true>(args, a_dtype, b_dtype, shape, stream, supported);
+    return launch_shuffle_async(args, a_dtype, b_dtype, shape, stream, supported);
 }
 
 // sparse mode: mask first, only selected coordinates touched (wash_shuffle_sparse.cuh)
