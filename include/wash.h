@@ -61,9 +61,12 @@ enum wash_mode {
                              per-thread asynchronous copies (cp.async).  Default.            */
     WASH_MODE_SPARSE = 1, /* draws the mask first; touches only selected coordinates          */
     WASH_MODE_STREAM_STAGED = 2,   /* as STREAM, staged by bulk asynchronous copies (TMA)     */
-    WASH_MODE_STREAM_REGISTERS = 3 /* as STREAM, the loads held in registers (kernels unrolled
+    WASH_MODE_STREAM_REGISTERS = 3,/* as STREAM, the loads held in registers (kernels unrolled
                                       for N in {2,3,4,5,6,8,10,12,16,20,24,32}; other N run
                                       the default kernel)                                     */
+    WASH_MODE_AUTO = 4             /* SPARSE when the call's probabilities select fewer than 3 %
+                                      of the coordinates in expectation, else STREAM (measured
+                                      crossover on B200: p between 0.05 and 0.2, depending on N) */
 };
 
 #define WASH_MAX_N 64            /* largest population                                     */

@@ -240,6 +240,7 @@ int shuffle_impl(wash_ctx *ctx, int which, uint64_t step, double p, const double
     args.step_lo = static_cast<uint32_t>(step);
     args.step_hi8 = static_cast<uint32_t>(step >> 32) << 8;
     args.stats = reinterpret_cast<unsigned long long *>(stats);
+    int mode = ctx->mode;
     // Counters: blocks that selected something add to the caller's two words directly when
     // that stays well below one atomic per nanosecond on one address (measured limit);
     // otherwise through the partial-sum slots and a small flush kernel.
@@ -249,11 +250,17 @@ int shuffle_impl(wash_ctx *ctx, int which, uint64_t step, double p, const double
         const double kernel_ns = bytes / 6000.0 + 2000.0;
         const double reporting_blocks = std::fmin(ctx->expected_selected, static_cast<double>(ctx->n_groups) / 64.0);
         args.stat_slots = (2.0 * reporting_blocks / kernel_ns > 0.35) ? ctx->stat_slots_dev : nullptr;
-        if (ctx->mode == WASH_MODE_SPARSE) args.stat_slots = nullptr;   // one wave of large blocks: a few hundred atomics at most
+        // WASH_MODE_AUTO: the expected share of selected coordinates decides
+        if (ctx->mode == WASH_MODE_AUTO) {
+            double coordinates = 0.0;
+            for (int s = 0; s < ctx->n_seg; ++s) coordinates += static_cast<double>(ctx->seg_host[s].numel);
+            mode = ctx->expected_selected < 0.03 * coordinates ? WASH_MODE_SPARSE : WASH_MODE_STREAM;
+        }
+        if (mode == WASH_MODE_SPARSE) args.stat_slots = nullptr;   // one wave of large blocks: a few hundred atomics at most
     }
     args.status = ctx->status_dev;
     bool supported = false;
-    cudaError_t err = wash::launch_shuffle(args, a_dtype, b_dtype, ctx->mode, ctx->shape, stream, &supported);
+    cudaError_t err = wash::launch_shuffle(args, a_dtype, b_dtype, mode, ctx->shape, stream, &supported);
     if (err != cudaSuccess) return cuda_fail(err, "shuffle kernel launch");
     if (!supported) return fail(WASH_ERR_UNSUPPORTED, "no shuffle kernel for dtypes (%d, %d)", a_dtype, b_dtype);
     return WASH_OK;
@@ -423,7 +430,7 @@ int wash_bind(wash_ctx *ctx, int32_t stack, int32_t dtype, void *dev_ptr, int64_
 int wash_set_mode(wash_ctx *ctx, int32_t mode)
 {
     if (!ctx) return fail(WASH_ERR_ARG, "ctx is NULL");
-    if (mode < WASH_MODE_STREAM || mode > WASH_MODE_STREAM_REGISTERS) return fail(WASH_ERR_ARG, "unknown mode %d", mode);
+    if (mode < WASH_MODE_STREAM || mode > WASH_MODE_AUTO) return fail(WASH_ERR_ARG, "unknown mode %d", mode);
     ctx->mode = mode;
     return WASH_OK;
 }

@@ -54,7 +54,7 @@ def test_staged_streaming_kernel_matches_oracle(N, layout, mode):
     c.close()
 
 
-@pytest.mark.parametrize("mode", [B.WASH_MODE_STREAM, B.WASH_MODE_SPARSE, B.WASH_MODE_STREAM_STAGED, B.WASH_MODE_STREAM_REGISTERS])
+@pytest.mark.parametrize("mode", [B.WASH_MODE_STREAM, B.WASH_MODE_SPARSE, B.WASH_MODE_STREAM_STAGED, B.WASH_MODE_STREAM_REGISTERS, B.WASH_MODE_AUTO])
 @pytest.mark.parametrize("layout", [0, 1])
 @pytest.mark.parametrize("dtype,opt_dtype", [("f32", "f32"), ("bf16", "f32"), ("bf16", "bf16"), ("f32", "bf16"), ("bf16", None)])
 def test_shuffle_both_stacks_and_dtypes(dtype, opt_dtype, layout, mode):
@@ -92,7 +92,7 @@ def test_separate_calls_equal_the_fused_call(layout):
 def test_sparse_mode_and_launch_shapes_give_the_same_bits(N):
     ref = Case(N, RAGGED, 0, seed=8)
     oracle.shuffle(ref.ora, ref.host, 0.1, seed=2, step=3)
-    for mode in (B.WASH_MODE_STREAM, B.WASH_MODE_SPARSE, B.WASH_MODE_STREAM_STAGED, B.WASH_MODE_STREAM_REGISTERS):
+    for mode in (B.WASH_MODE_STREAM, B.WASH_MODE_SPARSE, B.WASH_MODE_STREAM_STAGED, B.WASH_MODE_STREAM_REGISTERS, B.WASH_MODE_AUTO):
         for threads, bps in ((0, 0), (64, 1), (128, 2), (256, -1), (96, 0), (32, 4), (256, 2), (128, 1)):
             c = Case(N, RAGGED, 0, seed=8)
             B.wash_set_mode(c.gpu.ctx, mode)
@@ -234,3 +234,17 @@ def test_resume_from_a_host_copy_continues_bit_identically():
     assert torch.equal(a.dev.view(torch.int32), c.dev.view(torch.int32))
     assert torch.equal(a.dev_opt.view(torch.int32), c.dev_opt.view(torch.int32))
     a.close(); c.close()
+
+
+def test_auto_mode_takes_either_kernel_and_keeps_the_bits():
+    """WASH_MODE_AUTO picks the sparse kernel below 3 % expected selection and the streaming one
+    above; a per-layer vector is judged by its expectation over the whole model."""
+    N = 6
+    numel = [70000, 9, 3000]
+    c = Case(N, numel, 0, "f32", "f32", seed=21)
+    B.wash_set_mode(c.gpu.ctx, B.WASH_MODE_AUTO)
+    for step, (p, pl) in enumerate([(0.001, None), (0.5, None), (0.0, [0.01, 1.0, 0.2]), (0.0, [0.2, 0.0, 0.0])]):
+        B.wash_shuffle_both(c.gpu.ctx, step, p, pl, seed=77, stats=c.stats_dev)
+        oracle.shuffle(c.ora, c.host, p if pl is None else pl, seed=77, step=step, stack2=c.host_opt)
+        c.assert_equal("step %d" % step)
+    c.close()
