@@ -56,6 +56,10 @@ struct F32 {
     static __device__ __forceinline__ void store_elem(void *base, long long idx, uint32_t bits) { reinterpret_cast<uint32_t *>(base)[idx] = bits; }
     static __device__ __forceinline__ float to_float(uint32_t bits) { return __uint_as_float(bits); }
     static __device__ __forceinline__ uint32_t from_float(float f) { return __float_as_uint(f); }
+    static __device__ __forceinline__ vec pack_floats(float a, float b, float c, float d)
+    {
+        return make_uint4(__float_as_uint(a), __float_as_uint(b), __float_as_uint(c), __float_as_uint(d));
+    }
 };
 
 struct BF16 {
@@ -84,6 +88,20 @@ struct BF16 {
         if ((u & 0x7FFFFFFFu) > 0x7F800000u) return (u >> 16) | 0x0040u;
         u += 0x7FFFu + ((u >> 16) & 1u);
         return u >> 16;
+    }
+    // Two values per conversion instruction (round to nearest even, as from_float); the
+    // instruction turns every NaN into one canonical pattern, so the rare pair with a NaN
+    // is redone by from_float, which keeps sign and payload.
+    static __device__ __forceinline__ uint32_t pair_from_floats(float lo, float hi)
+    {
+        uint32_t r;
+        asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+        if (lo != lo || hi != hi) r = from_float(lo) | (from_float(hi) << 16);
+        return r;
+    }
+    static __device__ __forceinline__ vec pack_floats(float a, float b, float c, float d)
+    {
+        return make_uint2(pair_from_floats(a, b), pair_from_floats(c, d));
     }
 };
 

@@ -67,8 +67,7 @@ __global__ void __launch_bounds__(256) reduce_kernel(const __grid_constant__ Red
             if constexpr (OP == kOpAverage) {
                 const long long e0 = 4ll * static_cast<long long>(g);
                 if (gi.valid == 4) {
-                    TOUT::store_group(static_cast<char *>(a.out) + e0 * TOUT::kBytes,
-                                      TOUT::pack(TOUT::from_float(m[0]), TOUT::from_float(m[1]), TOUT::from_float(m[2]), TOUT::from_float(m[3])));
+                    TOUT::store_group(static_cast<char *>(a.out) + e0 * TOUT::kBytes, TOUT::pack_floats(m[0], m[1], m[2], m[3]));
                 } else {
 #pragma unroll
                     for (int c = 0; c < 4; ++c)
@@ -76,16 +75,16 @@ __global__ void __launch_bounds__(256) reduce_kernel(const __grid_constant__ Red
                 }
             } else {
                 // new value of (model n, coordinate c)
-                auto updated = [&](int n, int c) -> uint32_t {
-                    if constexpr (OP == kOpPapaAll) return T::from_float(m[c]);
+                auto updated = [&](int n, int c) -> float {
+                    if constexpr (OP == kOpPapaAll) return m[c];
                     const float x = T::to_float(group_value<T, LAYOUT, kCap>(v, n_models, n, c));
-                    return T::from_float(__fadd_rn(__fmul_rn(a.alpha, x), __fmul_rn(a.one_minus_alpha, m[c])));
+                    return __fadd_rn(__fmul_rn(a.alpha, x), __fmul_rn(a.one_minus_alpha, m[c]));
                 };
                 if (gi.valid == 4) {
 #pragma unroll
                     for (int j = 0; j < kCap; ++j) {
                         if (j >= n_models) break;
-                        uint32_t r[4];
+                        float r[4];
 #pragma unroll
                         for (int q = 0; q < 4; ++q) {
                             // element q of vector j is (model n, coordinate c):
@@ -93,7 +92,7 @@ __global__ void __launch_bounds__(256) reduce_kernel(const __grid_constant__ Red
                             const int c = LAYOUT == kLayoutNP ? q : (4 * j + q) / n_models;
                             r[q] = updated(n, c);
                         }
-                        T::store_group(group_vec_ptr<T, LAYOUT>(a.stack, a.pop, g, j), T::pack(r[0], r[1], r[2], r[3]));
+                        T::store_group(group_vec_ptr<T, LAYOUT>(a.stack, a.pop, g, j), T::pack_floats(r[0], r[1], r[2], r[3]));
                     }
                 } else {
                     const long long e0 = 4ll * static_cast<long long>(g);
@@ -102,7 +101,7 @@ __global__ void __launch_bounds__(256) reduce_kernel(const __grid_constant__ Red
                         if (c >= gi.valid) break;
 #pragma unroll
                         for (int n = 0; n < kCap; ++n)
-                            if (n < n_models) T::store_elem(a.stack, elem_index<LAYOUT>(a.pop, n, e0 + c), updated(n, c));
+                            if (n < n_models) T::store_elem(a.stack, elem_index<LAYOUT>(a.pop, n, e0 + c), T::from_float(updated(n, c)));
                     }
                 }
             }

@@ -9,7 +9,7 @@ import torch
 import oracle
 from paper_2405_17517_b200 import binding as B
 from paper_2405_17517_b200 import workloads as W
-from gpu_util import Case, bits, to_host_bits, ulp_distance_f32
+from gpu_util import Case, bits, to_device, to_host_bits, ulp_distance_f32
 
 pytestmark = pytest.mark.gpu
 
@@ -85,6 +85,43 @@ def test_special_values_follow_ieee():
     oracle.papa_ema(c.ora, c.host, 0.9)
     torch.cuda.synchronize()
     assert ulp_distance_f32(to_host_bits(c.dev), bits(c.host)).max() == 0     # NaN == NaN by class
+    c.close()
+
+
+@pytest.mark.parametrize("layout", [0, 1])
+def test_bf16_rounding_cases_follow_the_oracle(layout):
+    """Results that land on ties, overflow to infinity, stay denormal or are NaN, in whole
+    groups (the paired conversion) and in a ragged tail (the element-wise one)."""
+    N, d = 2, 4096 + 3
+    rng = np.random.default_rng(5)
+    dense = np.zeros((N, d), dtype=np.float32)
+    # model 0 = a bf16 value, model 1 = the next bf16 value away from zero: their mean lies
+    # halfway between two bf16 values, so the average is a tie for the rounding
+    b = W.to_bf16_bits(rng.standard_normal(d).astype(np.float32)).astype(np.uint32)
+    dense[0] = (b << 16).view(np.float32); dense[1] = ((b + 1) << 16).view(np.float32)
+    dense[:, 8:16] = np.float32(3.38e38)                    # sum overflows
+    dense[0, 16:24] = np.nan; dense[1, 24:32] = -np.inf
+    dense[0, 32:40] = np.inf; dense[1, 32:40] = -np.inf      # inf - inf
+    dense[:, 40:48] = np.float32(2e-40)                      # denormal results
+    dense[0, d - 2] = np.nan                                 # in the ragged tail
+    c = Case(N, [d], layout, "bf16", dense=dense)
+
+    def same(got16, want16, what):
+        dist = ulp_distance_f32(got16.astype(np.uint32) << 16, want16.astype(np.uint32) << 16)   # NaN == NaN by class
+        assert dist.max() == 0, what
+
+    for alpha in (0.5, 0.999):
+        B.papa_ema(c.gpu.ctx, B.WASH_STACK_PARAMS, alpha)
+        oracle.papa_ema(c.ora, c.host, alpha)
+        torch.cuda.synchronize()
+        same(to_host_bits(c.dev), bits(c.host), "ema %g" % alpha)
+        c.dev.copy_(to_device(c.host))
+    out = torch.zeros(c.P, dtype=torch.bfloat16, device="cuda")
+    B.population_average(c.gpu.ctx, B.WASH_STACK_PARAMS, out, B.WASH_BF16)
+    want = np.zeros(c.P, dtype=np.uint16)
+    oracle.population_average(c.ora, c.host, want)
+    same(to_host_bits(out), want, "average")
+    B.wash_check(c.gpu.ctx)
     c.close()
 
 
