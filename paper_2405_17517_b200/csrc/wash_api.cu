@@ -235,8 +235,7 @@ int shuffle_impl(wash_ctx *ctx, int which, uint64_t step, double p, const double
     args.b = b;
     args.group_lo = group_lo;
     args.group_hi = group_hi < ctx->n_groups ? group_hi : ctx->n_groups;
-    args.key0 = static_cast<uint32_t>(seed);
-    args.key1 = static_cast<uint32_t>(seed >> 32);
+    args.keys = wash::philox_keys(seed);
     args.step_lo = static_cast<uint32_t>(step);
     args.step_hi8 = static_cast<uint32_t>(step >> 32) << 8;
     args.stats = reinterpret_cast<unsigned long long *>(stats);
@@ -658,8 +657,7 @@ int exchange_args(wash_ctx *ctx, wash::ExchangeArgs *out)
     a.self = ctx->x_self;
     a.n_wtiles = ctx->x_wtiles;
     a.n_blocks = ctx->x_blocks;
-    a.key0 = static_cast<uint32_t>(ctx->x_seed);
-    a.key1 = static_cast<uint32_t>(ctx->x_seed >> 32);
+    a.keys = wash::philox_keys(ctx->x_seed);
     a.step_lo = static_cast<uint32_t>(ctx->x_step);
     a.step_hi8 = static_cast<uint32_t>(ctx->x_step >> 32) << 8;
     a.mask = ctx->x_mask;

@@ -8,26 +8,22 @@ namespace wash {
 
 // ---- Philox4x32-10 (Salmon et al., SC'11) ------------------------------------------
 // Ten rounds of two 32x32->64 multiplies; the key advances by the two Weyl constants
-// after every round.
+// after every round (the ten keys come ready-made from the host: PhiloxKeys).
 struct Philox4 {
     uint32_t x, y, z, w;
 };
 
-__device__ __forceinline__ Philox4 philox4x32_10(uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3,
-                                                 uint32_t k0, uint32_t k1)
+__device__ __forceinline__ Philox4 philox4x32_10(uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3, const PhiloxKeys &keys)
 {
     constexpr uint32_t kMul0 = 0xD2511F53u, kMul1 = 0xCD9E8D57u;
-    constexpr uint32_t kWeyl0 = 0x9E3779B9u, kWeyl1 = 0xBB67AE85u;
 #pragma unroll
     for (int r = 0; r < 10; ++r) {
         const uint32_t hi0 = __umulhi(kMul0, c0), lo0 = kMul0 * c0;
         const uint32_t hi1 = __umulhi(kMul1, c2), lo1 = kMul1 * c2;
-        c0 = hi1 ^ c1 ^ k0;
-        c2 = hi0 ^ c3 ^ k1;
+        c0 = hi1 ^ c1 ^ keys.k[2 * r];
+        c2 = hi0 ^ c3 ^ keys.k[2 * r + 1];
         c1 = lo1;
         c3 = lo0;
-        k0 += kWeyl0;
-        k1 += kWeyl1;
     }
     return Philox4{c0, c1, c2, c3};
 }

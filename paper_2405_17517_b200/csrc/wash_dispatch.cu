@@ -68,12 +68,12 @@ __global__ void __launch_bounds__(kStatSlots) flush_stats_kernel(StatSlot *slots
 }
 
 // Nothing but the mask's Philox blocks: one block of four words per thread, folded by XOR.
-__global__ void __launch_bounds__(256) philox_probe_kernel(unsigned long long n_blocks, uint32_t k0, uint32_t k1, uint32_t *checksum)
+__global__ void __launch_bounds__(256) philox_probe_kernel(unsigned long long n_blocks, const __grid_constant__ PhiloxKeys keys, uint32_t *checksum)
 {
     const unsigned long long i = static_cast<unsigned long long>(blockIdx.x) * blockDim.x + threadIdx.x;
     uint32_t fold = 0;
     if (i < n_blocks) {
-        const Philox4 w = philox4x32_10(static_cast<uint32_t>(i), 0u, 0u, static_cast<uint32_t>(i >> 32) << 8, k0, k1);
+        const Philox4 w = philox4x32_10(static_cast<uint32_t>(i), 0u, 0u, static_cast<uint32_t>(i >> 32) << 8, keys);
         fold = w.x ^ w.y ^ w.z ^ w.w;
     }
     fold = __reduce_xor_sync(0xFFFFFFFFu, fold);
@@ -85,7 +85,7 @@ cudaError_t launch_philox_probe(unsigned long long n_blocks, uint64_t seed, uint
     if (n_blocks == 0) return cudaSuccess;
     const unsigned long long grid = (n_blocks + 255) / 256;
     if (grid > 0x7FFFFFFFull) return cudaErrorInvalidConfiguration;
-    philox_probe_kernel<<<static_cast<unsigned>(grid), 256, 0, stream>>>(n_blocks, static_cast<uint32_t>(seed), static_cast<uint32_t>(seed >> 32), checksum);
+    philox_probe_kernel<<<static_cast<unsigned>(grid), 256, 0, stream>>>(n_blocks, philox_keys(seed), checksum);
     count_launch();
     return cudaGetLastError();
 }

@@ -43,8 +43,8 @@ __device__ __forceinline__ void routes_of(const ExchangeArgs &a, uint32_t elem, 
     const GroupInfo gi = find_group(a.pop, elem >> 2, a.status);
     const uint32_t coord = 4u * gi.cgroup + (elem & 3u);
     uint64_t packed = 0;
-    if (n_models <= 16) packed = draw_permutation_packed(n_models, coord, gi.tensor_id, a.step_lo, a.step_hi8, a.key0, a.key1);
-    else draw_permutation_u8(s_perm, kXThreads, n_models, coord, gi.tensor_id, a.step_lo, a.step_hi8, a.key0, a.key1);
+    if (n_models <= 16) packed = draw_permutation_packed(n_models, coord, gi.tensor_id, a.step_lo, a.step_hi8, a.keys);
+    else draw_permutation_u8(s_perm, kXThreads, n_models, coord, gi.tensor_id, a.step_lo, a.step_hi8, a.keys);
     unsigned long long nd = 0;
     uint32_t d = kNoDestination;
     for (int n = 0; n < n_models; ++n) {

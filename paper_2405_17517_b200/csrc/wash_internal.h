@@ -42,12 +42,29 @@ struct PopView {
     const uint32_t *tile_first;   // device, segment of the first group of every tile
 };
 
+// Philox's key schedule: round r of the ten uses (k[2r], k[2r+1]) = (seed_lo + r W0, seed_hi + r W1)
+// with the two Weyl constants.  It depends on the seed only, so the host computes it once per
+// launch and a round's key reaches the kernel as an operand instead of two additions.
+struct PhiloxKeys {
+    uint32_t k[20];
+};
+inline PhiloxKeys philox_keys(uint64_t seed)
+{
+    PhiloxKeys keys;
+    uint32_t k0 = static_cast<uint32_t>(seed), k1 = static_cast<uint32_t>(seed >> 32);
+    for (int r = 0; r < 10; ++r, k0 += 0x9E3779B9u, k1 += 0xBB67AE85u) {
+        keys.k[2 * r] = k0;
+        keys.k[2 * r + 1] = k1;
+    }
+    return keys;
+}
+
 struct ShuffleArgs {
     PopView pop;
     void *a;                      // first stack (device)
     void *b;                      // second stack or nullptr
     uint32_t group_lo, group_hi;  // groups of a row to process (whole row: 0 .. n_groups)
-    uint32_t key0, key1;          // seed
+    PhiloxKeys keys;              // from the seed
     uint32_t step_lo, step_hi8;   // step & 0xFFFFFFFF, (step >> 32) << 8
     unsigned long long *stats;    // device-accessible {selected, moved} or nullptr
     StatSlot *stat_slots;         // device, kStatSlots zeroed entries (left zeroed by every launch), or nullptr
@@ -76,7 +93,7 @@ struct ExchangeArgs {
     int self;                     // this worker's index in the population
     uint32_t n_wtiles;            // ceil(n_groups / kExchangeTileGroups)
     uint32_t n_blocks;            // grid of all three kernels; its warps share the warp tiles evenly, in order
-    uint32_t key0, key1;
+    PhiloxKeys keys;
     uint32_t step_lo, step_hi8;
     uint32_t *mask;               // [n_wtiles * 32] a word per lane = its four groups' bytes; low nibble of a byte:
                                   // selected coordinates, high nibble: those this worker receives

@@ -148,8 +148,7 @@ extern "C" int wash_shuffle_noalloc(int32_t N, int32_t n_tensors, const int64_t 
             args.b = nullptr;
             args.group_lo = 0;
             args.group_hi = n_groups;
-            args.key0 = static_cast<uint32_t>(seed);
-            args.key1 = static_cast<uint32_t>(seed >> 32);
+            args.keys = wash::philox_keys(seed);
             args.step_lo = static_cast<uint32_t>(step);
             args.step_hi8 = static_cast<uint32_t>(step >> 32) << 8;
             args.stats = reinterpret_cast<unsigned long long *>(stats);

@@ -26,12 +26,12 @@ namespace wash {
 // j = floor(word * (k+1) / 2^32).
 static __device__ __noinline__ void draw_permutation(uint32_t *s_perm, int ts, int n_models, uint32_t i,
                                               uint32_t tensor, uint32_t step_lo, uint32_t step_hi8,
-                                              uint32_t k0, uint32_t k1)
+                                              const PhiloxKeys &keys)
 {
     for (int n = 0; n < n_models; ++n) s_perm[n * ts] = n;
     Philox4 w{0, 0, 0, 0};
     for (int k = n_models - 1, m = 0; k >= 1; --k, ++m) {
-        if ((m & 3) == 0) w = philox4x32_10(i, tensor, step_lo, step_hi8 | (1u + (static_cast<uint32_t>(m) >> 2)), k0, k1);
+        if ((m & 3) == 0) w = philox4x32_10(i, tensor, step_lo, step_hi8 | (1u + (static_cast<uint32_t>(m) >> 2)), keys);
         const uint32_t r = w.x;
         w.x = w.y; w.y = w.z; w.z = w.w;
         const uint32_t j = __umulhi(r, static_cast<uint32_t>(k + 1));
@@ -67,7 +67,7 @@ __global__ void __launch_bounds__(256) shuffle_kernel(const __grid_constant__ Sh
         }
         const GroupInfo gi = find_group(a.pop, static_cast<uint32_t>(g), a.status);
         if (gi.thr == 0 || gi.valid == 0) continue;
-        const Philox4 w = philox4x32_10(gi.cgroup, gi.tensor_id, a.step_lo, a.step_hi8, a.key0, a.key1);
+        const Philox4 w = philox4x32_10(gi.cgroup, gi.tensor_id, a.step_lo, a.step_hi8, a.keys);
         uint32_t sel = 0;
         sel |= (static_cast<uint64_t>(w.x) < gi.thr && gi.valid > 0) ? 1u : 0u;
         sel |= (static_cast<uint64_t>(w.y) < gi.thr && gi.valid > 1) ? 2u : 0u;
@@ -77,7 +77,7 @@ __global__ void __launch_bounds__(256) shuffle_kernel(const __grid_constant__ Sh
 #pragma unroll
         for (int c = 0; c < 4; ++c) {
             if (!((sel >> c) & 1u)) continue;
-            draw_permutation(s_perm, ts, n_models, 4u * gi.cgroup + c, gi.tensor_id, a.step_lo, a.step_hi8, a.key0, a.key1);
+            draw_permutation(s_perm, ts, n_models, 4u * gi.cgroup + c, gi.tensor_id, a.step_lo, a.step_hi8, a.keys);
             const long long e = 4ll * static_cast<long long>(g) + c;
             // first stack
             if constexpr (STREAM) {

@@ -85,12 +85,12 @@ __device__ __forceinline__ uint32_t image_value(const unsigned char *image, int 
 // pi for coordinate i with pi(n) in nibble n of the result (N <= 16): the Fisher-Yates of
 // draw_permutation_u8 on a register instead of a shared-memory column.
 __device__ __forceinline__ uint64_t draw_permutation_packed(int n_models, uint32_t i, uint32_t tensor, uint32_t step_lo,
-                                                            uint32_t step_hi8, uint32_t k0, uint32_t k1)
+                                                            uint32_t step_hi8, const PhiloxKeys &keys)
 {
     uint64_t perm = 0xFEDCBA9876543210ull;
     Philox4 w{0, 0, 0, 0};
     for (int k = n_models - 1, m = 0; k >= 1; --k, ++m) {
-        if ((m & 3) == 0) w = philox4x32_10(i, tensor, step_lo, step_hi8 | (1u + (static_cast<uint32_t>(m) >> 2)), k0, k1);
+        if ((m & 3) == 0) w = philox4x32_10(i, tensor, step_lo, step_hi8 | (1u + (static_cast<uint32_t>(m) >> 2)), keys);
         const uint32_t r = w.x;
         w.x = w.y; w.y = w.z; w.z = w.w;
         const uint32_t sk = 4u * k, sj = 4u * __umulhi(r, static_cast<uint32_t>(k + 1));
@@ -138,8 +138,8 @@ __device__ __forceinline__ void serve_tile(const ShuffleArgs &a, const unsigned 
         const uint32_t t_owner = warp_base + owner;
         const long long e = 4ll * static_cast<long long>(g_block + t_owner) + c;
         uint64_t perm = 0;
-        if (n_models <= 16) perm = draw_permutation_packed(n_models, 4u * cgroup + c, tensor, a.step_lo, a.step_hi8, a.key0, a.key1);
-        else draw_permutation_u8(s_perm, T_, n_models, 4u * cgroup + c, tensor, a.step_lo, a.step_hi8, a.key0, a.key1);
+        if (n_models <= 16) perm = draw_permutation_packed(n_models, 4u * cgroup + c, tensor, a.step_lo, a.step_hi8, a.keys);
+        else draw_permutation_u8(s_perm, T_, n_models, 4u * cgroup + c, tensor, a.step_lo, a.step_hi8, a.keys);
         auto source_of = [&](int n) -> int {
             return n_models <= 16 ? static_cast<int>((perm >> (4 * n)) & 15ull) : static_cast<int>(s_perm[n * T_]);
         };
@@ -204,7 +204,7 @@ __global__ void __launch_bounds__(256, 5) shuffle_async_kernel(const __grid_cons
         if (threadIdx.x < in_tile[i]) {
             gi[i] = find_group(a.pop, static_cast<uint32_t>(g_first + static_cast<uint64_t>(i) * T_ + threadIdx.x), a.status);
             if (gi[i].thr != 0 && gi[i].valid != 0) {
-                const Philox4 w = philox4x32_10(gi[i].cgroup, gi[i].tensor_id, a.step_lo, a.step_hi8, a.key0, a.key1);
+                const Philox4 w = philox4x32_10(gi[i].cgroup, gi[i].tensor_id, a.step_lo, a.step_hi8, a.keys);
                 // word < thr with thr in [0, 2^32]: a 32-bit compare, or always when thr is 2^32
                 const uint32_t thr_lo = static_cast<uint32_t>(gi[i].thr);
                 const bool always = (gi[i].thr >> 32) != 0;

@@ -54,8 +54,8 @@ __global__ void __launch_bounds__(kSparseThreads, 4) shuffle_sparse_kernel(const
             const GroupInfo gi = find_group(a.pop, static_cast<uint32_t>(e >> 2), a.status);
             const uint32_t coord = 4u * gi.cgroup + static_cast<uint32_t>(e & 3);
             uint64_t perm = 0;
-            if (n_models <= 16) perm = draw_permutation_packed(n_models, coord, gi.tensor_id, a.step_lo, a.step_hi8, a.key0, a.key1);
-            else draw_permutation_u8(s_perm, kSparseThreads, n_models, coord, gi.tensor_id, a.step_lo, a.step_hi8, a.key0, a.key1);
+            if (n_models <= 16) perm = draw_permutation_packed(n_models, coord, gi.tensor_id, a.step_lo, a.step_hi8, a.keys);
+            else draw_permutation_u8(s_perm, kSparseThreads, n_models, coord, gi.tensor_id, a.step_lo, a.step_hi8, a.keys);
             auto source_of = [&](int n) -> int {
                 return n_models <= 16 ? static_cast<int>((perm >> (4 * n)) & 15ull) : static_cast<int>(s_perm[n * kSparseThreads]);
             };

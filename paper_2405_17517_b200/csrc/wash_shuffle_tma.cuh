@@ -101,12 +101,12 @@ __device__ __forceinline__ void bulk_load(uint32_t dst_smem, const void *src, ui
 // pi for coordinate i in a column of bytes: s_perm[n * stride]
 static __device__ __noinline__ void draw_permutation_u8(uint8_t *s_perm, int stride, int n_models, uint32_t i,
                                                         uint32_t tensor, uint32_t step_lo, uint32_t step_hi8,
-                                                        uint32_t k0, uint32_t k1)
+                                                        const PhiloxKeys &keys)
 {
     for (int n = 0; n < n_models; ++n) s_perm[n * stride] = static_cast<uint8_t>(n);
     Philox4 w{0, 0, 0, 0};
     for (int k = n_models - 1, m = 0; k >= 1; --k, ++m) {
-        if ((m & 3) == 0) w = philox4x32_10(i, tensor, step_lo, step_hi8 | (1u + (static_cast<uint32_t>(m) >> 2)), k0, k1);
+        if ((m & 3) == 0) w = philox4x32_10(i, tensor, step_lo, step_hi8 | (1u + (static_cast<uint32_t>(m) >> 2)), keys);
         const uint32_t r = w.x;
         w.x = w.y; w.y = w.z; w.z = w.w;
         const uint32_t j = __umulhi(r, static_cast<uint32_t>(k + 1));
@@ -271,7 +271,7 @@ __global__ void __launch_bounds__(32 * kProducerWarps + 512) shuffle_tma_kernel(
         if (g < a.s.pop.n_groups) {
             gi = find_group_forward(seg, a.s.pop.n_seg, cursor, static_cast<uint32_t>(g), a.s.status);
             if (gi.thr != 0 && gi.valid != 0) {
-                const Philox4 w = philox4x32_10(gi.cgroup, gi.tensor_id, a.s.step_lo, a.s.step_hi8, a.s.key0, a.s.key1);
+                const Philox4 w = philox4x32_10(gi.cgroup, gi.tensor_id, a.s.step_lo, a.s.step_hi8, a.s.keys);
                 sel |= (static_cast<uint64_t>(w.x) < gi.thr && gi.valid > 0) ? 1u : 0u;
                 sel |= (static_cast<uint64_t>(w.y) < gi.thr && gi.valid > 1) ? 2u : 0u;
                 sel |= (static_cast<uint64_t>(w.z) < gi.thr && gi.valid > 2) ? 4u : 0u;
@@ -290,7 +290,7 @@ __global__ void __launch_bounds__(32 * kProducerWarps + 512) shuffle_tma_kernel(
 #pragma unroll 1
             for (int c = 0; c < 4; ++c) {
                 if (!((sel >> c) & 1u)) continue;
-                draw_permutation_u8(s_perm, consumers, n_models, 4u * gi.cgroup + c, gi.tensor_id, a.s.step_lo, a.s.step_hi8, a.s.key0, a.s.key1);
+                draw_permutation_u8(s_perm, consumers, n_models, 4u * gi.cgroup + c, gi.tensor_id, a.s.step_lo, a.s.step_hi8, a.s.keys);
                 const long long e = 4ll * static_cast<long long>(g) + c;
                 for (int n = 0; n < n_models; ++n) {
                     const int src = s_perm[n * consumers];

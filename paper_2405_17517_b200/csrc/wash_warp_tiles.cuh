@@ -4,7 +4,7 @@
 // overlap, one table lookup serves all four, and its four mask nibbles fit one word.  A warp
 // visits a contiguous range of warp tiles in order.
 //
-// `A` is the kernel's argument struct; it has the fields pop, key0, key1, step_lo, step_hi8, status.
+// `A` is the kernel's argument struct; it has the fields pop, keys, step_lo, step_hi8, status.
 #pragma once
 #include "wash_device.cuh"
 
@@ -53,7 +53,7 @@ template <class A>
 __device__ __forceinline__ uint32_t draw_mask(const GroupInfo &gi, const A &a)
 {
     if (gi.thr == 0 || gi.valid == 0) return 0;
-    const Philox4 w = philox4x32_10(gi.cgroup, gi.tensor_id, a.step_lo, a.step_hi8, a.key0, a.key1);
+    const Philox4 w = philox4x32_10(gi.cgroup, gi.tensor_id, a.step_lo, a.step_hi8, a.keys);
     const uint32_t thr_lo = static_cast<uint32_t>(gi.thr);
     const bool always = (gi.thr >> 32) != 0;
     uint32_t m = 0;
