@@ -262,13 +262,16 @@ def run_ours(args, rank: int, world: int, local_rank: int) -> None:
     p_layer = wl.p_layer
     stream = torch.cuda.current_stream()
 
-    def step(i, ev=None):
-        if ev is not None:
-            ev[0].record(stream)
+    def step_shuffle(i):
         if opt_d is not None:
             B.wash_shuffle_both(pop.ctx, i, wl.p, p_layer, SEED, stream, stats_d)
         else:
             B.wash_shuffle(pop.ctx, i, wl.p, p_layer, SEED, stream, stats_d)
+
+    def step(i, ev=None):
+        if ev is not None:
+            ev[0].record(stream)
+        step_shuffle(i)
         if ev is not None:
             ev[1].record(stream)
         B.papa_ema(pop.ctx, B.WASH_STACK_PARAMS, ALPHA, stream)
@@ -318,6 +321,30 @@ def run_ours(args, rank: int, world: int, local_rank: int) -> None:
     k_ms = np.array([[e[i].elapsed_time(e[i + 1]) for i in range(3)] for e in events])   # shuffle, ema, average
     mean_ms = k_ms.mean(axis=0)
 
+    # ---- the shuffle alone, launched back to back (no event between launches), in the
+    # streaming mode and in the sparse mode: context for the per-kernel figures above, which
+    # carry an event pair per launch, and the parameter-swaps/s the sparse kernel reaches
+    def shuffle_alone(mode, n):
+        B.wash_set_mode(pop.ctx, mode)
+        first = args.warmup + 2 * args.steps + 1000
+        for k in range(3):
+            step_shuffle(first + k)
+        fence()
+        a0 = torch.cuda.Event(enable_timing=True)
+        a1 = torch.cuda.Event(enable_timing=True)
+        a0.record(stream)
+        for k in range(n):
+            step_shuffle(first + 3 + k)
+        a1.record(stream)
+        fence()
+        return a0.elapsed_time(a1) / n
+
+    alone_ms = None
+    if args.mode == "stream":
+        n_alone = max(1, min(args.steps, 300))
+        alone_ms = [shuffle_alone(B.WASH_MODE_STREAM, n_alone), shuffle_alone(B.WASH_MODE_SPARSE, n_alone)]
+        B.wash_set_mode(pop.ctx, B.WASH_MODE_STREAM)
+
     # ---- end to end through the host-buffer entry point --------------------------------
     e2e_steps = max(1, min(args.steps, 5))
     ops = B.WASH_OP_SHUFFLE | B.WASH_OP_EMA | B.WASH_OP_AVERAGE
@@ -337,10 +364,12 @@ def run_ours(args, rank: int, world: int, local_rank: int) -> None:
 
     # ---- max over ranks ------------------------------------------------------------------
     if dist is not None:
-        t = torch.tensor([total_ms, e2e_ms, mean_ms[0], mean_ms[1], mean_ms[2]], dtype=torch.float64, device="cuda")
+        t = torch.tensor([total_ms, e2e_ms, mean_ms[0], mean_ms[1], mean_ms[2]] + (alone_ms or [0.0, 0.0]), dtype=torch.float64, device="cuda")
         dist.all_reduce(t, op=dist.ReduceOp.MAX)
         total_ms, e2e_ms = float(t[0]), float(t[1])
-        mean_ms = t[2:].cpu().numpy()
+        mean_ms = t[2:5].cpu().numpy()
+        if alone_ms is not None:
+            alone_ms = [float(t[5]), float(t[6])]
         c = torch.tensor([selected_total, moved_total], dtype=torch.int64, device="cuda")
         dist.all_reduce(c, op=dist.ReduceOp.SUM)
         selected_total, moved_total = int(c[0]), int(c[1])
@@ -382,6 +411,17 @@ def run_ours(args, rank: int, world: int, local_rank: int) -> None:
             "gpu_launches": int(launches),
             "clocks": clocks,
         }
+        if alone_ms is not None:
+            sel_step = selected_total / args.steps
+            line["shuffle_back_to_back"] = {
+                "launches": max(1, min(args.steps, 300)),
+                "stream": {"ms": alone_ms[0], "GBps": ab["shuffle"] / (alone_ms[0] * 1e-3) / 1e9,
+                           "frac_of_hbm": ab["shuffle"] / (alone_ms[0] * 1e-3) / 1e9 / peak,
+                           "param_swaps_per_s": sel_step * wl.N / (alone_ms[0] * 1e-3)},
+                "sparse": {"ms": alone_ms[1], "param_swaps_per_s": sel_step * wl.N / (alone_ms[1] * 1e-3),
+                           "bound": "integer pipes (one Philox block per 4 coordinates), not HBM"},
+                "note": "the step's shuffle launched alone, two events around the whole series; WASH_MODE_AUTO picks the sparse kernel below 3 % expected selection",
+            }
         if world == 1 and not args.no_cpu_baseline:
             line["cpu_baseline"] = cpu_baseline(wl)
         print(json.dumps(line), flush=True)
@@ -394,8 +434,8 @@ def run_ours(args, rank: int, world: int, local_rank: int) -> None:
 # DRAM bytes per shuffle launch from the ncu capture summarised under profiles/ (None
 # until a capture of the current kernel exists).
 TRAFFIC = {
-    # shuffle_async_kernel<F32, F32, [N][P], 1>: 448.9 MB read + 6.0 MB written per launch
-    "cfg2_resnet18_n5": {"dram_bytes": 448.9e6 + 6.0e6,
+    # shuffle_async_kernel<F32, F32, [N][P], 1>: 448.9 MB read + 5.9 MB written per launch
+    "cfg2_resnet18_n5": {"dram_bytes": 448.9e6 + 5.9e6,
                          "source": "profiles/shuffle_async_kernel_cfg2_resnet18_n5.md"},
 }
 
