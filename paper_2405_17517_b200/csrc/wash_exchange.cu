@@ -100,19 +100,12 @@ __global__ void __launch_bounds__(kXThreads, kExchangeBlocksPerSm) exchange_plan
         __syncwarp();
         head += count;
     };
+    LaneSegment ls{1, 0, 0, 0, 0};
+    const uint32_t whole_tiles = a.pop.n_groups / kExchangeTileGroups;   // tiles with all 128 groups inside the row
     for (uint32_t t = t0; t < t1; ++t) {
-        const uint32_t g0 = t * kExchangeTileGroups + 4u * lane;
-        const LaneGroups lg = describe_groups(a, g0, cursor);
+        const uint32_t g0 = t * kExchangeTileGroups + 4u * lane;   // rows are shorter than 2^32 elements: no wrap
         uint32_t sel4 = 0;
-        if (lg.one_tensor) {
-            if (lg.thr != 0) {
-#pragma unroll
-                for (int q = 0; q < 4; ++q) sel4 |= draw_mask(lane_group(a, lg, g0, q), a) << (8 * q);
-            }
-        } else {
-#pragma unroll 1
-            for (int q = 0; q < 4; ++q) sel4 |= draw_mask(lane_group(a, lg, g0, q), a) << (8 * q);
-        }
+        if (!(t < whole_tiles && lane_masks_fast(a, g0, ls, &sel4))) sel4 = lane_masks_general(a, g0, ls, cursor);
         a.mask[static_cast<size_t>(t) * 32u + lane] = sel4;
         if (__any_sync(kFull, sel4 != 0)) {
             tail = ring_append(s_ring[warp], tail, sel4, t - t0);   // orders the mask stores before the rounds' atomics, too

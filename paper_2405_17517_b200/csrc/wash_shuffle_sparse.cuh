@@ -79,46 +79,15 @@ __global__ void __launch_bounds__(kSparseThreads, 4) shuffle_sparse_kernel(const
         __syncwarp();
         head += count;
     };
-    // The segment this lane's groups were last found in, kept in registers: while the lane's four
-    // groups lie among that segment's whole groups (and the tile lies wholly inside the range),
-    // a tile costs two compares, four Philox blocks and sixteen word compares.  Everything else
-    // -- a tensor's end, its ragged last group, the range's last tile, a threshold of 2^32 --
-    // takes the general path, which also refreshes the registers.
-    uint32_t c_begin = 1, c_full_end = 0, c_cgroup_off = 0, c_tensor = 0, c_thr = 0;
+    LaneSegment ls{1, 0, 0, 0, 0};
     const uint32_t whole_tiles = (a.group_hi - a.group_lo) / kWarpTileGroups;   // tiles with all 128 groups inside the range
     for (uint32_t t = t0; t < t1; ++t) {
         uint32_t sel4 = 0;
         const uint32_t g0 = a.group_lo + t * kWarpTileGroups + 4u * lane;   // meaningful (no wrap) when t < whole_tiles
-        if (t < whole_tiles && g0 >= c_begin && g0 + 4u <= c_full_end) {
-            if (c_thr != 0) {
-#pragma unroll
-                for (int q = 0; q < 4; ++q) {
-                    const Philox4 w = philox4x32_10(g0 + c_cgroup_off + q, c_tensor, a.step_lo, a.step_hi8, a.keys);
-                    const uint32_t m = (w.x < c_thr ? 1u : 0u) | (w.y < c_thr ? 2u : 0u) | (w.z < c_thr ? 4u : 0u) | (w.w < c_thr ? 8u : 0u);
-                    sel4 |= m << (8 * q);
-                }
-            }
-        } else {
+        if (!(t < whole_tiles && lane_masks_fast(a, g0, ls, &sel4))) {
             const uint64_t g0_wide = static_cast<uint64_t>(a.group_lo) + static_cast<uint64_t>(t) * kWarpTileGroups + 4u * lane;
-            if (g0_wide < a.group_hi) {   // ranges end on multiples of 4 groups: a lane's groups are all inside or all outside
-                const uint32_t g = static_cast<uint32_t>(g0_wide);
-                const LaneGroups lg = describe_groups(a, g, cursor);
-                if (lg.one_tensor) {
-                    if (lg.thr != 0) {
-#pragma unroll
-                        for (int q = 0; q < 4; ++q) sel4 |= draw_mask(lane_group(a, lg, g, q), a) << (8 * q);
-                    }
-                } else {
-#pragma unroll 1
-                    for (int q = 0; q < 4; ++q) sel4 |= draw_mask(lane_group(a, lg, g, q), a) << (8 * q);
-                }
-                const SegEntry &se = a.pop.seg[cursor];
-                c_begin = se.group_begin;
-                c_full_end = (se.thr >> 32) != 0 ? 0u : se.group_begin + se.numel / 4u;   // 2^32 selects always: general path
-                c_cgroup_off = se.cgroup_begin - se.group_begin;                           // modulo 2^32, as the sum above
-                c_tensor = se.tensor_id;
-                c_thr = static_cast<uint32_t>(se.thr);
-            }
+            // ranges end on multiples of 4 groups: a lane's groups are all inside or all outside
+            if (g0_wide < a.group_hi) sel4 = lane_masks_general(a, static_cast<uint32_t>(g0_wide), ls, cursor);
         }
         if (__any_sync(kFull, sel4 != 0)) {
             tail = ring_append(ring, tail, sel4, t - t0);

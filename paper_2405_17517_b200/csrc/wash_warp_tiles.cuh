@@ -64,6 +64,60 @@ __device__ __forceinline__ uint32_t draw_mask(const GroupInfo &gi, const A &a)
     return m & ((1u << gi.valid) - 1u);
 }
 
+// The segment a lane's groups were last found in, kept in registers.  While the lane's four
+// groups lie among that segment's whole groups a tile costs two compares, four Philox blocks
+// and sixteen word compares (lane_masks_fast); everything else -- a tensor's end, its ragged
+// last group, a threshold of 2^32 -- takes lane_masks_general, which also refreshes the
+// registers.  Starts empty: {1, 0, 0, 0, 0}.
+struct LaneSegment {
+    uint32_t begin, full_end;   // the segment's whole groups (full_end = 0: none take the fast path)
+    uint32_t cgroup_off;        // group index within the tensor = group + cgroup_off (modulo 2^32)
+    uint32_t tensor, thr;
+};
+
+// The masks of groups g0 .. g0+3 (a nibble per byte) if they are whole groups of the lane's
+// segment; false if the general path must take them.  g0 + 4 must not wrap.
+template <class A>
+__device__ __forceinline__ bool lane_masks_fast(const A &a, uint32_t g0, const LaneSegment &ls, uint32_t *sel4)
+{
+    if (g0 < ls.begin || g0 + 4u > ls.full_end) return false;
+    uint32_t m4 = 0;
+    if (ls.thr != 0) {
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            const Philox4 w = philox4x32_10(g0 + ls.cgroup_off + q, ls.tensor, a.step_lo, a.step_hi8, a.keys);
+            const uint32_t m = (w.x < ls.thr ? 1u : 0u) | (w.y < ls.thr ? 2u : 0u) | (w.z < ls.thr ? 4u : 0u) | (w.w < ls.thr ? 8u : 0u);
+            m4 |= m << (8 * q);
+        }
+    }
+    *sel4 = m4;
+    return true;
+}
+
+// The same for any four groups of the row (those beyond its end select nothing).
+template <class A>
+__device__ __forceinline__ uint32_t lane_masks_general(const A &a, uint32_t g0, LaneSegment &ls, uint32_t &cursor)
+{
+    uint32_t sel4 = 0;
+    const LaneGroups lg = describe_groups(a, g0, cursor);
+    if (lg.one_tensor) {
+        if (lg.thr != 0) {
+#pragma unroll
+            for (int q = 0; q < 4; ++q) sel4 |= draw_mask(lane_group(a, lg, g0, q), a) << (8 * q);
+        }
+    } else {
+#pragma unroll 1
+        for (int q = 0; q < 4; ++q) sel4 |= draw_mask(lane_group(a, lg, g0, q), a) << (8 * q);
+    }
+    const SegEntry &se = a.pop.seg[cursor];
+    ls.begin = se.group_begin;
+    ls.full_end = (se.thr >> 32) != 0 ? 0u : se.group_begin + se.numel / 4u;   // 2^32 selects always: general path
+    ls.cgroup_off = se.cgroup_begin - se.group_begin;
+    ls.tensor = se.tensor_id;
+    ls.thr = static_cast<uint32_t>(se.thr);
+    return sel4;
+}
+
 __device__ __forceinline__ uint32_t warp_exclusive_scan(uint32_t mine, uint32_t *total)
 {
     const uint32_t lane = threadIdx.x & 31u;
