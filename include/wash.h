@@ -64,9 +64,11 @@ enum wash_mode {
     WASH_MODE_STREAM_REGISTERS = 3,/* as STREAM, the loads held in registers (kernels unrolled
                                       for N in {2,3,4,5,6,8,10,12,16,20,24,32}; other N run
                                       the default kernel)                                     */
-    WASH_MODE_AUTO = 4             /* SPARSE when the call's probabilities select fewer than 3 %
-                                      of the coordinates in expectation, else STREAM (measured
-                                      crossover on B200: p between 0.05 and 0.2, depending on N) */
+    WASH_MODE_AUTO = 4             /* SPARSE when the call's probabilities select, in expectation,
+                                      fewer than 3 % of the coordinates of an [N][padded_P] stack
+                                      or 10 % of a [padded_P][N] stack, else STREAM (the measured
+                                      crossovers on B200: in the second layout the N values of a
+                                      coordinate share a DRAM access)                            */
 };
 
 #define WASH_MAX_N 64            /* largest population                                     */

@@ -253,7 +253,10 @@ int shuffle_impl(wash_ctx *ctx, int which, uint64_t step, double p, const double
         if (ctx->mode == WASH_MODE_AUTO) {
             double coordinates = 0.0;
             for (int s = 0; s < ctx->n_seg; ++s) coordinates += static_cast<double>(ctx->seg_host[s].numel);
-            mode = ctx->expected_selected < 0.03 * coordinates ? WASH_MODE_SPARSE : WASH_MODE_STREAM;
+            // measured crossover of the two kernels: serving a coordinate costs a 128-byte DRAM access per model
+            // and stack in [N][P], one or two for all N models in [P][N]
+            const double share = ctx->layout == WASH_LAYOUT_PN ? 0.10 : 0.03;
+            mode = ctx->expected_selected < share * coordinates ? WASH_MODE_SPARSE : WASH_MODE_STREAM;
         }
         if (mode == WASH_MODE_SPARSE) args.stat_slots = nullptr;   // one wave of large blocks: a few hundred atomics at most
     }
