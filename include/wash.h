@@ -48,7 +48,7 @@ enum wash_status {
     WASH_ERR_STATE = -2,       /* call not valid now (e.g. stack not bound)               */
     WASH_ERR_ALLOC = -3,       /* host or device allocation failed                        */
     WASH_ERR_CUDA = -4,        /* a CUDA runtime call or a launch failed                  */
-    WASH_ERR_UNSUPPORTED = -5, /* valid request this build has no kernel for              */
+    WASH_ERR_UNSUPPORTED = -5, /* valid request the library has no kernel for             */
     WASH_ERR_DEVICE_CHECK = -6 /* a device-side consistency check tripped (wash_check)    */
 };
 enum wash_layout { WASH_LAYOUT_NP = 0 /* [N][padded_P] */, WASH_LAYOUT_PN = 1 /* [padded_P][N] */ };

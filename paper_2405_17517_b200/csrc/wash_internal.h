@@ -120,7 +120,7 @@ struct LaunchShape {
 };
 
 // Each returns cudaSuccess or the launch error; *supported = false (and no launch) if
-// this build has no kernel for the combination.
+// the library has no kernel for the combination.
 cudaError_t launch_shuffle(const ShuffleArgs &args, int a_dtype, int b_dtype, int mode,
                            const LaunchShape &shape, cudaStream_t stream, bool *supported);
 cudaError_t launch_reduce(const ReduceArgs &args, int op, int dtype, int out_dtype,
