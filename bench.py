@@ -2,16 +2,21 @@
 """Benchmark of the WASH hot path on B200: one JSON line on stdout.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
-                    [--workload cfg2_resnet18_n5|cfg3_resnet50_n10|cfg4_resnet50_bf16_n8|cfg1_flat_n3]
+                    [--workload cfg3_resnet50_n10|cfg2_resnet18_n5|cfg4_resnet50_bf16_n8|cfg1_flat_n3]
 
 A step is one pass of the whole hot path over one synthetic population: the shuffle of
 the parameter and momentum stacks (WASH+Opt, one launch), PAPA's EMA on the parameters
-and the final average -- three kernel launches.  `value` is the bytes those kernels
-must stream (see algorithmic_bytes) divided by the step time, in GB/s, with the stacks
-resident in HBM; `e2e` is the same through wash_step_host with the stacks in pinned
-host memory (copies inside the timed region).  For N > 1 (torchrun) every rank holds
-its own shard of an N-times deeper population (tensor indices offset by rank), no
-communication: weak scaling.
+and the final average -- three kernel launches.  `value` is the shuffle's own
+throughput: the bytes the shuffle must move (see algorithmic_bytes) divided by the time
+of the shuffle kernel inside the step, in GB/s, with the stacks resident in HBM;
+`ms_per_step` and the `step` record cover the three kernels; `e2e` is the shuffle
+through wash_step_host with the stacks in pinned host memory (copies inside the timed
+region).  The timed block of --steps steps is repeated until at least half a second of
+GPU time has been measured; medians over the blocks are reported.  `configs` holds the
+other configurations and cells of the config-5 sweep, timed in the same run with both
+ceilings (HBM copy bandwidth and the integer pipes' Philox rate).  For N > 1 (torchrun)
+every rank holds its own shard of an N-times deeper population (tensor indices offset
+by rank), no communication: weak scaling.
 
 --impl reference times the CPU oracle (oracle/) on the host cores instead.
 """
@@ -61,6 +66,7 @@ class Workload:
         self.opt = cfg["opt"]
         self.E = 2 if self.bf16 else 4
         self.E_opt = 4 if self.opt else 0
+        self.Es = (self.E, 4) if self.opt else (self.E,)
         # rank r holds tensors r*T .. r*T+T-1 of a world_size-times deeper population
         self.tensor_id = np.arange(self.T, dtype=np.uint32) + np.uint32(rank * self.T)
         self.schedule = cfg["schedule"]     # None = uniform p; each arm derives p_layer with its own routine
@@ -161,9 +167,12 @@ def run_reference(args, rank: int, world: int) -> None:
     if wl.schedule == "decreasing":
         wl.p_layer = oracle.layer_probs(wl.T, wl.p, oracle.SCHEDULE_DECREASING)
 
-    def one_step(pop, a, b, out, step, p_layer):
+    def one_step(pop, a, b, out, step, p_layer, clock=None):
         p = wl.p if p_layer is None else p_layer
+        t0 = time.perf_counter()
         st = oracle.shuffle(pop, a, p, seed=SEED, step=step, stack2=b)
+        if clock is not None:
+            clock[0] += time.perf_counter() - t0
         oracle.papa_ema(pop, a, ALPHA)
         oracle.population_average(pop, a, out)
         return st
@@ -191,20 +200,24 @@ def run_reference(args, rank: int, world: int) -> None:
     for w in range(args.warmup):
         one_step(sub, sp, so, sout, w, sub_pl)
     sel = 0
+    clock = [0.0]
     t0 = time.perf_counter()
     for k in range(args.steps):
-        sel += one_step(sub, sp, so, sout, args.warmup + k, sub_pl)[0]
+        sel += one_step(sub, sp, so, sout, args.warmup + k, sub_pl, clock)[0]
     dt = time.perf_counter() - t0
     scale = sub_P / wl.P
-    bytes_step = wl.algorithmic_bytes(sel / max(args.steps, 1) / scale)["step"] * scale
-    gbs = bytes_step * args.steps / dt / 1e9
+    ab = wl.algorithmic_bytes(sel / max(args.steps, 1) / scale)
+    gbs = ab["shuffle"] * scale * args.steps / clock[0] / 1e9           # the headline metric: the shuffle's own throughput
     sample = "first %d of %d tensors (%d of %d coordinates per model) per step" % (n_t, wl.T, sub_P, wl.P)
     line = {
         "impl": "reference", "metric": METRIC, "value": gbs, "unit": "GB/s", "n_gpus": args.gpus, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": dt / max(args.steps, 1) * 1e3, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "bf16+f32" if wl.bf16 else "f32", "data": "synthetic",
+        "value_definition": "the oracle's shuffle: bytes the shuffle of both stacks must move / the time spent in the oracle's shuffle; "
+                            "ms_per_step is the whole step (shuffle + EMA + average) on the sample",
         "config": {"workload": wl.name, "N": wl.N, "tensors": wl.T, "P": wl.P, "p": wl.p, "sample": sample},
-        "param_swaps_per_s": sel * wl.N / dt,
+        "param_swaps_per_s": sel * wl.N / clock[0],
+        "step": {"ms": dt / max(args.steps, 1) * 1e3, "GBps": ab["step"] * scale * args.steps / dt / 1e9},
         "cpu_baseline": {"value": gbs, "unit": "GB/s", "cores": threads, "kind": "oracle", "sample": sample},
         "e2e": {"value": gbs, "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
@@ -213,6 +226,157 @@ def run_reference(args, rank: int, world: int) -> None:
 
 
 # ------------------------------------------------------------------------------------
+MIN_TIMED_S = 0.5          # the timed blocks are repeated until this much GPU time has been measured
+MAX_REPEATS = 400
+
+
+def philox_blocks(P: int, N: int, selected: float) -> float:
+    """Philox4x32-10 blocks one shuffle launch must draw: one per 4 coordinates for the mask and
+    ceil((N-1)/4) per selected coordinate for its permutation."""
+    return P / 4.0 + selected * ((N - 1 + 3) // 4)
+
+
+def sector_write_share(p_eff: float, N: int, E: int, layout: str) -> float:
+    """Share of a stack's 32-byte DRAM sectors that hold at least one moved value when every
+    coordinate is selected with probability p_eff (all N values of a selected coordinate are
+    counted as moved).  [N][P]: a sector holds 32/E neighbouring coordinates of one model;
+    [P][N]: a coordinate's N values lie side by side, a sector holds 32/(E N) coordinates (at
+    least part of one)."""
+    per_sector = 32.0 / E if layout == "[N][P]" else max(1.0, 32.0 / (E * N))
+    return 1.0 - (1.0 - p_eff) ** per_sector
+
+
+def measure_philox_rate(B, torch, stream) -> float:
+    """Philox blocks per second of a kernel that draws mask blocks and nothing else: the ceiling
+    the integer pipes put on any shuffle, measured in this run."""
+    chk = torch.zeros(1, dtype=torch.int32, device="cuda")
+    n_blocks = 1 << 28
+    for _ in range(3):
+        B.wash_philox_probe(n_blocks, SEED, chk, torch.cuda.current_device(), stream)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for _ in range(5):
+        B.wash_philox_probe(n_blocks, SEED, chk, torch.cuda.current_device(), stream)
+    e1.record(stream)
+    torch.cuda.synchronize()
+    return 5 * n_blocks / (e0.elapsed_time(e1) * 1e-3)
+
+
+def time_launches(torch, stream, launch, first_step: int, min_s: float = 0.06, blocks: int = 3, max_n: int = 2000):
+    """Median and minimum per-launch time (ms) of `launch(step)` issued back to back, two events
+    around each block of launches; the block length is chosen so that a block lasts min_s / blocks."""
+    for k in range(3):
+        launch(first_step + k)
+    torch.cuda.synchronize()
+    a0, a1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    a0.record(stream)
+    launch(first_step + 3)
+    a1.record(stream)
+    torch.cuda.synchronize()
+    est = max(a0.elapsed_time(a1) * 1e-3, 1e-6)
+    n = int(max(2, min(max_n, min_s / blocks / est)))
+    per = []
+    step = first_step + 4
+    for _ in range(blocks):
+        a0.record(stream)
+        for k in range(n):
+            launch(step + k)
+        a1.record(stream)
+        torch.cuda.synchronize()
+        per.append(a0.elapsed_time(a1) / n)
+        step += n
+    return float(np.median(per)), float(min(per)), n * blocks
+
+
+def shuffle_cell(B, torch, stream, pop, shuffle_fn, N, P, Es, p_eff, layout, peak, philox_rate, modes=("stream", "sparse")):
+    """Times one population's shuffle in the given modes and relates it to both ceilings:
+    t_HBM = bytes / measured copy bandwidth, t_ALU = Philox blocks / measured probe rate."""
+    stats = torch.zeros(2, dtype=torch.int64, device="cuda")
+    out = {}
+    E_sum = sum(Es)             # Es: element size of every stack the launch shuffles
+    for mode in modes:
+        B.wash_set_mode(pop.ctx, {"stream": B.WASH_MODE_STREAM, "sparse": B.WASH_MODE_SPARSE}[mode])
+        stats.zero_()
+        med, lo, n = time_launches(torch, stream, lambda i: shuffle_fn(i, stats), 100)
+        torch.cuda.synchronize()
+        sel = int(stats[0]) / (n + 4)          # time_launches issues 4 launches before its blocks
+        blocks = philox_blocks(P, N, sel)
+        t_alu = blocks / philox_rate
+        rec = {"ms": med, "ms_min": lo, "launches": n, "selected_per_launch": sel,
+               "param_swaps_per_s": sel * N / (med * 1e-3), "philox_blocks_per_launch": blocks,
+               "alu_frac": t_alu / (med * 1e-3)}
+        if mode == "stream":
+            algorithmic = N * P * E_sum + sel * N * E_sum                         # read everything, write the selected values
+            dram_model = sum(N * P * E * (1.0 + sector_write_share(p_eff, N, E, layout)) for E in Es)
+            t_hbm = algorithmic / (peak * 1e9)
+            t_hbm_sectors = dram_model / (peak * 1e9)
+            rec.update({"GBps": algorithmic / (med * 1e-3) / 1e9, "frac_of_hbm": t_hbm / (med * 1e-3),
+                        "dram_model_GBps": dram_model / (med * 1e-3) / 1e9, "hbm_frac_sector_model": t_hbm_sectors / (med * 1e-3),
+                        "bound": "alu" if t_alu > t_hbm_sectors else "hbm",
+                        "frac_of_bound": max(t_alu, t_hbm_sectors) / (med * 1e-3)})
+        else:
+            rec.update({"algorithmic_GBps": 2.0 * sel * N * E_sum / (med * 1e-3) / 1e9, "bound": "alu"})
+        out[mode] = rec
+    B.wash_set_mode(pop.ctx, B.WASH_MODE_STREAM)
+    return out
+
+
+def configs_record(B, torch, stream, peak, philox_rate, main_name, main_cell) -> dict:
+    """The other configurations, timed in the same run: configs 1-4 (device-generated values of
+    the configs' shapes: the shuffle's time does not depend on the values) and the cells
+    N in {2, 8, 32} x P = 2^27 x p in {1e-3, 1e-2, 1e-1} x both layouts of config 5."""
+    rec = {"note": "shuffle only, launched back to back (median of 3 blocks); frac_of_hbm = algorithmic bytes (read all + write "
+                   "selected values) / time / measured copy bandwidth; hbm_frac_sector_model counts writes in whole 32-byte sectors; "
+                   "alu_frac = Philox blocks per second / the probe's rate; bound = the larger of the two times",
+           "philox_probe_blocks_per_s": philox_rate}
+    for name in ("cfg1_flat_n3", "cfg2_resnet18_n5", "cfg3_resnet50_n10", "cfg4_resnet50_bf16_n8"):
+        if name == main_name:
+            rec[name] = main_cell
+            continue
+        wl = Workload(name)
+        pop = B.Population(wl.N, wl.numel, B.WASH_LAYOUT_NP, torch.cuda.current_device(), wl.tensor_id)
+        gen = torch.Generator(device="cuda").manual_seed(SEED)
+        params = (torch.randn(wl.N * pop.padded_P, generator=gen, device="cuda") * 0.05).to(torch.bfloat16 if wl.bf16 else torch.float32)
+        pop.bind(B.WASH_STACK_PARAMS, params)
+        opt = None
+        if wl.opt:
+            opt = torch.randn(wl.N * pop.padded_P, generator=gen, device="cuda") * 1e-3
+            pop.bind(B.WASH_STACK_OPT, opt)
+        p_layer = B.wash_layer_probs(wl.T, wl.p, B.WASH_SCHEDULE_DECREASING) if wl.schedule == "decreasing" else None
+        fn = (lambda i, st: B.wash_shuffle_both(pop.ctx, i, wl.p, p_layer, SEED, stream, st)) if wl.opt else \
+             (lambda i, st: B.wash_shuffle(pop.ctx, i, wl.p, p_layer, SEED, stream, st))
+        p_eff = wl.p if p_layer is None else float((p_layer * wl.numel).sum() / wl.P)
+        cell = shuffle_cell(B, torch, stream, pop, fn, wl.N, wl.P, wl.Es, p_eff, "[N][P]", peak, philox_rate)
+        cell["footprint_bytes"] = wl.N * pop.padded_P * (wl.E + wl.E_opt)
+        cell["l2"] = "beyond L2" if cell["footprint_bytes"] > 2.5e8 else "L2-resident"
+        rec[name] = cell
+        B.wash_check(pop.ctx)
+        pop.close()
+        del params, opt
+        torch.cuda.empty_cache()
+    cells = []
+    P = 1 << 27
+    for N in (2, 8, 32):
+        for layout, lname in ((B.WASH_LAYOUT_NP, "[N][P]"), (B.WASH_LAYOUT_PN, "[P][N]")):
+            pop = B.Population(N, [P], layout, torch.cuda.current_device())
+            gen = torch.Generator(device="cuda").manual_seed(N)
+            stack = torch.empty(N * pop.padded_P, device="cuda", dtype=torch.float32)
+            for lo in range(0, stack.numel(), 1 << 28):
+                stack[lo:lo + (1 << 28)].normal_(0.0, 0.05, generator=gen)
+            pop.bind(B.WASH_STACK_PARAMS, stack)
+            for p in (1e-3, 1e-2, 1e-1):
+                fn = lambda i, st, p=p: B.wash_shuffle(pop.ctx, i, p, None, SEED, stream, st)
+                cell = shuffle_cell(B, torch, stream, pop, fn, N, P, (4,), p, lname, peak, philox_rate)
+                cell.update({"N": N, "P": P, "p": p, "layout": lname})
+                cells.append(cell)
+            B.wash_check(pop.ctx)
+            pop.close()
+            del stack
+            torch.cuda.empty_cache()
+    rec["cfg5_cells"] = cells
+    return rec
+
+
 def run_ours(args, rank: int, world: int, local_rank: int) -> None:
     import torch
     from paper_2405_17517_b200 import binding as B
@@ -244,6 +408,7 @@ def run_ours(args, rank: int, world: int, local_rank: int) -> None:
 
     params_pin = to_torch(params_h).pin_memory()
     opt_pin = to_torch(opt_h).pin_memory() if opt_h is not None else None
+    del params_h, opt_h
     params_d = params_pin.cuda(non_blocking=True)
     opt_d = opt_pin.cuda(non_blocking=True) if opt_pin is not None else None
     avg_d = torch.zeros(pop.padded_P, dtype=params_d.dtype, device="cuda")
@@ -252,34 +417,33 @@ def run_ours(args, rank: int, world: int, local_rank: int) -> None:
     pop.bind(B.WASH_STACK_PARAMS, params_d)
     if opt_d is not None:
         pop.bind(B.WASH_STACK_OPT, opt_d)
-    if args.mode != "stream":
-        B.wash_set_mode(pop.ctx, {"sparse": B.WASH_MODE_SPARSE, "staged": B.WASH_MODE_STREAM_STAGED, "registers": B.WASH_MODE_STREAM_REGISTERS}[args.mode])
+    mode_code = {"stream": B.WASH_MODE_STREAM, "sparse": B.WASH_MODE_SPARSE, "auto": B.WASH_MODE_AUTO}[args.mode]
+    B.wash_set_mode(pop.ctx, mode_code)
     if args.threads or args.blocks_per_sm:
         B.wash_set_launch(pop.ctx, args.threads, args.blocks_per_sm)
     pdt = B.WASH_BF16 if wl.bf16 else B.WASH_F32
     if wl.schedule == "decreasing":
         wl.p_layer = B.wash_layer_probs(wl.T, wl.p, B.WASH_SCHEDULE_DECREASING)
     p_layer = wl.p_layer
+    p_eff = wl.p if p_layer is None else float((p_layer * wl.numel).sum() / wl.P)
     stream = torch.cuda.current_stream()
 
-    def step_shuffle(i):
+    def step_shuffle(i, st=stats_d):
         if opt_d is not None:
-            B.wash_shuffle_both(pop.ctx, i, wl.p, p_layer, SEED, stream, stats_d)
+            B.wash_shuffle_both(pop.ctx, i, wl.p, p_layer, SEED, stream, st)
         else:
-            B.wash_shuffle(pop.ctx, i, wl.p, p_layer, SEED, stream, stats_d)
+            B.wash_shuffle(pop.ctx, i, wl.p, p_layer, SEED, stream, st)
 
-    def step(i, ev=None):
-        if ev is not None:
-            ev[0].record(stream)
+    def step(i, ev):
+        """One pass of the hot path: shuffle of both stacks, PAPA's EMA, the average; an event
+        before and after each kernel, on the launching stream."""
+        ev[0].record(stream)
         step_shuffle(i)
-        if ev is not None:
-            ev[1].record(stream)
+        ev[1].record(stream)
         B.papa_ema(pop.ctx, B.WASH_STACK_PARAMS, ALPHA, stream)
-        if ev is not None:
-            ev[2].record(stream)
+        ev[2].record(stream)
         B.population_average(pop.ctx, B.WASH_STACK_PARAMS, avg_d, pdt, stream)
-        if ev is not None:
-            ev[3].record(stream)
+        ev[3].record(stream)
 
     def fence():
         torch.cuda.synchronize()
@@ -287,141 +451,152 @@ def run_ours(args, rank: int, world: int, local_rank: int) -> None:
             dist.barrier()
             torch.cuda.synchronize()
 
+    K = args.steps
+    events = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(K)]
     for w in range(args.warmup):
-        step(w)
+        step(w, events[0])
     fence()
     stats_d.zero_()
     launches0 = B.wash_launch_count()
-    events = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(args.steps)]
     sampler = ClockSampler(physical_gpu_index(local_rank))
     sampler.start()
-    fence()
+
+    # ---- timed blocks of exactly K steps each, repeated until MIN_TIMED_S of GPU time --------
     t_begin = torch.cuda.Event(enable_timing=True)
     t_end = torch.cuda.Event(enable_timing=True)
-    t_begin.record(stream)
-    for k in range(args.steps):
-        step(args.warmup + k, events[k] if args.inline_kernel_events else None)
-    t_end.record(stream)
-    fence()
+    block_ms, kernel_ms = [], []          # per block: total time (max over ranks), mean time of each kernel
+    next_step = args.warmup
+    repeats_wanted = 1
+    while len(block_ms) < repeats_wanted:
+        fence()
+        t_begin.record(stream)
+        for k in range(K):
+            step(next_step + k, events[k])
+        t_end.record(stream)
+        fence()
+        next_step += K
+        total = t_begin.elapsed_time(t_end)
+        per_kernel = np.array([[e[i].elapsed_time(e[i + 1]) for i in range(3)] for e in events]).mean(axis=0)
+        if dist is not None:
+            t = torch.tensor([total] + per_kernel.tolist(), dtype=torch.float64, device="cuda")
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            total, per_kernel = float(t[0]), t[1:].cpu().numpy()
+        block_ms.append(total)
+        kernel_ms.append(per_kernel)
+        if len(block_ms) == 1:       # the same count on every rank: derived from the all-reduced first block
+            repeats_wanted = int(min(MAX_REPEATS, max(1, np.ceil(MIN_TIMED_S * 1e3 / max(total, 1e-3)))))
     clocks = sampler.stop()
     launches = B.wash_launch_count() - launches0
     B.wash_check(pop.ctx)
-    total_ms = t_begin.elapsed_time(t_end)
+    repeats = len(block_ms)
     st = stats_d.cpu().numpy().view(np.uint64)
     selected_total, moved_total = int(st[0]), int(st[1])
-    if not args.inline_kernel_events:
-        # Per-kernel times come from a second, instrumented pass over the same steps' work:
-        # an event between every two launches costs the step about 5 % (measured), so the
-        # timed region above carries none.
-        fence()
-        for k in range(min(args.steps, 300)):
-            step(args.warmup + args.steps + k, events[k])
-        fence()
-        events = events[:min(args.steps, 300)]
-    k_ms = np.array([[e[i].elapsed_time(e[i + 1]) for i in range(3)] for e in events])   # shuffle, ema, average
-    mean_ms = k_ms.mean(axis=0)
+    steps_timed = K * repeats
+    block_ms = np.array(block_ms)
+    kernel_ms = np.array(kernel_ms)
+    med_ms = np.median(kernel_ms, axis=0)          # shuffle, ema, average
+    min_ms = kernel_ms.min(axis=0)
+    step_ms = float(np.median(block_ms)) / K
+    step_ms_min = float(block_ms.min()) / K
 
-    # ---- the shuffle alone, launched back to back (no event between launches), in the
-    # streaming mode and in the sparse mode: context for the per-kernel figures above, which
-    # carry an event pair per launch, and the parameter-swaps/s the sparse kernel reaches
-    def shuffle_alone(mode, n):
-        B.wash_set_mode(pop.ctx, mode)
-        first = args.warmup + 2 * args.steps + 1000
-        for k in range(3):
-            step_shuffle(first + k)
-        fence()
-        a0 = torch.cuda.Event(enable_timing=True)
-        a1 = torch.cuda.Event(enable_timing=True)
-        a0.record(stream)
-        for k in range(n):
-            step_shuffle(first + 3 + k)
-        a1.record(stream)
-        fence()
-        return a0.elapsed_time(a1) / n
-
-    alone_ms = None
-    if args.mode == "stream":
-        n_alone = max(1, min(args.steps, 300))
-        alone_ms = [shuffle_alone(B.WASH_MODE_STREAM, n_alone), shuffle_alone(B.WASH_MODE_SPARSE, n_alone)]
-        B.wash_set_mode(pop.ctx, B.WASH_MODE_STREAM)
+    # ---- the shuffle alone, launched back to back, in the streaming and the sparse mode, with
+    # both ceilings (world == 1; with several ranks only the streaming time is taken)
+    peak, peak_src = measured_peak()
+    philox_rate = measure_philox_rate(B, torch, stream)
+    fence()
+    main_cell = shuffle_cell(B, torch, stream, pop, lambda i, st_: step_shuffle(i, st_), wl.N, wl.P, wl.Es, p_eff,
+                             "[N][P]", peak, philox_rate)
+    B.wash_set_mode(pop.ctx, mode_code)
+    fence()
 
     # ---- end to end through the host-buffer entry point --------------------------------
-    e2e_steps = max(1, min(args.steps, 5))
-    ops = B.WASH_OP_SHUFFLE | B.WASH_OP_EMA | B.WASH_OP_AVERAGE
-    B.wash_step_host(pop.ctx, ops, params_pin, opt_pin, avg_pin, 0, wl.p, p_layer, SEED, ALPHA, stream)   # warm
-    fence()
-    e0 = torch.cuda.Event(enable_timing=True)
-    e1 = torch.cuda.Event(enable_timing=True)
-    e0.record(stream)
-    for k in range(e2e_steps):
-        B.wash_step_host(pop.ctx, ops, params_pin, opt_pin, avg_pin, 1 + k, wl.p, p_layer, SEED, ALPHA, stream)
-    e1.record(stream)
-    fence()
-    e2e_ms = e0.elapsed_time(e1)
+    # The headline metric (the shuffle) through wash_step_host with the stacks in pinned host
+    # memory: copy in, shuffle, copy out, every step, inside the timed region; then the same
+    # with the whole step (shuffle + EMA + average).
+    e2e_steps = max(1, min(K, 5))
+
+    def host_steps(ops, first):
+        B.wash_step_host(pop.ctx, ops, params_pin, opt_pin, avg_pin, first, wl.p, p_layer, SEED, ALPHA, stream)   # warm
+        fence()
+        e0 = torch.cuda.Event(enable_timing=True)
+        e1 = torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        sel = 0
+        for k in range(e2e_steps):
+            sel += B.wash_step_host(pop.ctx, ops, params_pin, opt_pin, avg_pin, first + 1 + k, wl.p, p_layer, SEED, ALPHA, stream)[0]
+        e1.record(stream)
+        fence()
+        return e0.elapsed_time(e1), sel
+
+    e2e_ms, sel_e2e = host_steps(B.WASH_OP_SHUFFLE, 0)
+    e2e_full_ms, _ = host_steps(B.WASH_OP_SHUFFLE | B.WASH_OP_EMA | B.WASH_OP_AVERAGE, 100)
     stack_bytes = params_pin.numel() * params_pin.element_size() + (opt_pin.numel() * opt_pin.element_size() if opt_pin is not None else 0)
     h2d = stack_bytes
-    d2h = stack_bytes + avg_pin.numel() * avg_pin.element_size() + 16
+    d2h = stack_bytes + 16
+    d2h_full = stack_bytes + avg_pin.numel() * avg_pin.element_size() + 16
 
-    # ---- max over ranks ------------------------------------------------------------------
+    # ---- max / sum over ranks ----------------------------------------------------------------
     if dist is not None:
-        t = torch.tensor([total_ms, e2e_ms, mean_ms[0], mean_ms[1], mean_ms[2]] + (alone_ms or [0.0, 0.0]), dtype=torch.float64, device="cuda")
+        t = torch.tensor([e2e_ms, e2e_full_ms], dtype=torch.float64, device="cuda")
         dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms, e2e_ms = float(t[0]), float(t[1])
-        mean_ms = t[2:5].cpu().numpy()
-        if alone_ms is not None:
-            alone_ms = [float(t[5]), float(t[6])]
-        c = torch.tensor([selected_total, moved_total], dtype=torch.int64, device="cuda")
+        e2e_ms, e2e_full_ms = float(t[0]), float(t[1])
+        c = torch.tensor([selected_total, moved_total, sel_e2e], dtype=torch.int64, device="cuda")
         dist.all_reduce(c, op=dist.ReduceOp.SUM)
-        selected_total, moved_total = int(c[0]), int(c[1])
+        selected_total, moved_total, sel_e2e = int(c[0]), int(c[1]), int(c[2])
 
     if rank == 0:
-        sel_per_step_rank = selected_total / args.steps / world
+        sel_per_step_rank = selected_total / steps_timed / world
         ab = wl.algorithmic_bytes(sel_per_step_rank)
-        step_ms = total_ms / args.steps
-        value = ab["step"] * world / (step_ms * 1e-3) / 1e9
-        peak, peak_src = measured_peak()
-        shuffle_gbs = ab["shuffle"] / (mean_ms[0] * 1e-3) / 1e9
+        shuffle_gbs = ab["shuffle"] / (med_ms[0] * 1e-3) / 1e9          # one rank's kernel
+        blocks_launch = philox_blocks(wl.P, wl.N, sel_per_step_rank)
+        traffic = TRAFFIC.get((wl.name, args.mode), {})
         line = {
-            "metric": METRIC, "value": value, "unit": "GB/s", "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+            "metric": METRIC, "value": shuffle_gbs * world, "unit": "GB/s", "n_gpus": world, "steps": K, "warmup": args.warmup,
             "ms_per_step": step_ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "bf16+f32" if wl.bf16 else "f32", "data": "synthetic",
-            "value_definition": "bytes the three kernels of one step must stream (shuffle: read both stacks + write selected; "
-                                "EMA: read+write parameters; average: read parameters + write one row) / step time, all ranks",
+            "value_definition": "the shuffle's own throughput: bytes the shuffle of both stacks must move (read every value, write the "
+                                "selected ones) / the shuffle kernel's time inside the step (CUDA events on the launching stream, median "
+                                "over the timed blocks of the per-block mean, max over ranks), summed over ranks; ms_per_step is the whole "
+                                "step (shuffle + EMA + average)",
+            "repeats": repeats, "steps_timed": steps_timed, "timed_gpu_s": float(block_ms.sum()) * 1e-3,
+            "ms_per_step_min": step_ms_min,
             "config": {"workload": wl.name, "N": wl.N, "tensors": wl.T, "P": wl.P, "p": wl.p,
                        "per_layer_p": wl.p_layer is not None, "opt_state": wl.opt, "layout": "[N][P]", "mode": args.mode,
                        "footprint_bytes_per_gpu": stack_bytes, "l2": "inputs larger than L2 (no flush)" if stack_bytes > 2.5e8 else "L2-resident: footprint below 2x L2",
                        "sharding": "one population shard per rank, no collective"},
-            "param_swaps_per_s": selected_total * wl.N / (total_ms * 1e-3),
-            "moved_values_per_s": moved_total / (total_ms * 1e-3),
-            "selected_coords_per_step": selected_total / args.steps,
-            "kernel_times": "CUDA events on the launching stream, " + ("inside the timed region" if args.inline_kernel_events
-                                                                      else "instrumented pass of %d steps right after the timed region" % min(args.steps, 300)),
+            "param_swaps_per_s": sel_per_step_rank * wl.N * world / (med_ms[0] * 1e-3),
+            "moved_values_per_s": moved_total / steps_timed / (med_ms[0] * 1e-3),
+            "selected_coords_per_step": selected_total / steps_timed,
+            "step": {"kernels": "wash_shuffle_both + papa_ema + population_average" if wl.opt else "wash_shuffle + papa_ema + population_average",
+                     "ms": step_ms, "ms_min": step_ms_min, "GBps": ab["step"] * world / (step_ms * 1e-3) / 1e9,
+                     "bytes": "shuffle: read both stacks + write selected; EMA: read + write parameters; average: read parameters + write one row"},
+            "kernel_times": "CUDA events on the launching stream around every kernel, inside the timed blocks; median (and min) over %d blocks of the mean over the block's %d steps" % (repeats, K),
             "kernels": {
-                "shuffle": {"ms": float(mean_ms[0]), "GBps": shuffle_gbs, "frac_of_hbm": shuffle_gbs / peak},
-                "papa_ema": {"ms": float(mean_ms[1]), "GBps": ab["ema"] / (mean_ms[1] * 1e-3) / 1e9},
-                "population_average": {"ms": float(mean_ms[2]), "GBps": ab["average"] / (mean_ms[2] * 1e-3) / 1e9},
+                "shuffle": {"ms": float(med_ms[0]), "ms_min": float(min_ms[0]), "GBps": shuffle_gbs, "frac_of_hbm": shuffle_gbs / peak},
+                "papa_ema": {"ms": float(med_ms[1]), "ms_min": float(min_ms[1]), "GBps": ab["ema"] / (med_ms[1] * 1e-3) / 1e9,
+                             "frac_of_hbm": ab["ema"] / (med_ms[1] * 1e-3) / 1e9 / peak},
+                "population_average": {"ms": float(med_ms[2]), "ms_min": float(min_ms[2]), "GBps": ab["average"] / (med_ms[2] * 1e-3) / 1e9,
+                                       "frac_of_hbm": ab["average"] / (med_ms[2] * 1e-3) / 1e9 / peak},
             },
             "roofline": {"kernel": "shuffle kernel, mode %s (params + momentum)" % args.mode, "bound": "hbm", "achieved": shuffle_gbs,
                          "peak": peak, "peak_source": peak_src, "unit": "GB/s", "frac": shuffle_gbs / peak,
-                         "traffic": TRAFFIC.get(wl.name, {}).get("dram_bytes") if args.mode == "stream" else None,
-                         "traffic_source": TRAFFIC.get(wl.name, {}).get("source") if args.mode == "stream" else None},
-            "e2e": {"value": ab["step"] * world / (e2e_ms / e2e_steps * 1e-3) / 1e9, "unit": "GB/s",
-                    "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": e2e_steps,
-                    "api": "wash_step_host (pinned host stacks)"},
+                         "alu_frac": blocks_launch / philox_rate / (med_ms[0] * 1e-3),
+                         "alu_peak_philox_blocks_per_s": philox_rate,
+                         "traffic": traffic.get("dram_bytes"), "traffic_source": traffic.get("source")},
+            "e2e": {"value": wl.algorithmic_bytes(sel_e2e / e2e_steps / world)["shuffle"] * world / (e2e_ms / e2e_steps * 1e-3) / 1e9, "unit": "GB/s",
+                    "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": e2e_steps, "ms_per_step": e2e_ms / e2e_steps,
+                    "api": "wash_step_host(WASH_OP_SHUFFLE) on pinned host stacks: copy in, shuffle, copy out inside the timed region",
+                    "full_step": {"ms_per_step": e2e_full_ms / e2e_steps, "d2h_bytes_per_step": d2h_full,
+                                  "GBps": ab["step"] * world / (e2e_full_ms / e2e_steps * 1e-3) / 1e9,
+                                  "api": "wash_step_host with shuffle + EMA + average"}},
             "gpu_launches": int(launches),
             "clocks": clocks,
+            "shuffle_back_to_back": main_cell,
         }
-        if alone_ms is not None:
-            sel_step = selected_total / args.steps
-            line["shuffle_back_to_back"] = {
-                "launches": max(1, min(args.steps, 300)),
-                "stream": {"ms": alone_ms[0], "GBps": ab["shuffle"] / (alone_ms[0] * 1e-3) / 1e9,
-                           "frac_of_hbm": ab["shuffle"] / (alone_ms[0] * 1e-3) / 1e9 / peak,
-                           "param_swaps_per_s": sel_step * wl.N / (alone_ms[0] * 1e-3)},
-                "sparse": {"ms": alone_ms[1], "param_swaps_per_s": sel_step * wl.N / (alone_ms[1] * 1e-3),
-                           "bound": "integer pipes (one Philox block per 4 coordinates), not HBM"},
-                "note": "the step's shuffle launched alone, two events around the whole series; WASH_MODE_AUTO picks the sparse kernel below 3 % expected selection",
-            }
+        if clocks.get("sm_mhz"):
+            line["roofline"]["ms_x_sm_mhz"] = float(med_ms[0]) * clocks["sm_mhz"]
+        if world == 1 and not args.no_configs:
+            line["configs"] = configs_record(B, torch, stream, peak, philox_rate, wl.name, main_cell)
         if world == 1 and not args.no_cpu_baseline:
             line["cpu_baseline"] = cpu_baseline(wl)
         print(json.dumps(line), flush=True)
@@ -431,12 +606,10 @@ def run_ours(args, rank: int, world: int, local_rank: int) -> None:
         dist.destroy_process_group()
 
 
-# DRAM bytes per shuffle launch from the ncu capture summarised under profiles/ (None
-# until a capture of the current kernel exists).
+# DRAM bytes per shuffle launch (dram__bytes_read.sum + dram__bytes_write.sum of one ncu capture
+# of the kernel as it stands, summarised under profiles/), per (workload, mode).  A workload
+# without a capture of the current kernel has no entry and the bench line says null.
 TRAFFIC = {
-    # shuffle_async_kernel<F32, F32, [N][P], 1>: 448.9 MB read + 5.9 MB written per launch
-    "cfg2_resnet18_n5": {"dram_bytes": 448.9e6 + 5.9e6,
-                         "source": "profiles/shuffle_async_kernel_cfg2_resnet18_n5.md"},
 }
 
 
@@ -450,18 +623,22 @@ def cpu_baseline(wl: Workload) -> dict:
     threads = oracle.max_threads()
     oracle.set_threads(threads)
     p = wl.p if wl.schedule is None else oracle.layer_probs(wl.T, wl.p, oracle.SCHEDULE_DECREASING)
-    steps, sel, t0 = 0, 0, time.perf_counter()
+    steps, sel, t_shuffle, t0 = 0, 0, 0.0, time.perf_counter()
     while True:
+        t1 = time.perf_counter()
         sel += oracle.shuffle(pop, params, p, seed=SEED, step=steps, stack2=opt)[0]
+        t_shuffle += time.perf_counter() - t1
         oracle.papa_ema(pop, params, ALPHA)
         oracle.population_average(pop, params, out)
         steps += 1
         dt = time.perf_counter() - t0
         if dt > 10.0 or steps >= 2000:
             break
-    gbs = wl.algorithmic_bytes(sel / steps)["step"] * steps / dt / 1e9
-    return {"value": gbs, "unit": "GB/s", "cores": threads, "kind": "oracle",
-            "sample": "%d full steps of the same workload (%.1f s)" % (steps, dt), "ms_per_step": dt / steps * 1e3}
+    ab = wl.algorithmic_bytes(sel / steps)
+    return {"value": ab["shuffle"] * steps / t_shuffle / 1e9, "unit": "GB/s", "cores": threads, "kind": "oracle",
+            "sample": "%d full steps of the same workload (%.1f s); value = the shuffle's bytes / the time inside the oracle's shuffle" % (steps, dt),
+            "ms_per_step": dt / steps * 1e3, "step_GBps": ab["step"] * steps / dt / 1e9,
+            "param_swaps_per_s": sel * wl.N / t_shuffle}
 
 
 def run_sweep(args) -> None:
@@ -604,16 +781,15 @@ def run_exchange(args) -> None:
 def main() -> None:
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=2000)
+    ap.add_argument("--steps", type=int, default=100)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="cfg2_resnet18_n5", choices=sorted(W.CONFIGS))
-    ap.add_argument("--mode", default="stream", choices=["stream", "sparse", "staged", "registers"])
+    ap.add_argument("--workload", default="cfg3_resnet50_n10", choices=sorted(W.CONFIGS))
+    ap.add_argument("--mode", default="stream", choices=["stream", "sparse", "auto"])
     ap.add_argument("--threads", type=int, default=0)
     ap.add_argument("--blocks-per-sm", type=int, default=0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--inline-kernel-events", action="store_true",
-                    help="record the per-kernel events inside the timed region instead of in a second pass")
+    ap.add_argument("--no-configs", action="store_true", help="skip the record of the other configurations (configs 1-4, cells of config 5)")
     ap.add_argument("--sweep", action="store_true", help="config-5 sweep of the shuffle kernel (many JSON lines)")
     ap.add_argument("--sweep-modes", default="stream,sparse")
     ap.add_argument("--sweep-N", default="", help="comma list; default 2,4,8,16,32")

@@ -301,7 +301,7 @@ int wash_exchange_counts(wash_ctx *ctx, uint64_t *host_need, uint64_t *host_sele
  * wash_create puts the context's lookup tables in device memory with cudaMalloc.  Two
  * kinds of caller cannot afford that: a process in which a framework's memory pool has
  * already taken the whole GPU (an allocation from this library would fail or compete
- * with the pool), and a latency-critical loop in which cudaMalloc / cudaFree, which
+ * with the pool), and a loop in which cudaMalloc / cudaFree, which
  * synchronise the whole device, would stall work that other streams have in flight.
  * wash_shuffle_noalloc runs the same streaming shuffle as wash_shuffle on ONE stack
  * without any context and without allocating device or pinned memory: its tables live
@@ -330,7 +330,15 @@ int wash_exchange_counts(wash_ctx *ctx, uint64_t *host_need, uint64_t *host_sele
  *
  * First use: the first call on each device looks up that device's address of the array
  * (cudaGetSymbolAddress, with the device made current for the duration of the call).
- * Make that first call before any stream capture begins. */
+ * Make that first call before any stream capture begins.
+ *
+ * Every call uploads its two tables (up to 288 KiB) with two host-to-device copies from
+ * ordinary pageable host memory, ordered on `stream`; the host arrays are freed when the
+ * call returns, so a stream that is in capture mode is refused with WASH_ERR_STATE.
+ *
+ * Device-side checks: the kernel is given no status word, so a group that falls outside
+ * the tables (which this call builds itself from numel) would be skipped without a report;
+ * there is no wash_check for this entry point. */
 int wash_shuffle_noalloc(int32_t N, int32_t n_tensors, const int64_t *numel, int32_t layout,
                          int32_t dtype, void *dev_stack, int64_t n_elems, uint64_t step, double p,
                          const double *p_layer, uint64_t seed, int32_t device, void *stream,

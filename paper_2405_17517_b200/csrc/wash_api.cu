@@ -106,6 +106,7 @@ struct wash_ctx {
     int64_t x_capacity[2][2] = {{0, 0}, {0, 0}};
     void *x_own[2][2] = {{nullptr, nullptr}, {nullptr, nullptr}};        // staging buffers this library allocated
     std::vector<void *> x_opened;          // peers' buffers mapped by wash_exchange_staging_open
+    bool x_opened_set[2][2] = {{false, false}, {false, false}};   // [parity][stack]: that set's peers are mapped
     bool x_planned = false;
     uint64_t x_step = 0, x_seed = 0;
 };
@@ -165,17 +166,22 @@ uint64_t threshold_of(double p) { return static_cast<uint64_t>(std::floor(p * 42
 // probabilities (uploaded, in stream order, only when they changed).
 int sync_table(wash_ctx *ctx, double p, const double *p_layer, cudaStream_t stream)
 {
-    bool changed = !ctx->seg_uploaded;
+    // every probability is checked before the first threshold of the host mirror changes: a
+    // rejected call must leave the mirror equal to the device table
     for (int s = 0; s < ctx->n_seg; ++s) {
         const double ps = p_layer ? p_layer[s] : p;
         if (!(ps >= 0.0 && ps <= 1.0)) return fail(WASH_ERR_ARG, "probability of tensor %d is %g, not in [0,1]", s, ps);
-        const uint64_t thr = threshold_of(ps);
+    }
+    bool changed = !ctx->seg_uploaded;
+    for (int s = 0; s < ctx->n_seg; ++s) {
+        const uint64_t thr = threshold_of(p_layer ? p_layer[s] : p);
         if (thr != ctx->seg_host[s].thr) {
             ctx->seg_host[s].thr = thr;
             changed = true;
         }
     }
     if (!changed) return WASH_OK;
+    ctx->seg_uploaded = false;   // until the copy below is queued, the mirror is ahead of the device table
     ctx->expected_selected = 0.0;
     for (int s = 0; s < ctx->n_seg; ++s)
         ctx->expected_selected += static_cast<double>(ctx->seg_host[s].numel) * static_cast<double>(ctx->seg_host[s].thr) / 4294967296.0;
@@ -547,69 +553,84 @@ int wash_step_host(wash_ctx *ctx, int32_t ops, void *host_params, void *host_opt
             for (cudaEvent_t &e : ctx->pipe_event)
                 if ((err = cudaEventCreateWithFlags(&e, cudaEventDisableTiming)) != cudaSuccess) return cuda_fail(err, "cudaEventCreate");
         }
-        cudaEvent_t *ev_in = ctx->pipe_event, *ev_done = ctx->pipe_event + kPipeChunks;
-        cudaEvent_t ev_start = ctx->pipe_event[2 * kPipeChunks], ev_out = ctx->pipe_event[2 * kPipeChunks + 1];
-        if ((ops & WASH_OP_SHUFFLE) && (err = cudaMemsetAsync(ctx->stats_dev, 0, sizeof(wash_stats), stream)) != cudaSuccess) return cuda_fail(err, "cudaMemsetAsync(stats)");
-        if ((ops & WASH_OP_AVERAGE) && (err = cudaMemsetAsync(ctx->avg_dev, 0, avg_bytes, stream)) != cudaSuccess) return cuda_fail(err, "cudaMemsetAsync(average row)");
-        // the copy streams start after whatever the caller's stream has queued so far
-        if ((err = cudaEventRecord(ev_start, stream)) != cudaSuccess ||
-            (err = cudaStreamWaitEvent(ctx->copy_in, ev_start, 0)) != cudaSuccess ||
-            (err = cudaStreamWaitEvent(ctx->copy_out, ev_start, 0)) != cudaSuccess) return cuda_fail(err, "pipeline set-up");
-        const uint32_t per = ((ctx->n_groups + kPipeChunks - 1) / kPipeChunks + 255u) & ~255u;   // groups per range
-        // moves the elements [e0, e0 + count) of every model between a host and the device stack
-        auto copy_range = [&](void *dst, const void *src, int dtype, size_t e0, size_t count, cudaMemcpyKind kind, cudaStream_t s) {
-            const size_t eb = elem_bytes(dtype);
-            if (ctx->layout == WASH_LAYOUT_NP) {
-                const size_t pitch = static_cast<size_t>(ctx->padded_P) * eb;
-                return cudaMemcpy2DAsync(static_cast<char *>(dst) + e0 * eb, pitch, static_cast<const char *>(src) + e0 * eb, pitch,
-                                         count * eb, static_cast<size_t>(ctx->N), kind, s);
+        // Once a copy is queued on the side streams, an error must not leave them running into the
+        // caller's host buffers: the pipeline runs inside a lambda and every exit waits for all
+        // three streams (their own status is ignored then; the first error is what is returned).
+        auto pipeline = [&]() -> int {
+            cudaEvent_t *ev_in = ctx->pipe_event, *ev_done = ctx->pipe_event + kPipeChunks;
+            cudaEvent_t ev_start = ctx->pipe_event[2 * kPipeChunks], ev_out = ctx->pipe_event[2 * kPipeChunks + 1];
+            if ((ops & WASH_OP_SHUFFLE) && (err = cudaMemsetAsync(ctx->stats_dev, 0, sizeof(wash_stats), stream)) != cudaSuccess) return cuda_fail(err, "cudaMemsetAsync(stats)");
+            if ((ops & WASH_OP_AVERAGE) && (err = cudaMemsetAsync(ctx->avg_dev, 0, avg_bytes, stream)) != cudaSuccess) return cuda_fail(err, "cudaMemsetAsync(average row)");
+            // the copy streams start after whatever the caller's stream has queued so far
+            if ((err = cudaEventRecord(ev_start, stream)) != cudaSuccess ||
+                (err = cudaStreamWaitEvent(ctx->copy_in, ev_start, 0)) != cudaSuccess ||
+                (err = cudaStreamWaitEvent(ctx->copy_out, ev_start, 0)) != cudaSuccess) return cuda_fail(err, "pipeline set-up");
+            const uint32_t per = ((ctx->n_groups + kPipeChunks - 1) / kPipeChunks + 255u) & ~255u;   // groups per range
+            // moves the elements [e0, e0 + count) of every model between a host and the device stack
+            auto copy_range = [&](void *dst, const void *src, int dtype, size_t e0, size_t count, cudaMemcpyKind kind, cudaStream_t s) {
+                const size_t eb = elem_bytes(dtype);
+                if (ctx->layout == WASH_LAYOUT_NP) {
+                    const size_t pitch = static_cast<size_t>(ctx->padded_P) * eb;
+                    return cudaMemcpy2DAsync(static_cast<char *>(dst) + e0 * eb, pitch, static_cast<const char *>(src) + e0 * eb, pitch,
+                                             count * eb, static_cast<size_t>(ctx->N), kind, s);
+                }
+                const size_t off = e0 * ctx->N * eb;
+                return cudaMemcpyAsync(static_cast<char *>(dst) + off, static_cast<const char *>(src) + off, count * ctx->N * eb, kind, s);
+            };
+            const int od = ctx->stack_dtype[WASH_STACK_OPT];
+            for (int k = 0; k < kPipeChunks; ++k) {
+                const uint32_t g0 = static_cast<uint32_t>(k) * per;
+                if (g0 >= ctx->n_groups) break;
+                const uint32_t g1 = g0 + per < ctx->n_groups ? g0 + per : ctx->n_groups;
+                const size_t e0 = 4ull * g0, count = 4ull * (g1 - g0);
+                if ((err = copy_range(ctx->stack_ptr[WASH_STACK_PARAMS], host_params, pd, e0, count, cudaMemcpyHostToDevice, ctx->copy_in)) != cudaSuccess)
+                    return cuda_fail(err, "copy of a parameter range to the device");
+                if (host_opt && (err = copy_range(ctx->stack_ptr[WASH_STACK_OPT], host_opt, od, e0, count, cudaMemcpyHostToDevice, ctx->copy_in)) != cudaSuccess)
+                    return cuda_fail(err, "copy of an optimizer-state range to the device");
+                if ((err = cudaEventRecord(ev_in[k], ctx->copy_in)) != cudaSuccess || (err = cudaStreamWaitEvent(stream, ev_in[k], 0)) != cudaSuccess)
+                    return cuda_fail(err, "pipeline event");
+                if (ops & WASH_OP_SHUFFLE) {
+                    rc = shuffle_impl(ctx, host_opt ? 2 : 0, step, p, p_layer, seed, stream, ctx->stats_dev, g0, g1);
+                    if (rc != WASH_OK) return rc;
+                }
+                if (ops & WASH_OP_EMA) {
+                    rc = reduce_impl(ctx, wash::kOpEma, WASH_STACK_PARAMS, nullptr, WASH_F32, alpha, 0, ctx->n_seg, nullptr, stream, g0, g1);
+                    if (rc != WASH_OK) return rc;
+                }
+                if (ops & WASH_OP_AVERAGE) {
+                    rc = reduce_impl(ctx, wash::kOpAverage, WASH_STACK_PARAMS, ctx->avg_dev, pd, 0.0f, 0, ctx->n_seg, nullptr, stream, g0, g1);
+                    if (rc != WASH_OK) return rc;
+                }
+                if ((err = cudaEventRecord(ev_done[k], stream)) != cudaSuccess || (err = cudaStreamWaitEvent(ctx->copy_out, ev_done[k], 0)) != cudaSuccess)
+                    return cuda_fail(err, "pipeline event");
+                if ((err = copy_range(host_params, ctx->stack_ptr[WASH_STACK_PARAMS], pd, e0, count, cudaMemcpyDeviceToHost, ctx->copy_out)) != cudaSuccess)
+                    return cuda_fail(err, "copy of a parameter range to the host");
+                if (host_opt && (err = copy_range(host_opt, ctx->stack_ptr[WASH_STACK_OPT], od, e0, count, cudaMemcpyDeviceToHost, ctx->copy_out)) != cudaSuccess)
+                    return cuda_fail(err, "copy of an optimizer-state range to the host");
+                if ((ops & WASH_OP_AVERAGE) &&
+                    (err = cudaMemcpyAsync(static_cast<char *>(host_avg) + e0 * elem_bytes(pd), static_cast<char *>(ctx->avg_dev) + e0 * elem_bytes(pd),
+                                           count * elem_bytes(pd), cudaMemcpyDeviceToHost, ctx->copy_out)) != cudaSuccess)
+                    return cuda_fail(err, "copy of an average range to the host");
             }
-            const size_t off = e0 * ctx->N * eb;
-            return cudaMemcpyAsync(static_cast<char *>(dst) + off, static_cast<const char *>(src) + off, count * ctx->N * eb, kind, s);
+            // the caller's stream continues only when the last range is back on the host
+            if ((err = cudaEventRecord(ev_out, ctx->copy_out)) != cudaSuccess || (err = cudaStreamWaitEvent(stream, ev_out, 0)) != cudaSuccess)
+                return cuda_fail(err, "pipeline event");
+            if ((ops & WASH_OP_SHUFFLE) && (err = cudaMemcpyAsync(&st, ctx->stats_dev, sizeof st, cudaMemcpyDeviceToHost, stream)) != cudaSuccess)
+                return cuda_fail(err, "copy of the counters to the host");
+            if ((err = cudaStreamSynchronize(stream)) != cudaSuccess) return cuda_fail(err, "cudaStreamSynchronize");
+            if (host_stats) *host_stats = st;
+            return WASH_OK;
         };
-        const int od = ctx->stack_dtype[WASH_STACK_OPT];
-        for (int k = 0; k < kPipeChunks; ++k) {
-            const uint32_t g0 = static_cast<uint32_t>(k) * per;
-            if (g0 >= ctx->n_groups) break;
-            const uint32_t g1 = g0 + per < ctx->n_groups ? g0 + per : ctx->n_groups;
-            const size_t e0 = 4ull * g0, count = 4ull * (g1 - g0);
-            if ((err = copy_range(ctx->stack_ptr[WASH_STACK_PARAMS], host_params, pd, e0, count, cudaMemcpyHostToDevice, ctx->copy_in)) != cudaSuccess)
-                return cuda_fail(err, "copy of a parameter range to the device");
-            if (host_opt && (err = copy_range(ctx->stack_ptr[WASH_STACK_OPT], host_opt, od, e0, count, cudaMemcpyHostToDevice, ctx->copy_in)) != cudaSuccess)
-                return cuda_fail(err, "copy of an optimizer-state range to the device");
-            if ((err = cudaEventRecord(ev_in[k], ctx->copy_in)) != cudaSuccess || (err = cudaStreamWaitEvent(stream, ev_in[k], 0)) != cudaSuccess)
-                return cuda_fail(err, "pipeline event");
-            if (ops & WASH_OP_SHUFFLE) {
-                rc = shuffle_impl(ctx, host_opt ? 2 : 0, step, p, p_layer, seed, stream, ctx->stats_dev, g0, g1);
-                if (rc != WASH_OK) return rc;
-            }
-            if (ops & WASH_OP_EMA) {
-                rc = reduce_impl(ctx, wash::kOpEma, WASH_STACK_PARAMS, nullptr, WASH_F32, alpha, 0, ctx->n_seg, nullptr, stream, g0, g1);
-                if (rc != WASH_OK) return rc;
-            }
-            if (ops & WASH_OP_AVERAGE) {
-                rc = reduce_impl(ctx, wash::kOpAverage, WASH_STACK_PARAMS, ctx->avg_dev, pd, 0.0f, 0, ctx->n_seg, nullptr, stream, g0, g1);
-                if (rc != WASH_OK) return rc;
-            }
-            if ((err = cudaEventRecord(ev_done[k], stream)) != cudaSuccess || (err = cudaStreamWaitEvent(ctx->copy_out, ev_done[k], 0)) != cudaSuccess)
-                return cuda_fail(err, "pipeline event");
-            if ((err = copy_range(host_params, ctx->stack_ptr[WASH_STACK_PARAMS], pd, e0, count, cudaMemcpyDeviceToHost, ctx->copy_out)) != cudaSuccess)
-                return cuda_fail(err, "copy of a parameter range to the host");
-            if (host_opt && (err = copy_range(host_opt, ctx->stack_ptr[WASH_STACK_OPT], od, e0, count, cudaMemcpyDeviceToHost, ctx->copy_out)) != cudaSuccess)
-                return cuda_fail(err, "copy of an optimizer-state range to the host");
-            if ((ops & WASH_OP_AVERAGE) &&
-                (err = cudaMemcpyAsync(static_cast<char *>(host_avg) + e0 * elem_bytes(pd), static_cast<char *>(ctx->avg_dev) + e0 * elem_bytes(pd),
-                                       count * elem_bytes(pd), cudaMemcpyDeviceToHost, ctx->copy_out)) != cudaSuccess)
-                return cuda_fail(err, "copy of an average range to the host");
+        const int prc = pipeline();
+        if (prc != WASH_OK) {
+            const std::string first = g_last_error;
+            cudaStreamSynchronize(ctx->copy_in);
+            cudaStreamSynchronize(stream);
+            cudaStreamSynchronize(ctx->copy_out);
+            cudaGetLastError();
+            g_last_error = first;
         }
-        // the caller's stream continues only when the last range is back on the host
-        if ((err = cudaEventRecord(ev_out, ctx->copy_out)) != cudaSuccess || (err = cudaStreamWaitEvent(stream, ev_out, 0)) != cudaSuccess)
-            return cuda_fail(err, "pipeline event");
-        if ((ops & WASH_OP_SHUFFLE) && (err = cudaMemcpyAsync(&st, ctx->stats_dev, sizeof st, cudaMemcpyDeviceToHost, stream)) != cudaSuccess)
-            return cuda_fail(err, "copy of the counters to the host");
-        if ((err = cudaStreamSynchronize(stream)) != cudaSuccess) return cuda_fail(err, "cudaStreamSynchronize");
-        if (host_stats) *host_stats = st;
-        return WASH_OK;
+        return prc;
     }
     if ((err = cudaMemcpyAsync(ctx->stack_ptr[WASH_STACK_PARAMS], host_params, p_bytes, cudaMemcpyHostToDevice, stream)) != cudaSuccess)
         return cuda_fail(err, "copy of the parameter stack to the device");
@@ -797,16 +818,34 @@ int wash_exchange_staging_open(wash_ctx *ctx, int32_t stack, int32_t parity, con
     if (!ctx->x_own[parity][stack]) return fail(WASH_ERR_STATE, "create this worker's buffer first (wash_exchange_staging_create)");
     DeviceGuard guard(ctx->device);
     if (guard.err != cudaSuccess) return cuda_fail(guard.err, "cudaSetDevice");
+    if (ctx->x_opened_set[parity][stack]) return fail(WASH_ERR_STATE, "the peers' buffers of staging set %d of stack %d are already open", parity, stack);
     std::vector<void *> buffers(static_cast<size_t>(ctx->N), nullptr);
+    std::vector<void *> mapped;   // what this call opened: closed again if it fails part-way
+    auto roll_back = [&]() {
+        for (void *peer : mapped) cudaIpcCloseMemHandle(peer);
+        cudaGetLastError();
+    };
     for (int n = 0; n < ctx->N; ++n) {
         if (n == ctx->x_self) { buffers[n] = ctx->x_own[parity][stack]; continue; }
         cudaIpcMemHandle_t handle;
         std::memcpy(&handle, static_cast<const char *>(handles) + static_cast<size_t>(n) * WASH_IPC_HANDLE_BYTES, sizeof handle);
         cudaError_t err = cudaIpcOpenMemHandle(&buffers[n], handle, cudaIpcMemLazyEnablePeerAccess);
-        if (err != cudaSuccess) return cuda_fail(err, "cudaIpcOpenMemHandle (is worker's buffer in another process on a device this one can reach?)");
-        ctx->x_opened.push_back(buffers[n]);
+        if (err != cudaSuccess) {
+            roll_back();
+            return cuda_fail(err, "cudaIpcOpenMemHandle (is worker's buffer in another process on a device this one can reach?)");
+        }
+        mapped.push_back(buffers[n]);
     }
-    return wash_exchange_staging(ctx, stack, parity, buffers.data(), ctx->x_capacity[parity][stack]);
+    const int rc = wash_exchange_staging(ctx, stack, parity, buffers.data(), ctx->x_capacity[parity][stack]);
+    if (rc != WASH_OK) {
+        const std::string first = g_last_error;
+        roll_back();
+        g_last_error = first;
+        return rc;
+    }
+    ctx->x_opened.insert(ctx->x_opened.end(), mapped.begin(), mapped.end());
+    ctx->x_opened_set[parity][stack] = true;
+    return WASH_OK;
 }
 
 int wash_exchange_plan(wash_ctx *ctx, uint64_t step, double p, const double *p_layer, uint64_t seed, void *stream_v)

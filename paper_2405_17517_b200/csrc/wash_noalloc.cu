@@ -4,9 +4,9 @@
 // in device memory by cudaMalloc at wash_create time.  Some callers cannot do that:
 // a training process whose framework has already claimed all of the GPU's memory for
 // its own pool (a cudaMalloc from a library would fail, or would have to be carved out
-// of the pool by hand), and latency-sensitive loops in which the implicit device-wide
-// synchronisation of cudaMalloc / cudaFree would stall kernels that other streams have
-// in flight.  For them the same kernel is launched with its tables in a fixed array
+// of the pool by hand), and loops in which the implicit device-wide synchronisation of
+// cudaMalloc / cudaFree would stall kernels that other streams have in flight (each call
+// here still makes two small pageable host-to-device copies, ordered on its stream).  For them the same kernel is launched with its tables in a fixed array
 // that is part of the library image: it exists on every GPU that loads libwash.so, from
 // load to exit, and costs kScratchBytes there whether or not this entry point is used.
 #include <cmath>
@@ -123,8 +123,16 @@ extern "C" int wash_shuffle_noalloc(int32_t N, int32_t n_tensors, const int64_t 
         scratch = g_scratch_addr[device];
         sm_count = g_sm_count[device];
     }
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
     if (rc == WASH_OK) {
-        cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
+        // the table uploads below read host arrays that die with this call: a captured copy
+        // would read freed memory at replay
+        cudaStreamCaptureStatus capture = cudaStreamCaptureStatusNone;
+        err = cudaStreamIsCapturing(stream, &capture);
+        if (err != cudaSuccess) rc = fail(WASH_ERR_CUDA, cudaGetErrorString(err));
+        else if (capture != cudaStreamCaptureStatusNone) rc = fail(WASH_ERR_STATE, "the stream is in capture mode: wash_shuffle_noalloc copies its tables from host arrays that do not outlive the call");
+    }
+    if (rc == WASH_OK) {
         SegEntry *seg_dev = reinterpret_cast<SegEntry *>(scratch);
         uint32_t *tile_dev = reinterpret_cast<uint32_t *>(scratch + kSegBytes);
         // Both tables are rewritten in full and the counters' partial sums are zeroed, in

@@ -1,7 +1,8 @@
 """GPU parity at the benchmark's full sizes: the ResNet populations of configs 2-4 in the
-launch configuration bench.py times (default mode and launch shape), compared with the
-oracle bit for bit, and a multi-gigabyte flat population of config 5 checked on sampled
-coordinate ranges that the oracle recomputes on its own."""
+launch configurations bench.py times (streaming, sparse and automatic mode, default launch
+shape), compared with the oracle bit for bit; config 5's parity grid (2^20 coordinates, every
+N, p and layout of the sweep, host-generated values); and multi-gigabyte flat populations of
+config 5 checked on sampled coordinate ranges that the oracle recomputes on its own."""
 import numpy as np
 import pytest
 import torch
@@ -24,8 +25,14 @@ def _resnet_case(name):
     return cfg, c, len(table)
 
 
-def test_config2_resnet18_n5_full_size():
+MODES = [B.WASH_MODE_STREAM, B.WASH_MODE_SPARSE, B.WASH_MODE_AUTO]
+MODE_IDS = ["stream", "sparse", "auto"]
+
+
+@pytest.mark.parametrize("mode", MODES, ids=MODE_IDS)
+def test_config2_resnet18_n5_full_size(mode):
     cfg, c, T = _resnet_case("cfg2_resnet18_n5")
+    B.wash_set_mode(c.gpu.ctx, mode)
     oracle.set_threads(oracle.max_threads())
     tot = [0, 0]
     for step in range(4):
@@ -46,36 +53,44 @@ def test_config2_resnet18_n5_full_size():
     c.close()
 
 
-def test_config3_resnet50_n10_thousand_steps_per_layer_p():
-    """N = 10, 161 tensors, p_t = 0.01 (1 - t/160), momentum shuffled along, 1000 steps;
-    compared at steps 0, 1, 10, 100 and 999, counters at the end."""
+@pytest.mark.parametrize("mode,steps", [(B.WASH_MODE_STREAM, 1000), (B.WASH_MODE_SPARSE, 50), (B.WASH_MODE_AUTO, 50)], ids=MODE_IDS)
+def test_config3_resnet50_n10_per_layer_p_many_steps(mode, steps):
+    """N = 10, 161 tensors, p_t = 0.01 (1 - t/160), momentum shuffled along, 1000 steps in the
+    streaming mode (50 in the others); compared at steps 0, 1, 10, 100 (where reached) and the
+    last, counters at the end."""
     cfg, c, T = _resnet_case("cfg3_resnet50_n10")
+    B.wash_set_mode(c.gpu.ctx, mode)
     oracle.set_threads(oracle.max_threads())
     pl = B.wash_layer_probs(T, cfg["p"], B.WASH_SCHEDULE_DECREASING)
     assert np.array_equal(pl, oracle.layer_probs(T, cfg["p"]))
     tot = [0, 0]
-    for step in range(1000):
+    for step in range(steps):
         B.wash_shuffle_both(c.gpu.ctx, step, cfg["p"], pl, seed=3, stats=c.stats_dev)
         s = oracle.shuffle(c.ora, c.host, pl, seed=3, step=step, stack2=c.host_opt)
         tot[0] += s[0]; tot[1] += s[1]
-        if step in (0, 1, 10, 100, 999):
+        if step in (0, 1, 10, 100, steps - 1):
             c.assert_equal("cfg3 step %d" % step)
     assert c.gpu_stats() == tuple(tot)
     # the paper's communicated fraction for this schedule, measured: sum_t q_t d_t / P per step
     numel = np.asarray(c.numel, dtype=np.float64)
-    expect = (np.floor(pl * 2.0 ** 32) / 2.0 ** 32 * numel).sum() * 1000
+    expect = (np.floor(pl * 2.0 ** 32) / 2.0 ** 32 * numel).sum() * steps
     assert abs(tot[0] - expect) < 5 * np.sqrt(expect)
     oracle.set_threads(1)
     c.close()
 
 
-def test_config4_resnet50_bf16_weights_fp32_momentum():
+@pytest.mark.parametrize("mode", MODES, ids=MODE_IDS)
+def test_config4_resnet50_bf16_weights_fp32_momentum(mode):
     cfg, c, T = _resnet_case("cfg4_resnet50_bf16_n8")
+    B.wash_set_mode(c.gpu.ctx, mode)
     oracle.set_threads(oracle.max_threads())
+    tot = [0, 0]
     for step in range(3):
         B.wash_shuffle_both(c.gpu.ctx, step, cfg["p"], None, seed=5, stats=c.stats_dev)
-        oracle.shuffle(c.ora, c.host, cfg["p"], seed=5, step=step, stack2=c.host_opt)
+        s = oracle.shuffle(c.ora, c.host, cfg["p"], seed=5, step=step, stack2=c.host_opt)
+        tot[0] += s[0]; tot[1] += s[1]
     c.assert_equal("cfg4 shuffle")
+    assert c.gpu_stats() == tuple(tot)
     for alpha in (0.999, 0.001):
         B.papa_ema(c.gpu.ctx, B.WASH_STACK_PARAMS, alpha)
         oracle.papa_ema(c.ora, c.host, alpha)
@@ -86,6 +101,29 @@ def test_config4_resnet50_bf16_weights_fp32_momentum():
         want = np.zeros(c.P, dtype=np_dtype)
         oracle.population_average(c.ora, c.host, want)
         assert (to_host_bits(out) == bits(want)).all()
+    oracle.set_threads(1)
+    c.close()
+
+
+@pytest.mark.parametrize("mode", [B.WASH_MODE_STREAM, B.WASH_MODE_SPARSE], ids=["stream", "sparse"])
+@pytest.mark.parametrize("layout", [0, 1], ids=["NP", "PN"])
+@pytest.mark.parametrize("p", [1e-4, 1e-3, 1e-2, 0.1, 1.0])
+@pytest.mark.parametrize("N", [2, 4, 8, 16, 32])
+def test_config5_parity_grid(N, p, layout, mode):
+    """Config 5's parity cells: one flat fp32 tensor of 2^20 coordinates per model, values
+    0.05 randn generated on the host, every N, p and layout of the sweep in both kernels;
+    the whole stack and the counters compared with the oracle after two steps."""
+    P = 1 << 20
+    c = Case(N, [P], layout, dense=W.flat_population(N, P, seed=100 + N, std=0.05))
+    B.wash_set_mode(c.gpu.ctx, mode)
+    oracle.set_threads(oracle.max_threads())
+    tot = [0, 0]
+    for step in (0, 1):
+        B.wash_shuffle(c.gpu.ctx, step, p, None, seed=55, stats=c.stats_dev)
+        s = oracle.shuffle(c.ora, c.host, p, seed=55, step=step)
+        tot[0] += s[0]; tot[1] += s[1]
+    c.assert_equal("N=%d p=%g layout=%d mode=%d" % (N, p, layout, mode))
+    assert c.gpu_stats() == tuple(tot)
     oracle.set_threads(1)
     c.close()
 

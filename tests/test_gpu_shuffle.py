@@ -212,6 +212,28 @@ def test_argument_and_state_errors():
     B.wash_destroy(ctx)
 
 
+def test_a_rejected_probability_vector_leaves_the_context_consistent():
+    """A call refused for one bad entry of p_layer must not change the thresholds the next
+    call compares with: the following valid call (which repeats the good entries) has to
+    upload its table and match the oracle."""
+    N, numel = 4, [3000, 2000, 500]
+    c = Case(N, numel, 0, "f32", "f32", seed=13)
+    B.wash_shuffle_both(c.gpu.ctx, 0, 0.0, [0.1, 0.1, 0.1], seed=3, stats=c.stats_dev)
+    st = list(oracle.shuffle(c.ora, c.host, [0.1, 0.1, 0.1], seed=3, step=0, stack2=c.host_opt))
+    for bad in ([0.5, 2.0, 0.0], [0.5, 0.25, float("nan")]):
+        with pytest.raises(B.WashError) as e:
+            B.wash_shuffle_both(c.gpu.ctx, 1, 0.0, bad, seed=3, stats=c.stats_dev)
+        assert e.value.code == B.WASH_ERR_ARG
+    c.assert_equal("after the refused calls")          # nothing ran
+    for step, pl in ((1, [0.5, 0.0, 0.0]), (2, [0.5, 0.25, 0.0]), (3, [0.1, 0.1, 0.1])):
+        B.wash_shuffle_both(c.gpu.ctx, step, 0.0, pl, seed=3, stats=c.stats_dev)
+        s = oracle.shuffle(c.ora, c.host, pl, seed=3, step=step, stack2=c.host_opt)
+        st[0] += s[0]; st[1] += s[1]
+        c.assert_equal("step %d" % step)
+    assert c.gpu_stats() == tuple(st)
+    c.close()
+
+
 def test_resume_from_a_host_copy_continues_bit_identically():
     """The shuffle is a pure function of (stack bits, seed, step, tensor table, p): 20 steps
     in one context equal 10 steps, a round trip of the stacks through host memory into a

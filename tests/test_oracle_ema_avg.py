@@ -55,6 +55,55 @@ def test_ema_contracts_consensus_distance_by_alpha_squared_and_keeps_the_mean():
     assert np.abs(mean_after - mean_before).max() < 1e-6
 
 
+@pytest.mark.parametrize("layout", [0, 1])
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_consensus_distance_per_model_and_per_tensor_range(layout, dtype):
+    """Fig. 2's quantity from its definition, written out per model with exact rational
+    arithmetic on a small stack and with numpy's binary64 on a larger one: distinct models
+    (a sum landing in another model's slot shows), a range that leaves out the first and the
+    last tensor (an ignored bound shows), the plain unit scale (a constant factor shows)."""
+    N, numel = 4, [5, 12, 3, 9, 6]
+    pop, off, P = _pop(N, numel, layout)
+    dense = W.flat_population(N, sum(numel), seed=21, std=1.0)
+    dense *= (1.0 + np.arange(N, dtype=np.float32))[:, None]         # models at visibly different distances
+    if dtype == "bf16":
+        x = W.to_stack(W.to_bf16_bits(dense), numel, off, P, layout)
+        vals = W.bf16_bits_to_f32(W.to_bf16_bits(dense))
+    else:
+        x = W.to_stack(dense, numel, off, P, layout)
+        vals = dense
+    bounds = np.concatenate([[0], np.cumsum(numel)])
+    for lo, hi in ((0, 5), (1, 4), (2, 3), (4, 5), (3, 3)):
+        got = oracle.consensus_sq(pop, x, lo, hi)
+        cols = range(int(bounds[lo]), int(bounds[hi]))
+        want = []
+        for n in range(N):
+            acc = Fraction(0)
+            for i in cols:
+                mean = sum(Fraction(float(vals[m, i])) for m in range(N)) / N
+                acc += (Fraction(float(vals[n, i])) - mean) ** 2
+            want.append(float(acc))
+        assert np.allclose(got, want, rtol=1e-13, atol=0), (lo, hi, got, want)
+        if hi > lo:
+            assert len(set(np.round(got, 9))) == N                   # the models really differ
+    # a larger stack against numpy, every model and two ranges
+    N, numel = 7, [1000, 64, 333, 2048, 17]
+    pop, off, P = _pop(N, numel, layout)
+    dense = W.flat_population(N, sum(numel), seed=5, std=0.3) + np.linspace(-1, 1, N, dtype=np.float32)[:, None]
+    x = W.to_stack(dense, numel, off, P, layout)
+    th = dense.astype(np.float64)
+    bounds = np.concatenate([[0], np.cumsum(numel)])
+    for lo, hi in ((0, 5), (1, 4)):
+        sl = th[:, bounds[lo]:bounds[hi]]
+        want = ((sl - sl.mean(axis=0, keepdims=True)) ** 2).sum(axis=1)
+        assert np.allclose(oracle.consensus_sq(pop, x, lo, hi), want, rtol=1e-11, atol=0)
+    # Fig. 2's distance itself, (1/N) sum_n ||theta_n - mean||, for one hand-made case:
+    # two models at +-1 on d coordinates are each sqrt(d) away from their mean
+    pop2, off2, P2 = _pop(2, [16], layout)
+    x2 = W.to_stack(np.stack([np.ones(16, np.float32), -np.ones(16, np.float32)]), [16], off2, P2, layout)
+    assert oracle.consensus_sq(pop2, x2).tolist() == [16.0, 16.0]
+
+
 def test_ema_special_cases():
     # N = 2, alpha = 1/2 on a coarse grid: every operation is exact, so the result is
     # exactly halfway between the model and the midpoint of the two

@@ -34,6 +34,10 @@ MUTATIONS = {
     "slot counts include fixed points": ("need[n] += (perm[n] != n);", "need[n] += 1;", "test_oracle_exchange.py"),
     "slots numbered per sender": ("const int64_t slot = next[n]++;\n                if (perm[n] != self) continue;           /* another worker fills this slot   */",
                                   "if (perm[n] != self) continue;\n                const int64_t slot = next[n]++;", "test_oracle_exchange.py"),
+    "consensus sum lands in the next model's slot": ("sq_out[n] += dlt * dlt;", "sq_out[(n + 1) % pop->N] += dlt * dlt;", "test_oracle_ema_avg.py"),
+    "consensus ignores the first tensor of its range": ("for (int s = seg_lo; s < seg_hi; ++s) {\n        for (int64_t c = 0; c < pop->numel[s]; ++c) {\n            int64_t elem = pop->offset[s] + c;\n            double mean = 0.0;",
+                                                        "for (int s = 0; s < seg_hi; ++s) {\n        for (int64_t c = 0; c < pop->numel[s]; ++c) {\n            int64_t elem = pop->offset[s] + c;\n            double mean = 0.0;", "test_oracle_ema_avg.py"),
+    "consensus divides the mean by N-1": ("mean /= (double)pop->N;", "mean /= (double)(pop->N - 1);", "test_oracle_ema_avg.py"),
     "last layer still shuffled": ("(double)l / (double)(L - 1);", "(double)l / (double)(L);", "test_oracle_ema_avg.py"),
 }
 
