@@ -288,7 +288,8 @@ def time_launches(torch, stream, launch, first_step: int, min_s: float = 0.06, b
     return float(np.median(per)), float(min(per)), n * blocks
 
 
-def shuffle_cell(B, torch, stream, pop, shuffle_fn, N, P, Es, p_eff, layout, peak, philox_rate, modes=("stream", "sparse")):
+def shuffle_cell(B, torch, stream, pop, shuffle_fn, N, P, Es, p_eff, layout, peak, philox_rate, modes=("stream", "sparse"),
+                 consensus_fn=None):
     """Times one population's shuffle in the given modes and relates it to both ceilings:
     t_HBM = bytes / measured copy bandwidth, t_ALU = Philox blocks / measured probe rate."""
     stats = torch.zeros(2, dtype=torch.int64, device="cuda")
@@ -318,6 +319,11 @@ def shuffle_cell(B, torch, stream, pop, shuffle_fn, N, P, Es, p_eff, layout, pea
             rec.update({"algorithmic_GBps": 2.0 * sel * N * E_sum / (med * 1e-3) / 1e9, "bound": "alu"})
         out[mode] = rec
     B.wash_set_mode(pop.ctx, B.WASH_MODE_STREAM)
+    if consensus_fn is not None:
+        # the streaming shuffle with the distance to the consensus (per quarter of the tensor
+        # table) gathered in the same pass
+        med, lo, n = time_launches(torch, stream, lambda i: consensus_fn(i, stats), 100)
+        out["stream_with_consensus"] = {"ms": med, "ms_min": lo, "launches": n, "ratio_to_stream": med / out["stream"]["ms"]}
     return out
 
 
@@ -346,7 +352,10 @@ def configs_record(B, torch, stream, peak, philox_rate, main_name, main_cell) ->
         fn = (lambda i, st: B.wash_shuffle_both(pop.ctx, i, wl.p, p_layer, SEED, stream, st)) if wl.opt else \
              (lambda i, st: B.wash_shuffle(pop.ctx, i, wl.p, p_layer, SEED, stream, st))
         p_eff = wl.p if p_layer is None else float((p_layer * wl.numel).sum() / wl.P)
-        cell = shuffle_cell(B, torch, stream, pop, fn, wl.N, wl.P, wl.Es, p_eff, "[N][P]", peak, philox_rate)
+        sq = torch.zeros(4 * wl.N, dtype=torch.float64, device="cuda")
+        quarters = [0, wl.T // 4, wl.T // 2, 3 * wl.T // 4, wl.T] if wl.T >= 4 else [0, wl.T]
+        cfn = lambda i, st: B.wash_shuffle_consensus(pop.ctx, B.WASH_STACK_BOTH if wl.opt else B.WASH_STACK_PARAMS, i, wl.p, p_layer, SEED, stream, st, quarters, sq)
+        cell = shuffle_cell(B, torch, stream, pop, fn, wl.N, wl.P, wl.Es, p_eff, "[N][P]", peak, philox_rate, consensus_fn=cfn)
         cell["footprint_bytes"] = wl.N * pop.padded_P * (wl.E + wl.E_opt)
         cell["l2"] = "beyond L2" if cell["footprint_bytes"] > 2.5e8 else "L2-resident"
         rec[name] = cell
@@ -504,8 +513,12 @@ def run_ours(args, rank: int, world: int, local_rank: int) -> None:
     peak, peak_src = measured_peak()
     philox_rate = measure_philox_rate(B, torch, stream)
     fence()
+    sq_d = torch.zeros(4 * wl.N, dtype=torch.float64, device="cuda")
+    quarters = [0, wl.T // 4, wl.T // 2, 3 * wl.T // 4, wl.T] if wl.T >= 4 else [0, wl.T]
     main_cell = shuffle_cell(B, torch, stream, pop, lambda i, st_: step_shuffle(i, st_), wl.N, wl.P, wl.Es, p_eff,
-                             "[N][P]", peak, philox_rate)
+                             "[N][P]", peak, philox_rate,
+                             consensus_fn=lambda i, st_: B.wash_shuffle_consensus(pop.ctx, B.WASH_STACK_BOTH if wl.opt else B.WASH_STACK_PARAMS, i, wl.p,
+                                                                                  p_layer, SEED, stream, st_, quarters, sq_d))
     B.wash_set_mode(pop.ctx, mode_code)
     fence()
 

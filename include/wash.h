@@ -168,6 +168,33 @@ int wash_shuffle_opt_state(wash_ctx *ctx, uint64_t step, double p, const double 
 int wash_shuffle_both(wash_ctx *ctx, uint64_t step, double p, const double *p_layer,
                       uint64_t seed, void *stream, wash_stats *stats);
 
+/* The shuffling step with the distance to the consensus gathered in the same pass.
+ * The streaming shuffle already brings every coordinate's N values on chip; this call
+ * also sums, per model and per range of tensors, the squared deviation from the mean over
+ * the models (the quantity of Eq. 2 and Eq. 5; Fig. 2 plots its square root averaged over
+ * models, Fig. 4 the same per quarter of the parameters) -- no second read of the stack.
+ * The values are those before the exchange; by Eq. 5 the exchange leaves the total over the
+ * models unchanged.
+ *   stacks         WASH_STACK_PARAMS, WASH_STACK_OPT or WASH_STACK_BOTH: what is shuffled
+ *                  (as wash_shuffle / wash_shuffle_opt_state / wash_shuffle_both); the
+ *                  statistic is taken on the first of them (the parameters unless only the
+ *                  optimizer state is shuffled);
+ *   n_ranges       1 .. WASH_MAX_CONSENSUS_RANGES;
+ *   tensor_bounds  HOST array of n_ranges + 1 ascending tensor indices in [0, n_tensors]:
+ *                  range r covers tensors tensor_bounds[r] .. tensor_bounds[r+1]-1 (tensors
+ *                  outside every range are shuffled but not measured);
+ *   dev_sq_out     DEVICE array [n_ranges][N] of doubles the caller has zeroed:
+ *                  dev_sq_out[r][n] += sum over the range's coordinates of
+ *                  (x_n^i - mean^i)^2, in binary64 (sums arrive through atomics, so the
+ *                  last bits depend on their order).
+ * Always runs the streaming kernel, whatever wash_set_mode says.  Other arguments, errors
+ * and the bits of the stacks: as wash_shuffle. */
+#define WASH_STACK_BOTH 2
+#define WASH_MAX_CONSENSUS_RANGES 8
+int wash_shuffle_consensus(wash_ctx *ctx, int32_t stacks, uint64_t step, double p, const double *p_layer,
+                           uint64_t seed, void *stream, wash_stats *stats, int32_t n_ranges,
+                           const int32_t *tensor_bounds, double *dev_sq_out);
+
 /* ---- comparison operators --------------------------------------------------------- */
 
 /* PAPA's EMA (Eq. 1), in place on the chosen stack, 0 < alpha < 1:

@@ -20,7 +20,8 @@ WASH_OK = 0
 WASH_ERR_ARG, WASH_ERR_STATE, WASH_ERR_ALLOC, WASH_ERR_CUDA, WASH_ERR_UNSUPPORTED, WASH_ERR_DEVICE_CHECK = -1, -2, -3, -4, -5, -6
 WASH_LAYOUT_NP, WASH_LAYOUT_PN = 0, 1
 WASH_F32, WASH_BF16 = 0, 1
-WASH_STACK_PARAMS, WASH_STACK_OPT = 0, 1
+WASH_STACK_PARAMS, WASH_STACK_OPT, WASH_STACK_BOTH = 0, 1, 2
+WASH_MAX_CONSENSUS_RANGES = 8
 WASH_SCHEDULE_DECREASING, WASH_SCHEDULE_CONSTANT, WASH_SCHEDULE_INCREASING = 0, 1, 2
 WASH_MODE_STREAM, WASH_MODE_SPARSE, WASH_MODE_STREAM_STAGED, WASH_MODE_STREAM_REGISTERS, WASH_MODE_AUTO = 0, 1, 2, 3, 4
 WASH_OP_SHUFFLE, WASH_OP_EMA, WASH_OP_AVERAGE = 1, 2, 4
@@ -62,6 +63,7 @@ def load() -> ctypes.CDLL:
     L.wash_layer_probs.argtypes = [i32, dbl, i32, dblp]
     for name in ("wash_shuffle", "wash_shuffle_opt_state", "wash_shuffle_both"):
         getattr(L, name).argtypes = [vp, u64, dbl, dblp, u64, vp, vp]
+    L.wash_shuffle_consensus.argtypes = [vp, i32, u64, dbl, dblp, u64, vp, vp, i32, ctypes.POINTER(i32), vp]
     L.papa_ema.argtypes = [vp, i32, ctypes.c_float, vp]
     L.population_average.argtypes = [vp, i32, vp, i32, vp]
     L.papa_all.argtypes = [vp, i32, vp]
@@ -190,6 +192,15 @@ def wash_shuffle_opt_state(ctx, step, p, p_layer=None, seed=0, stream=None, stat
 
 def wash_shuffle_both(ctx, step, p, p_layer=None, seed=0, stream=None, stats=None) -> None:
     _shuffle(load().wash_shuffle_both, ctx, step, p, p_layer, seed, stream, stats)
+
+
+def wash_shuffle_consensus(ctx, stacks: int, step, p, p_layer=None, seed=0, stream=None, stats=None,
+                           tensor_bounds=(0, 0), dev_sq_out=None) -> None:
+    """tensor_bounds: n_ranges + 1 ascending tensor indices; dev_sq_out: [n_ranges][N] doubles on the device"""
+    keep, pl = _dbl_or_null(p_layer)
+    tb = np.ascontiguousarray(tensor_bounds, dtype=np.int32)
+    _check(load().wash_shuffle_consensus(ctx, stacks, step, float(p), pl, seed, _stream(stream), _ptr(stats), tb.size - 1,
+                                         tb.ctypes.data_as(ctypes.POINTER(ctypes.c_int32)), _ptr(dev_sq_out)))
 
 
 def papa_ema(ctx, stack: int, alpha: float, stream=None) -> None:

@@ -85,6 +85,7 @@ struct wash_ctx {
     uint32_t *status_dev = nullptr;
     wash_stats *stats_dev = nullptr;       // for wash_step_host
     wash::StatSlot *stat_slots_dev = nullptr;
+    double *sq_slots_dev = nullptr;        // partial sums of wash_shuffle_consensus, allocated on first use, zero between calls
     double expected_selected = 0.0;        // sum over tensors of numel * thr / 2^32, for the current thresholds
     void *avg_dev = nullptr;               // for wash_step_host, allocated on first use
     size_t avg_bytes = 0;
@@ -122,6 +123,7 @@ void release(wash_ctx *ctx)
     if (ctx->status_dev) cudaFree(ctx->status_dev);
     if (ctx->stats_dev) cudaFree(ctx->stats_dev);
     if (ctx->stat_slots_dev) cudaFree(ctx->stat_slots_dev);
+    if (ctx->sq_slots_dev) cudaFree(ctx->sq_slots_dev);
     if (ctx->avg_dev) cudaFree(ctx->avg_dev);
     if (ctx->x_mask) cudaFree(ctx->x_mask);
     if (ctx->x_warp_total) cudaFree(ctx->x_warp_total);
@@ -211,7 +213,8 @@ int ensure_table(wash_ctx *ctx, cudaStream_t stream)
 
 // which: 0 = parameters, 1 = optimizer state, 2 = both
 int shuffle_impl(wash_ctx *ctx, int which, uint64_t step, double p, const double *p_layer, uint64_t seed,
-                 void *stream_v, wash_stats *stats, uint32_t group_lo = 0, uint32_t group_hi = 0xFFFFFFFFu)
+                 void *stream_v, wash_stats *stats, uint32_t group_lo = 0, uint32_t group_hi = 0xFFFFFFFFu,
+                 const wash::SqArgs *sq = nullptr, double *sq_out = nullptr)
 {
     if (!ctx) return fail(WASH_ERR_ARG, "ctx is NULL");
     if (step >> 56) return fail(WASH_ERR_ARG, "step must be below 2^56");
@@ -264,6 +267,11 @@ int shuffle_impl(wash_ctx *ctx, int which, uint64_t step, double p, const double
             const double share = ctx->layout == WASH_LAYOUT_PN ? 0.10 : 0.03;
             mode = ctx->expected_selected < share * coordinates ? WASH_MODE_SPARSE : WASH_MODE_STREAM;
         }
+        if (sq) {   // the statistic is gathered by the streaming kernel only
+            mode = WASH_MODE_STREAM;
+            args.stat_slots = ctx->stat_slots_dev;
+            args.sq = *sq;
+        }
         if (mode == WASH_MODE_SPARSE) args.stat_slots = nullptr;   // one wave of large blocks: a few hundred atomics at most
     }
     args.status = ctx->status_dev;
@@ -271,6 +279,7 @@ int shuffle_impl(wash_ctx *ctx, int which, uint64_t step, double p, const double
     cudaError_t err = wash::launch_shuffle(args, a_dtype, b_dtype, mode, ctx->shape, stream, &supported);
     if (err != cudaSuccess) return cuda_fail(err, "shuffle kernel launch");
     if (!supported) return fail(WASH_ERR_UNSUPPORTED, "no shuffle kernel for dtypes (%d, %d)", a_dtype, b_dtype);
+    if (sq && (err = wash::launch_sq_flush(*sq, ctx->N, sq_out, stream)) != cudaSuccess) return cuda_fail(err, "consensus flush launch");
     return WASH_OK;
 }
 
@@ -478,6 +487,39 @@ int wash_shuffle_opt_state(wash_ctx *ctx, uint64_t step, double p, const double 
 int wash_shuffle_both(wash_ctx *ctx, uint64_t step, double p, const double *p_layer, uint64_t seed, void *stream, wash_stats *stats)
 {
     return shuffle_impl(ctx, 2, step, p, p_layer, seed, stream, stats);
+}
+
+int wash_shuffle_consensus(wash_ctx *ctx, int32_t stacks, uint64_t step, double p, const double *p_layer, uint64_t seed,
+                           void *stream, wash_stats *stats, int32_t n_ranges, const int32_t *tensor_bounds, double *dev_sq_out)
+{
+    if (!ctx) return fail(WASH_ERR_ARG, "ctx is NULL");
+    if (stacks != WASH_STACK_PARAMS && stacks != WASH_STACK_OPT && stacks != WASH_STACK_BOTH) return fail(WASH_ERR_ARG, "stacks must be WASH_STACK_PARAMS, WASH_STACK_OPT or WASH_STACK_BOTH");
+    if (n_ranges < 1 || n_ranges > WASH_MAX_CONSENSUS_RANGES) return fail(WASH_ERR_ARG, "n_ranges = %d, must be in [1, %d]", n_ranges, WASH_MAX_CONSENSUS_RANGES);
+    if (!tensor_bounds || !dev_sq_out) return fail(WASH_ERR_ARG, "tensor_bounds and dev_sq_out must not be NULL");
+    wash::SqArgs sq;
+    for (int r = 0; r <= n_ranges; ++r) {
+        const int32_t b = tensor_bounds[r];
+        if (b < 0 || b > ctx->n_seg || (r > 0 && b < tensor_bounds[r - 1]))
+            return fail(WASH_ERR_ARG, "tensor_bounds must ascend within [0, %d]; entry %d is %d", ctx->n_seg, r, b);
+        sq.seg_bound[r] = static_cast<uint32_t>(b);
+    }
+    for (int r = n_ranges + 1; r <= wash::kMaxSqRanges; ++r) sq.seg_bound[r] = sq.seg_bound[n_ranges];
+    sq.n_ranges = n_ranges;
+    sq.inv_n = 1.0 / static_cast<double>(ctx->N);
+    if (!ctx->sq_slots_dev) {
+        DeviceGuard guard(ctx->device);
+        if (guard.err != cudaSuccess) return cuda_fail(guard.err, "cudaSetDevice");
+        const size_t bytes = sizeof(double) * wash::kSqSlots * wash::kMaxSqRanges * static_cast<size_t>(ctx->N);
+        cudaError_t err = cudaMalloc(&ctx->sq_slots_dev, bytes);
+        if (err != cudaSuccess) {
+            cudaGetLastError();
+            ctx->sq_slots_dev = nullptr;
+            return fail(WASH_ERR_ALLOC, "device allocation of the consensus partial sums failed: %s", cudaGetErrorString(err));
+        }
+        if ((err = cudaMemset(ctx->sq_slots_dev, 0, bytes)) != cudaSuccess) return cuda_fail(err, "cudaMemset(consensus partial sums)");
+    }
+    sq.slots = ctx->sq_slots_dev;
+    return shuffle_impl(ctx, stacks, step, p, p_layer, seed, stream, stats, 0, 0xFFFFFFFFu, &sq, dev_sq_out);
 }
 
 int papa_ema(wash_ctx *ctx, int32_t stack, float alpha, void *stream)

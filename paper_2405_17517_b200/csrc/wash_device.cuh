@@ -166,10 +166,11 @@ struct GroupInfo {
     uint32_t cgroup;      // index of the group within its tensor (coordinate / 4)
     int valid;            // coordinates of this group that exist (0..4)
     uint64_t thr;
+    uint32_t seg;         // index of the group's segment in the table
 };
 
 // Describes group g given its segment's table entry (two 16-byte halves).
-__device__ __forceinline__ GroupInfo group_info(uint4 lo, uint4 hi, uint32_t g, uint32_t *status);
+__device__ __forceinline__ GroupInfo group_info(uint4 lo, uint4 hi, uint32_t g, uint32_t seg, uint32_t *status);
 
 __device__ __forceinline__ GroupInfo find_group(const PopView &pop, uint32_t g, uint32_t *status)
 {
@@ -178,7 +179,7 @@ __device__ __forceinline__ GroupInfo find_group(const PopView &pop, uint32_t g, 
     while (s < last && g >= __ldg(&pop.seg[s].group_end)) ++s;
     const uint4 lo = __ldg(reinterpret_cast<const uint4 *>(pop.seg + s));       // begin, end, tensor, cgroup_begin
     const uint4 hi = __ldg(reinterpret_cast<const uint4 *>(pop.seg + s) + 1);   // numel, -, thr
-    return group_info(lo, hi, g, status);
+    return group_info(lo, hi, g, s, status);
 }
 
 // As find_group, for a caller that visits groups in increasing order: `cursor` is the
@@ -193,12 +194,13 @@ __device__ __forceinline__ GroupInfo find_group_forward(const SegEntry *seg, int
     cursor = s;
     const uint4 lo = reinterpret_cast<const uint4 *>(seg + s)[0];
     const uint4 hi = reinterpret_cast<const uint4 *>(seg + s)[1];
-    return group_info(lo, hi, g, status);
+    return group_info(lo, hi, g, s, status);
 }
 
-__device__ __forceinline__ GroupInfo group_info(uint4 lo, uint4 hi, uint32_t g, uint32_t *status)
+__device__ __forceinline__ GroupInfo group_info(uint4 lo, uint4 hi, uint32_t g, uint32_t seg, uint32_t *status)
 {
     GroupInfo gi;
+    gi.seg = seg;
     if (g < lo.x || g >= lo.y) {   // table inconsistent with the row: report, touch nothing
         if (status) atomicOr(status, 1u);
         gi.tensor_id = 0; gi.cgroup = 0; gi.valid = 0; gi.thr = 0;

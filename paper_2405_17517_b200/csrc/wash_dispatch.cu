@@ -67,6 +67,27 @@ __global__ void __launch_bounds__(kStatSlots) flush_stats_kernel(StatSlot *slots
     }
 }
 
+// Adds the kSqSlots partial copies of the [range][model] table of squared distances into the
+// caller's array and leaves the slots zeroed for the next launch.
+__global__ void __launch_bounds__(256) sq_flush_kernel(double *slots, int count, double *out)
+{
+    for (int j = threadIdx.x; j < count; j += blockDim.x) {
+        double s = 0.0;
+        for (int k = 0; k < kSqSlots; ++k) {
+            s += slots[k * count + j];
+            slots[k * count + j] = 0.0;
+        }
+        out[j] += s;
+    }
+}
+
+cudaError_t launch_sq_flush(const SqArgs &sq, int N, double *out, cudaStream_t stream)
+{
+    sq_flush_kernel<<<1, 256, 0, stream>>>(sq.slots, sq.n_ranges * N, out);
+    count_launch();
+    return cudaGetLastError();
+}
+
 // Nothing but the mask's Philox blocks: one block of four words per thread, folded by XOR.
 __global__ void __launch_bounds__(256) philox_probe_kernel(unsigned long long n_blocks, const __grid_constant__ PhiloxKeys keys, uint32_t *checksum)
 {

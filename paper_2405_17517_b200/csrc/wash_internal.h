@@ -59,6 +59,18 @@ inline PhiloxKeys philox_keys(uint64_t seed)
     return keys;
 }
 
+// Distance to the consensus gathered inside the streaming shuffle: up to kMaxSqRanges ranges of
+// segments, per range and model a binary64 sum, gathered in kSqSlots partial copies (atomics on
+// one address per model would serialise) that sq_flush_kernel adds into the caller's array.
+constexpr int kMaxSqRanges = 8;
+constexpr int kSqSlots = 64;
+struct SqArgs {
+    double *slots = nullptr;                // device: [kSqSlots][n_ranges][N], zero between launches; nullptr = statistic off
+    int n_ranges = 0;
+    double inv_n = 0.0;                     // 1 / N
+    uint32_t seg_bound[kMaxSqRanges + 1];   // range r = segments seg_bound[r] .. seg_bound[r+1]-1
+};
+
 struct ShuffleArgs {
     PopView pop;
     void *a;                      // first stack (device)
@@ -69,6 +81,7 @@ struct ShuffleArgs {
     unsigned long long *stats;    // device-accessible {selected, moved} or nullptr
     StatSlot *stat_slots;         // device, kStatSlots zeroed entries (left zeroed by every launch), or nullptr
     uint32_t *status;             // device status word
+    SqArgs sq;                    // consensus distance of the first stack (streaming kernel only)
 };
 
 struct ReduceArgs {
@@ -125,6 +138,9 @@ cudaError_t launch_shuffle(const ShuffleArgs &args, int a_dtype, int b_dtype, in
                            const LaunchShape &shape, cudaStream_t stream, bool *supported);
 cudaError_t launch_reduce(const ReduceArgs &args, int op, int dtype, int out_dtype,
                           const LaunchShape &shape, cudaStream_t stream, bool *supported);
+
+// adds the slots' sums into out[n_ranges][N] and zeroes the slots
+cudaError_t launch_sq_flush(const SqArgs &sq, int N, double *out, cudaStream_t stream);
 
 cudaError_t launch_philox_probe(unsigned long long n_blocks, uint64_t seed, uint32_t *checksum, cudaStream_t stream);
 

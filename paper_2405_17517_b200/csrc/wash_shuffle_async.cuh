@@ -166,10 +166,97 @@ __device__ __forceinline__ void serve_tile(const ShuffleArgs &a, const unsigned 
     __syncwarp();   // the warp's list is rewritten by the next tile
 }
 
+// the four values of model n in the group of block thread t, widened to binary32
+template <class T, int LAYOUT>
+__device__ __forceinline__ void image_group(const unsigned char *image, int n_models, uint32_t t, int n, float (&x)[4])
+{
+    if (LAYOUT == kLayoutNP) {
+        const typename T::vec v = reinterpret_cast<const typename T::vec *>(image)[static_cast<uint32_t>(n) * blockDim.x + t];
+#pragma unroll
+        for (int c = 0; c < 4; ++c) x[c] = T::to_float(T::get(v, c));
+    } else {
+#pragma unroll
+        for (int c = 0; c < 4; ++c) x[c] = T::to_float(image_value<T, LAYOUT>(image, n_models, t, n, c));
+    }
+}
+
+// Distance to the consensus (Eq. 2 / Eq. 5; Fig. 2 plots its square root averaged over models)
+// of one tile, from the image the copies have already brought into shared memory: for the four
+// coordinates of a lane's group the binary64 mean over the models, then per model the sum of the
+// squared deviations, summed over the warp by a butterfly and added to one of kSqSlots partial
+// copies of the [range][model] table.  The exchange preserves the quantity (Eq. 5), so the values
+// before it serve.  Called by all threads of the block; `exists`: the thread has a group in this
+// tile.  WHOLE: every lane of the warp has a whole group of one and the same range (the usual
+// case, decided by the caller with one vote), so nothing is predicated per coordinate.
+template <class T, int LAYOUT, bool WHOLE>
+__device__ __forceinline__ void consensus_warp(const ShuffleArgs &a, const unsigned char *image, int valid, uint32_t r1,
+                                               uint32_t r_lo, uint32_t r_hi)
+{
+    const int n_models = a.pop.N;
+    const uint32_t lane = threadIdx.x & 31u;
+    double mean[4] = {0.0, 0.0, 0.0, 0.0};
+    if (WHOLE || r1) {
+        float x[4];
+        for (int n = 0; n < n_models; ++n) {
+            image_group<T, LAYOUT>(image, n_models, threadIdx.x, n, x);
+#pragma unroll
+            for (int c = 0; c < 4; ++c) mean[c] += static_cast<double>(x[c]);
+        }
+        const double count = static_cast<double>(n_models);
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {   // sum / N: the reciprocal's product, corrected by its remainder
+            const double q = mean[c] * a.sq.inv_n;
+            mean[c] = fma(fma(-q, count, mean[c]), a.sq.inv_n, q);
+        }
+    }
+    const uint32_t slot = (blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5)) % kSqSlots;
+    for (uint32_t r = r_lo; r <= r_hi; ++r) {   // one trip unless the warp's groups lie in several ranges
+        double *table = a.sq.slots + (static_cast<size_t>(slot) * a.sq.n_ranges + (r - 1)) * n_models;
+        double keep = 0.0;   // lane l keeps the warp's sum of model l (mod 32)
+        for (int n = 0; n < n_models; ++n) {
+            double s = 0.0;
+            if (WHOLE || r1 == r) {
+                float x[4];
+                image_group<T, LAYOUT>(image, n_models, threadIdx.x, n, x);
+#pragma unroll
+                for (int c = 0; c < 4; ++c)
+                    if (WHOLE || c < valid) {   // padding beyond the tensor's end holds no coordinate
+                        const double d = static_cast<double>(x[c]) - mean[c];
+                        s = fma(d, d, s);
+                    }
+            }
+#pragma unroll
+            for (int off = 16; off > 0; off >>= 1) s += __shfl_xor_sync(0xFFFFFFFFu, s, off);
+            if (static_cast<uint32_t>(n & 31) == lane) keep = s;
+            if ((n & 31) == 31 || n == n_models - 1) {
+                const int n_lane = (n & ~31) + static_cast<int>(lane);
+                if (n_lane <= n && keep != 0.0) atomicAdd(table + n_lane, keep);
+                keep = 0.0;
+            }
+        }
+    }
+}
+
+template <class T, int LAYOUT>
+__device__ __forceinline__ void consensus_tile(const ShuffleArgs &a, const unsigned char *image, const GroupInfo &gi, bool exists)
+{
+    // this lane's range, counted from 1 (0: its group lies in none, or does not exist)
+    uint32_t r1 = 0;
+    if (exists && gi.valid > 0 && gi.seg >= a.sq.seg_bound[0] && gi.seg < a.sq.seg_bound[a.sq.n_ranges]) {
+        r1 = 1;
+        for (int k = 1; k < a.sq.n_ranges; ++k) r1 += gi.seg >= a.sq.seg_bound[k] ? 1u : 0u;
+    }
+    const uint32_t r_hi = __reduce_max_sync(0xFFFFFFFFu, r1);
+    if (r_hi == 0) return;
+    const uint32_t r_lo = __reduce_min_sync(0xFFFFFFFFu, r1 ? r1 : 0xFFFFFFFFu);
+    if (__all_sync(0xFFFFFFFFu, r1 == r_hi && gi.valid == 4)) consensus_warp<T, LAYOUT, true>(a, image, 4, r1, r_hi, r_hi);
+    else consensus_warp<T, LAYOUT, false>(a, image, exists ? gi.valid : 0, r1, r_lo, r_hi);
+}
+
 // G = tiles per block (one group per thread and tile).  Small populations move few bytes per
 // group (N * 16 for fp32), so a thread takes G = 2 groups, T apart, to keep more bytes in
 // flight per SM; the two Philox draws overlap as well.
-template <class TA, class TB, int LAYOUT, int G>
+template <class TA, class TB, int LAYOUT, int G, bool STAT>
 __global__ void __launch_bounds__(256, 5) shuffle_async_kernel(const __grid_constant__ ShuffleArgs a)
 {
     extern __shared__ __align__(128) unsigned char smem_raw[];
@@ -226,6 +313,11 @@ __global__ void __launch_bounds__(256, 5) shuffle_async_kernel(const __grid_cons
     constexpr bool kSharedCopies = LAYOUT == kLayoutPN || TA::kBytes == 2 || (kHasB && TB::kBytes == 2);   // a group's bytes were copied by other threads
     if (kSharedCopies) __syncthreads();
     else __syncwarp();
+    if constexpr (STAT) {
+#pragma unroll
+        for (int i = 0; i < G; ++i)
+            consensus_tile<TA, LAYOUT>(a, smem_raw + i * (a_bytes + b_bytes), gi[i], threadIdx.x < in_tile[i]);
+    }
 #pragma unroll
     for (int i = 0; i < G; ++i) {
         const unsigned char *image_a = smem_raw + i * (a_bytes + b_bytes);
@@ -249,7 +341,9 @@ cudaError_t launch_shuffle_async_tiles(const ShuffleArgs &args, const LaunchShap
     if (shape.threads <= 0)
         while (threads > 32 && per_thread * threads > 44 * 1024) threads >>= 1;
     const size_t smem = (per_thread * threads + 15) & ~static_cast<size_t>(15);
-    auto kernel = args.pop.layout == kLayoutNP ? shuffle_async_kernel<TA, TB, kLayoutNP, G> : shuffle_async_kernel<TA, TB, kLayoutPN, G>;
+    const bool np = args.pop.layout == kLayoutNP;
+    auto kernel = args.sq.slots ? (np ? shuffle_async_kernel<TA, TB, kLayoutNP, G, true> : shuffle_async_kernel<TA, TB, kLayoutPN, G, true>)
+                                : (np ? shuffle_async_kernel<TA, TB, kLayoutNP, G, false> : shuffle_async_kernel<TA, TB, kLayoutPN, G, false>);
     KernelFit fit;
     cudaError_t err = kernel_fit(reinterpret_cast<const void *>(kernel), threads, smem, &fit);
     if (err != cudaSuccess) return err;

@@ -149,6 +149,73 @@ def test_consensus_distance(N, dtype, layout):
     c.close()
 
 
+@pytest.mark.parametrize("layout", [0, 1])
+@pytest.mark.parametrize("N,dtype,opt_dtype,stacks", [(5, "f32", "f32", 2), (8, "bf16", "f32", 2), (13, "f32", None, 0),
+                                                     (3, "f32", "bf16", 1), (40, "f32", None, 0), (2, "bf16", None, 0)])
+def test_consensus_distance_inside_the_streaming_shuffle(N, dtype, opt_dtype, stacks, layout):
+    """wash_shuffle_consensus: the stacks end as after the plain shuffle (bit-exact against the
+    oracle), and the per-model, per-range sums equal the oracle's on the stack as it was before
+    the step (1e-12 relative: binary64 sums in another order) and the standalone kernel's."""
+    numel = [70001, 33, 7, 1, 4, 8, 5003, 2048, 30000]
+    p_layer = [0.3, 1.0, 0.5, 1.0, 0.0, 0.9, 0.05, 0.01, 0.002]
+    c = Case(N, numel, layout, dtype, opt_dtype, seed=N)
+    measured = c.host_opt if stacks == 1 else c.host          # the first stack of the launch
+    measured_code = B.WASH_STACK_OPT if stacks == 1 else B.WASH_STACK_PARAMS
+    bounds = [1, 3, 3, 7, 9]                                      # four ranges, one empty, tensor 0 in none
+    for step in (0, 1):
+        want = np.stack([oracle.consensus_sq(c.ora, measured, lo, hi) for lo, hi in zip(bounds[:-1], bounds[1:])])
+        alone = torch.zeros(len(bounds) - 1, N, dtype=torch.float64, device="cuda")
+        for r, (lo, hi) in enumerate(zip(bounds[:-1], bounds[1:])):
+            B.wash_consensus_sq(c.gpu.ctx, measured_code, lo, hi, alone[r])
+        out = torch.zeros(len(bounds) - 1, N, dtype=torch.float64, device="cuda")
+        B.wash_shuffle_consensus(c.gpu.ctx, stacks, step, 0.0, p_layer, seed=5, stats=c.stats_dev, tensor_bounds=bounds, dev_sq_out=out)
+        st = oracle.shuffle(c.ora, c.host_opt if stacks == 1 else c.host, p_layer, seed=5, step=step,
+                            stack2=c.host_opt if stacks == 2 else None)
+        c.assert_equal("step %d" % step)
+        got = out.cpu().numpy()
+        assert np.allclose(got, want, rtol=1e-12, atol=0), (got, want)
+        assert np.allclose(got, alone.cpu().numpy(), rtol=1e-12, atol=0)
+        assert (got[1] == 0).all() and (got[0] > 0).all()
+    # the whole model as one range, accumulated on top of what the array holds
+    whole = torch.full((1, N), 1.0, dtype=torch.float64, device="cuda")
+    want = oracle.consensus_sq(c.ora, measured)
+    B.wash_shuffle_consensus(c.gpu.ctx, stacks, 2, 0.0, p_layer, seed=5, tensor_bounds=[0, len(numel)], dev_sq_out=whole)
+    oracle.shuffle(c.ora, c.host_opt if stacks == 1 else c.host, p_layer, seed=5, step=2, stack2=c.host_opt if stacks == 2 else None)
+    c.assert_equal("whole model")
+    assert np.allclose(whole.cpu().numpy()[0] - 1.0, want, rtol=1e-11, atol=0)
+    for bad in ([0], [3, 2], [0, len(numel) + 1], list(range(10))):
+        with pytest.raises(B.WashError) as e:
+            B.wash_shuffle_consensus(c.gpu.ctx, stacks, 3, 0.1, None, tensor_bounds=bad, dev_sq_out=whole)
+        assert e.value.code == B.WASH_ERR_ARG
+    c.close()
+
+
+def test_consensus_inside_the_shuffle_at_config2_size():
+    """ResNet-18 population of config 2: per quarter of the tensor table (Fig. 4) from one pass."""
+    cfg = W.CONFIGS["cfg2_resnet18_n5"]
+    table = W.table_from_spec(cfg["table"])
+    N, T = cfg["N"], len(table)
+    c = Case(N, W.numels(table), 0, "f32", "f32", dense=W.init_population(table, N, seed=0), dense_opt=W.init_momentum(table, N, seed=1))
+    oracle.set_threads(oracle.max_threads())
+    bounds = [0, T // 4, T // 2, 3 * T // 4, T]
+    want = np.stack([oracle.consensus_sq(c.ora, c.host, lo, hi) for lo, hi in zip(bounds[:-1], bounds[1:])])
+    out = torch.zeros(4, N, dtype=torch.float64, device="cuda")
+    B.wash_shuffle_consensus(c.gpu.ctx, B.WASH_STACK_BOTH, 0, cfg["p"], None, seed=0, stats=c.stats_dev, tensor_bounds=bounds, dev_sq_out=out)
+    st = oracle.shuffle(c.ora, c.host, cfg["p"], seed=0, step=0, stack2=c.host_opt)
+    c.assert_equal("cfg2")
+    assert c.gpu_stats() == st
+    # The oracle adds a range's d terms one after the other in binary64 (a priori error d u,
+    # u = 2^-53, of a sum of positive terms); the kernel adds them in another order.  Hence
+    # the bar d u per range (2e-10 for the largest quarter), not the 1e-12 of the small cases.
+    got = out.cpu().numpy()
+    cum = np.concatenate([[0], np.cumsum(c.numel)])
+    for r, (lo, hi) in enumerate(zip(bounds[:-1], bounds[1:])):
+        d = float(cum[hi] - cum[lo])
+        assert np.allclose(got[r], want[r], rtol=max(1e-12, d * 2.0 ** -53), atol=0), (r, got[r], want[r])
+    oracle.set_threads(1)
+    c.close()
+
+
 def test_step_over_host_buffers():
     N, numel = 5, [3000, 17, 64]
     c = Case(N, numel, 0, "f32", "f32", seed=12)
