@@ -663,8 +663,7 @@ def run_sweep(args) -> None:
     torch.cuda.set_device(0)
     B.load()
     peak, _ = measured_peak()
-    modes = {"stream": B.WASH_MODE_STREAM, "sparse": B.WASH_MODE_SPARSE, "registers": B.WASH_MODE_STREAM_REGISTERS,
-             "staged": B.WASH_MODE_STREAM_STAGED}
+    modes = {"stream": B.WASH_MODE_STREAM, "sparse": B.WASH_MODE_SPARSE}
     stream = torch.cuda.current_stream()
     # integer-pipe ceiling of the mask: Philox blocks per second with no memory traffic
     chk = torch.zeros(1, dtype=torch.int32, device="cuda")

@@ -60,11 +60,7 @@ enum wash_mode {
                              coordinates; the stack travels global -> shared memory by
                              per-thread asynchronous copies (cp.async).  Default.            */
     WASH_MODE_SPARSE = 1, /* draws the mask first; touches only selected coordinates          */
-    WASH_MODE_STREAM_STAGED = 2,   /* as STREAM, staged by bulk asynchronous copies (TMA)     */
-    WASH_MODE_STREAM_REGISTERS = 3,/* as STREAM, the loads held in registers (kernels unrolled
-                                      for N in {2,3,4,5,6,8,10,12,16,20,24,32}; other N run
-                                      the default kernel)                                     */
-    WASH_MODE_AUTO = 4             /* SPARSE when the call's probabilities select, in expectation,
+    WASH_MODE_AUTO = 2             /* SPARSE when the call's probabilities select, in expectation,
                                       fewer than 3 % of the coordinates of an [N][padded_P] stack
                                       or 10 % of a [padded_P][N] stack, else STREAM (the measured
                                       crossovers on B200: in the second layout the N values of a
@@ -129,9 +125,7 @@ int wash_set_mode(wash_ctx *ctx, int32_t mode);
  * > 0 a persistent grid of SM count x min(blocks_per_sm, resident blocks per SM) blocks
  * that stride over the groups, < 0 one group of 4 coordinates per thread.  For
  * WASH_MODE_STREAM blocks_per_sm = 1 or 2 fixes the number of groups a thread takes
- * (default: 2 when a group of all models is at most 64 bytes, else 1).  For
- * WASH_MODE_STREAM_STAGED `threads` is the tile size in groups (32, 64, 128 or 256)
- * and blocks_per_sm the number of consumer teams per block. */
+ * (default: 2 when a group of all models is at most 64 bytes, else 1). */
 int wash_set_launch(wash_ctx *ctx, int32_t threads, int32_t blocks_per_sm);
 
 /* ---- the shuffling step ----------------------------------------------------------- */

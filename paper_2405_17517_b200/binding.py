@@ -23,7 +23,7 @@ WASH_F32, WASH_BF16 = 0, 1
 WASH_STACK_PARAMS, WASH_STACK_OPT, WASH_STACK_BOTH = 0, 1, 2
 WASH_MAX_CONSENSUS_RANGES = 8
 WASH_SCHEDULE_DECREASING, WASH_SCHEDULE_CONSTANT, WASH_SCHEDULE_INCREASING = 0, 1, 2
-WASH_MODE_STREAM, WASH_MODE_SPARSE, WASH_MODE_STREAM_STAGED, WASH_MODE_STREAM_REGISTERS, WASH_MODE_AUTO = 0, 1, 2, 3, 4
+WASH_MODE_STREAM, WASH_MODE_SPARSE, WASH_MODE_AUTO = 0, 1, 2
 WASH_OP_SHUFFLE, WASH_OP_EMA, WASH_OP_AVERAGE = 1, 2, 4
 WASH_MAX_N = 64
 WASH_ALIGN_ELEMS = 8

@@ -2,9 +2,9 @@
 
     python -m paper_2405_17517_b200.build [--force] [--verbose]
 
-wash_inst.cu is compiled once per population size listed in csrc/wash_nlist.h (plus
-once for the run-time-N kernels); the objects are compiled in parallel and linked with
-the C ABI into paper_2405_17517_b200/libwash.so.
+wash_inst.cu (the dense operators) is compiled once per population size listed in
+csrc/wash_nlist.h (plus once for run-time N); the objects are compiled in parallel and
+linked with the C ABI into paper_2405_17517_b200/libwash.so.
 """
 from __future__ import annotations
 
@@ -63,7 +63,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
     os.makedirs(BUILD, exist_ok=True)
     jobs = [(os.path.join(CSRC, "wash_api.cu"), os.path.join(BUILD, "wash_api.o"), [], verbose),
             (os.path.join(CSRC, "wash_dispatch.cu"), os.path.join(BUILD, "wash_dispatch.o"), [], verbose)]
-    for name in ("wash_noalloc", "wash_tma", "wash_exchange"):
+    for name in ("wash_noalloc", "wash_shuffle", "wash_exchange"):
         jobs.append((os.path.join(CSRC, name + ".cu"), os.path.join(BUILD, name + ".o"), [], verbose))
     for n in [0] + population_sizes():
         jobs.append((os.path.join(CSRC, "wash_inst.cu"), os.path.join(BUILD, "wash_inst_n%d.o" % n), ["-DWASH_N=%d" % n], verbose))

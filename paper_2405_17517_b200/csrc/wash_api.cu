@@ -447,7 +447,7 @@ int wash_bind(wash_ctx *ctx, int32_t stack, int32_t dtype, void *dev_ptr, int64_
 int wash_set_mode(wash_ctx *ctx, int32_t mode)
 {
     if (!ctx) return fail(WASH_ERR_ARG, "ctx is NULL");
-    if (mode < WASH_MODE_STREAM || mode > WASH_MODE_AUTO) return fail(WASH_ERR_ARG, "unknown mode %d", mode);
+    if (mode != WASH_MODE_STREAM && mode != WASH_MODE_SPARSE && mode != WASH_MODE_AUTO) return fail(WASH_ERR_ARG, "unknown mode %d", mode);
     ctx->mode = mode;
     return WASH_OK;
 }
@@ -587,7 +587,7 @@ int wash_step_host(wash_ctx *ctx, int32_t ops, void *host_params, void *host_opt
     // range to the device, the kernels on the previous one and the copy of the one before
     // back to the host overlap (the PCIe link is full duplex, and the draws are keyed by
     // global coordinates, so a range can be processed on its own).
-    if (ctx->mode != WASH_MODE_STREAM_STAGED && ctx->n_groups >= (1u << 18)) {
+    if (ctx->n_groups >= (1u << 18)) {
         if (!ctx->copy_in) {
             if ((err = cudaStreamCreateWithFlags(&ctx->copy_in, cudaStreamNonBlocking)) != cudaSuccess ||
                 (err = cudaStreamCreateWithFlags(&ctx->copy_out, cudaStreamNonBlocking)) != cudaSuccess)
@@ -969,9 +969,8 @@ int wash_check(wash_ctx *ctx, void *stream_v)
     if (err != cudaSuccess) return cuda_fail(err, "reading the status word");
     if (status) {
         cudaMemsetAsync(ctx->status_dev, 0, sizeof(uint32_t), stream);
-        return fail(WASH_ERR_DEVICE_CHECK, "device status 0x%x:%s%s%s", status,
+        return fail(WASH_ERR_DEVICE_CHECK, "device status 0x%x:%s%s", status,
                     (status & 1u) ? " a group outside its segment table;" : "",
-                    (status & 2u) ? " a bounded wait of the staged shuffle ran out;" : "",
                     (status & 4u) ? " an exchange step needed more slots than the staging buffers hold;" : "");
     }
     return WASH_OK;

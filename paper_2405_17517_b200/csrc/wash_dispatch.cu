@@ -6,31 +6,16 @@
 
 namespace wash {
 
-#define WASH_DECL(n)                                                                                     \
-    cudaError_t launch_shuffle_stream_n##n(const ShuffleArgs &, int, int, const LaunchShape &, cudaStream_t, bool *); \
-    cudaError_t launch_reduce_n##n(const ReduceArgs &, int, int, int, const LaunchShape &, cudaStream_t, bool *);
+#define WASH_DECL(n) cudaError_t launch_reduce_n##n(const ReduceArgs &, int, int, int, const LaunchShape &, cudaStream_t, bool *);
 WASH_N_LIST(WASH_DECL)
 #undef WASH_DECL
 cudaError_t launch_shuffle_sparse(const ShuffleArgs &, int, int, const LaunchShape &, cudaStream_t, bool *);
-cudaError_t launch_shuffle_staged(const ShuffleArgs &, int, int, const LaunchShape &, cudaStream_t, bool *);
-cudaError_t launch_shuffle_async_staged(const ShuffleArgs &, int, int, const LaunchShape &, cudaStream_t, bool *);
+cudaError_t launch_shuffle_stream(const ShuffleArgs &, int, int, const LaunchShape &, cudaStream_t, bool *);
 cudaError_t launch_reduce_n0(const ReduceArgs &, int, int, int, const LaunchShape &, cudaStream_t, bool *);
 
 static std::atomic<uint64_t> g_launches{0};
 void count_launch() { g_launches.fetch_add(1, std::memory_order_relaxed); }
 uint64_t launch_count() { return g_launches.load(std::memory_order_relaxed); }
-
-bool has_unrolled_kernels(int N)
-{
-    switch (N) {
-#define WASH_CASE(n) case n:
-        WASH_N_LIST(WASH_CASE)
-#undef WASH_CASE
-        return true;
-    default:
-        return false;
-    }
-}
 
 // Sums the partial statistics into the caller's counters and zeroes them again.
 // (Warp shuffles, then eight partial sums: 64-bit atomics on one shared-memory word are
@@ -115,18 +100,7 @@ static cudaError_t launch_shuffle_kernel(const ShuffleArgs &args, int a_dtype, i
                                          const LaunchShape &shape, cudaStream_t stream, bool *supported)
 {
     if (mode == kModeSparse) return launch_shuffle_sparse(args, a_dtype, b_dtype, shape, stream, supported);
-    if (mode == kModeStreamStaged) return launch_shuffle_staged(args, a_dtype, b_dtype, shape, stream, supported);
-    if (mode == kModeStreamRegisters) {
-        switch (args.pop.N) {
-#define WASH_CASE(n) case n: return launch_shuffle_stream_n##n(args, a_dtype, b_dtype, shape, stream, supported);
-            WASH_N_LIST(WASH_CASE)
-#undef WASH_CASE
-        default:
-            break;   // no unrolled kernel for this N: the default kernel gives the same bits
-        }
-    }
-    // default streaming kernel: staged through shared memory with cp.async, any N
-    return launch_shuffle_async_staged(args, a_dtype, b_dtype, shape, stream, supported);
+    return launch_shuffle_stream(args, a_dtype, b_dtype, shape, stream, supported);
 }
 
 cudaError_t launch_shuffle(const ShuffleArgs &args, int a_dtype, int b_dtype, int mode,

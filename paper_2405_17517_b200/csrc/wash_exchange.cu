@@ -25,8 +25,7 @@
 #include "wash_device.cuh"
 #include "wash_launch.cuh"
 #include "wash_warp_tiles.cuh"
-#include "wash_shuffle_tma.cuh"     // draw_permutation_u8
-#include "wash_shuffle_async.cuh"   // draw_permutation_packed
+#include "wash_permutation.cuh"
 
 namespace wash {
 

@@ -1,7 +1,6 @@
-// One translation unit per population size: compiled with -DWASH_N=<n> for every n of
-// WASH_N_LIST (unrolled kernels) and with -DWASH_N=0 (run-time-N kernels, which include
-// the reduce kernels for population sizes without an unrolled instantiation).
-#include "wash_shuffle.cuh"
+// One translation unit per population size for the dense operators (EMA, average, PAPA-all,
+// consensus distance): compiled with -DWASH_N=<n> for every n of WASH_N_LIST (loops over the
+// models unrolled) and with -DWASH_N=0 (run-time N, for the other population sizes).
 #include "wash_reduce.cuh"
 
 #ifndef WASH_N
@@ -12,14 +11,6 @@
 #define WASH_CAT(a, b) WASH_CAT2(a, b)
 
 namespace wash {
-
-#if WASH_N > 0
-cudaError_t WASH_CAT(launch_shuffle_stream_n, WASH_N)(const ShuffleArgs &args, int a_dtype, int b_dtype,
-                                                      const LaunchShape &shape, cudaStream_t stream, bool *supported)
-{
-    return launch_shuffle_n<WASH_N, true>(args, a_dtype, b_dtype, shape, stream, supported);
-}
-#endif
 
 cudaError_t WASH_CAT(launch_reduce_n, WASH_N)(const ReduceArgs &args, int op, int dtype, int out_dtype,
                                               const LaunchShape &shape, cudaStream_t stream, bool *supported)

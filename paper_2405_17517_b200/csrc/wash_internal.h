@@ -9,7 +9,7 @@ constexpr int kMaxN = 64;          // largest population (WASH_MAX_N)
 constexpr int kTileShift = 8;      // lookup tile = 256 groups = 1024 coordinates
 constexpr int kDtypeF32 = 0, kDtypeBF16 = 1, kDtypeNone = -1;
 constexpr int kLayoutNP = 0, kLayoutPN = 1;
-constexpr int kModeStream = 0, kModeSparse = 1, kModeStreamStaged = 2, kModeStreamRegisters = 3;
+constexpr int kModeStream = 0, kModeSparse = 1;
 
 // One row of a stack is cut into groups of 4 consecutive elements; a group never
 // straddles two tensors because tensors start on multiples of 8 elements.
@@ -143,9 +143,6 @@ cudaError_t launch_reduce(const ReduceArgs &args, int op, int dtype, int out_dty
 cudaError_t launch_sq_flush(const SqArgs &sq, int N, double *out, cudaStream_t stream);
 
 cudaError_t launch_philox_probe(unsigned long long n_blocks, uint64_t seed, uint32_t *checksum, cudaStream_t stream);
-
-// true if a streaming shuffle kernel was compiled for this population size
-bool has_unrolled_kernels(int N);
 
 void count_launch();
 

@@ -19,7 +19,7 @@
 #pragma once
 #include "wash_device.cuh"
 #include "wash_launch.cuh"
-#include "wash_shuffle_tma.cuh"   // draw_permutation_u8
+#include "wash_permutation.cuh"
 
 namespace wash {
 
@@ -82,24 +82,6 @@ __device__ __forceinline__ uint32_t image_value(const unsigned char *image, int 
     return reinterpret_cast<const uint16_t *>(image)[elem];
 }
 
-// pi for coordinate i with pi(n) in nibble n of the result (N <= 16): the Fisher-Yates of
-// draw_permutation_u8 on a register instead of a shared-memory column.
-__device__ __forceinline__ uint64_t draw_permutation_packed(int n_models, uint32_t i, uint32_t tensor, uint32_t step_lo,
-                                                            uint32_t step_hi8, const PhiloxKeys &keys)
-{
-    uint64_t perm = 0xFEDCBA9876543210ull;
-    Philox4 w{0, 0, 0, 0};
-    for (int k = n_models - 1, m = 0; k >= 1; --k, ++m) {
-        if ((m & 3) == 0) w = philox4x32_10(i, tensor, step_lo, step_hi8 | (1u + (static_cast<uint32_t>(m) >> 2)), keys);
-        const uint32_t r = w.x;
-        w.x = w.y; w.y = w.z; w.z = w.w;
-        const uint32_t sk = 4u * k, sj = 4u * __umulhi(r, static_cast<uint32_t>(k + 1));
-        const uint64_t diff = ((perm >> sk) ^ (perm >> sj)) & 15ull;   // swap nibbles k and j
-        perm ^= (diff << sk) | (diff << sj);
-    }
-    return perm;
-}
-
 // Serves the selected coordinates of one tile of T groups (one group per thread): the warp's
 // selected coordinates are listed in shared memory and dealt out to the lanes 32 at a time:
 // with a few selected coordinates per warp (p around 0.01-0.1) one round serves them all,
@@ -140,9 +122,6 @@ __device__ __forceinline__ void serve_tile(const ShuffleArgs &a, const unsigned 
         uint64_t perm = 0;
         if (n_models <= 16) perm = draw_permutation_packed(n_models, 4u * cgroup + c, tensor, a.step_lo, a.step_hi8, a.keys);
         else draw_permutation_u8(s_perm, T_, n_models, 4u * cgroup + c, tensor, a.step_lo, a.step_hi8, a.keys);
-        auto source_of = [&](int n) -> int {
-            return n_models <= 16 ? static_cast<int>((perm >> (4 * n)) & 15ull) : static_cast<int>(s_perm[n * T_]);
-        };
         // model n's value of this coordinate sits at out0 + n*out_step in the stack and at
         // element img0 + n*img_step of the image: no multiplication left inside the loop
         const long long out_step = LAYOUT == kLayoutNP ? a.pop.padded_P : 1;
@@ -150,8 +129,9 @@ __device__ __forceinline__ void serve_tile(const ShuffleArgs &a, const unsigned 
         const uint32_t img_step = LAYOUT == kLayoutNP ? T_ * 4u : 1u;
         const uint32_t img0 = LAYOUT == kLayoutNP ? t_owner * 4u + c : (4u * t_owner + c) * n_models;
         long long out = out0;
-        for (int n = 0; n < n_models; ++n, out += out_step) {
-            const uint32_t src = static_cast<uint32_t>(source_of(n));
+        uint64_t rest = perm;   // nibble n on top of the low end when model n's turn comes
+        for (int n = 0; n < n_models; ++n, out += out_step, rest >>= 4) {
+            const uint32_t src = n_models <= 16 ? static_cast<uint32_t>(rest) & 15u : static_cast<uint32_t>(s_perm[n * T_]);
             if (src == static_cast<uint32_t>(n)) continue;
             const uint32_t from = img0 + src * img_step;
             TA::store_elem(a.a, out, TA::kBytes == 4 ? reinterpret_cast<const uint32_t *>(image_a)[from]

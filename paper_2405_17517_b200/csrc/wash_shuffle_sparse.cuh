@@ -13,8 +13,7 @@
 #include "wash_device.cuh"
 #include "wash_launch.cuh"
 #include "wash_warp_tiles.cuh"
-#include "wash_shuffle_tma.cuh"     // draw_permutation_u8
-#include "wash_shuffle_async.cuh"   // draw_permutation_packed
+#include "wash_permutation.cuh"
 
 namespace wash {
 
@@ -56,21 +55,24 @@ __global__ void __launch_bounds__(kSparseThreads, 4) shuffle_sparse_kernel(const
             uint64_t perm = 0;
             if (n_models <= 16) perm = draw_permutation_packed(n_models, coord, gi.tensor_id, a.step_lo, a.step_hi8, a.keys);
             else draw_permutation_u8(s_perm, kSparseThreads, n_models, coord, gi.tensor_id, a.step_lo, a.step_hi8, a.keys);
-            auto source_of = [&](int n) -> int {
-                return n_models <= 16 ? static_cast<int>((perm >> (4 * n)) & 15ull) : static_cast<int>(s_perm[n * kSparseThreads]);
+            // nibble n of `perm` (N <= 16) or byte n of the column is the model whose value model n takes
+            auto source_of = [&](int n, uint64_t rest) -> int {
+                return n_models <= 16 ? static_cast<int>(static_cast<uint32_t>(rest) & 15u) : static_cast<int>(s_perm[n * kSparseThreads]);
             };
             // all N old values first (the exchange is in place), then the moved ones back
             for (int n = 0; n < n_models; ++n) s_col[n * kSparseThreads] = TA::load_elem(a.a, elem_index<LAYOUT>(a.pop, n, e));
-            for (int n = 0; n < n_models; ++n) {
-                const int src = source_of(n);
+            uint64_t rest = perm;
+            for (int n = 0; n < n_models; ++n, rest >>= 4) {
+                const int src = source_of(n, rest);
                 if (src == n) continue;
                 TA::store_elem(a.a, elem_index<LAYOUT>(a.pop, n, e), s_col[src * kSparseThreads]);
                 ++moved;
             }
             if constexpr (kHasB) {
                 for (int n = 0; n < n_models; ++n) s_col[n * kSparseThreads] = TB::load_elem(a.b, elem_index<LAYOUT>(a.pop, n, e));
-                for (int n = 0; n < n_models; ++n) {
-                    const int src = source_of(n);
+                rest = perm;
+                for (int n = 0; n < n_models; ++n, rest >>= 4) {
+                    const int src = source_of(n, rest);
                     if (src != n) TB::store_elem(a.b, elem_index<LAYOUT>(a.pop, n, e), s_col[src * kSparseThreads]);
                 }
             }
