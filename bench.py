@@ -790,6 +790,93 @@ def run_exchange(args) -> None:
         torch.cuda.empty_cache()
 
 
+def run_exchange_ranks(args, rank: int, world: int, local_rank: int) -> None:
+    """The paper's own deployment: one model per rank, the ranks of the process group being the
+    population.  Every rank builds an ExchangeWorker on its model's row (and momentum), runs
+    --steps steps (plan, send by peer stores, barrier, receive) and rank 0 prints one JSON line:
+    step time (CUDA events on the launching stream, max over ranks), values and bytes a rank
+    receives per step, and whether the plan's slot counts equal the oracle's for the last step.
+    With one GPU per rank the group is NCCL and the barrier between send and receive is an
+    all-reduce on the stream; when the ranks have to share a device the group is gloo and the
+    barrier is on the host (a functional stand-in, not a measurement of the link)."""
+    import torch
+    import torch.distributed as dist
+    from paper_2405_17517_b200 import binding as B
+    from paper_2405_17517_b200.exchange import ExchangeWorker
+
+    if world < 2:
+        raise SystemExit("--exchange-ranks needs a population: launch with torchrun, --nproc-per-node >= 2")
+    own_gpu = torch.cuda.device_count() >= world
+    device = local_rank if own_gpu else 0
+    torch.cuda.set_device(device)
+    if own_gpu:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", device))
+    else:
+        dist.init_process_group("gloo")
+    B.load()
+    wl = Workload(args.workload)
+    N = world                                   # the population is the process group
+    stream = torch.cuda.current_stream()
+    ctx_probe = B.wash_create(N, wl.numel, B.WASH_LAYOUT_NP, device)
+    P = B.wash_stack_elems(ctx_probe, wl.T)[0]
+    B.wash_destroy(ctx_probe)
+    gen = torch.Generator(device="cuda").manual_seed(SEED + 31 * rank)
+    row = (torch.randn(P, generator=gen, device="cuda") * 0.05).to(torch.bfloat16 if wl.bf16 else torch.float32)
+    opt = torch.randn(P, generator=gen, device="cuda") * 1e-3 if wl.opt else None
+    p_layer = B.wash_layer_probs(wl.T, wl.p, B.WASH_SCHEDULE_DECREASING) if wl.schedule == "decreasing" else None
+    p_eff = wl.p if p_layer is None else float((p_layer * wl.numel).sum() / wl.P)
+    capacity = max(1 << 14, int(4 * p_eff * wl.P))
+    worker = ExchangeWorker(wl.numel, row, opt, capacity=capacity, device=device)
+    stats = torch.zeros(2, dtype=torch.int64, device="cuda")
+
+    def fence():
+        torch.cuda.synchronize()
+        dist.barrier()
+
+    for w in range(args.warmup):
+        worker.step(w, wl.p, p_layer, SEED)
+    fence()
+    worker.check()
+    K = args.steps
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(K + 1)]
+    t0 = time.perf_counter()
+    ev[0].record(stream)
+    for k in range(K):
+        worker.step(args.warmup + k, wl.p, p_layer, SEED, stats)
+        ev[k + 1].record(stream)
+    fence()
+    wall = time.perf_counter() - t0
+    worker.check()
+    per_step = np.array([ev[k].elapsed_time(ev[k + 1]) for k in range(K)])
+    need, selected = B.wash_exchange_counts(worker.ctx, N)          # the plan of the last step
+    t = torch.tensor([float(np.median(per_step)), float(per_step.min()), wall / K * 1e3], dtype=torch.float64,
+                     device="cuda" if own_gpu else "cpu")
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    c = torch.tensor([int(stats[1])], dtype=torch.int64, device="cuda" if own_gpu else "cpu")
+    dist.all_reduce(c, op=dist.ReduceOp.SUM)
+    if rank == 0:
+        import oracle
+        offsets, padded_P = W.padded_offsets(wl.numel)
+        ora = oracle.Population(N, wl.numel, offsets, padded_P, oracle.LAYOUT_NP)
+        oracle.set_threads(oracle.max_threads())
+        want_need, want_sel = oracle.exchange_counts(ora, wl.p if p_layer is None else p_layer, SEED, args.warmup + K - 1)
+        received = int(c[0]) / K / N                       # values one rank receives per step
+        elem = wl.E + wl.E_opt
+        step_ms = float(t[0]) if own_gpu else float(t[2])  # host-ordered steps are not bracketed by stream events alone
+        print(json.dumps({
+            "arm": "exchange-ranks", "workload": wl.name, "ranks": N, "backend": "nccl" if own_gpu else "gloo (ranks share device 0, barrier on the host)",
+            "steps": K, "warmup": args.warmup, "step_us": step_ms * 1e3, "step_us_min": float(t[1]) * 1e3 if own_gpu else None,
+            "selected_coords_per_step": selected, "values_received_per_rank_per_step": received,
+            "expected_values_per_rank_per_step": p_eff * wl.P * (N - 1) / N,
+            "link_bytes_in_per_rank_per_step": received * elem, "model_bytes_per_rank": wl.P * elem,
+            "counts_match_oracle": bool(list(need) == [int(x) for x in want_need] and selected == want_sel),
+            "staging_capacity_elems": worker.capacity,
+            "timing": "CUDA events on the launching stream per step, median, max over ranks" if own_gpu else "wall clock per step, max over ranks",
+        }), flush=True)
+    worker.close()
+    dist.destroy_process_group()
+
+
 def main() -> None:
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -810,6 +897,8 @@ def main() -> None:
     ap.add_argument("--sweep-layout", default="", choices=["", "np", "pn"])
     ap.add_argument("--exchange-warm", action="store_true", help="with --exchange: no L2 flush between steps")
     ap.add_argument("--exchange", action="store_true", help="time one worker of the one-model-per-device form (JSON line per workload)")
+    ap.add_argument("--exchange-ranks", action="store_true",
+                    help="under torchrun: the ranks are the population, one model per rank, steps through ExchangeWorker (one JSON line)")
     args = ap.parse_args()
     args.workload_given = any(a == "--workload" or a.startswith("--workload=") for a in sys.argv[1:])
     if args.warmup < 3 and args.impl == "ours":
@@ -822,6 +911,9 @@ def main() -> None:
         return
     if args.exchange:
         run_exchange(args)
+        return
+    if args.exchange_ranks:
+        run_exchange_ranks(args, rank, world, local_rank)
         return
     if args.impl == "reference":
         run_reference(args, rank, world)

@@ -14,14 +14,19 @@
 //   [N][P]: vector j of thread t at (j*T + t) * vec      (T = threads per block); fp32 vectors
 //           are copied by their own thread, bf16 rows cooperatively in 16-byte pieces
 //   [P][N]: the block's T*4N elements are contiguous in global memory and are copied
-//           as they lie, vector k*T + t by thread t; thread t's coordinate c of model n
-//           is element (4t + c)*N + n of that image.
+//           vector by vector, vector k*T + t by thread t; a group's 4N elements stay together
+//           and, when N is even, are followed by one vector of padding, so that a group spans
+//           an odd number of vectors and the lanes of a warp (one group each) fall into
+//           different shared-memory banks: thread t's coordinate c of model n is element
+//           t*pn_group_elems(N) + c*N + n of that image.
 #pragma once
 #include "wash_device.cuh"
 #include "wash_launch.cuh"
 #include "wash_permutation.cuh"
 
 namespace wash {
+
+constexpr uint32_t kDenseMinSelected = 64;   // selected coordinates of a warp's 128 from which every lane serves its own group
 
 template <int BYTES>
 __device__ __forceinline__ void cp_async(uint32_t dst_smem, const void *src)
@@ -34,6 +39,12 @@ __device__ __forceinline__ void cp_async(uint32_t dst_smem, const void *src)
 __device__ __forceinline__ void cp_async_wait_all()
 {
     asm volatile("cp.async.wait_all;" ::: "memory");
+}
+
+// elements a group takes in the [P][N] image: its 4N values, plus one vector of padding when N is even
+__device__ __forceinline__ uint32_t pn_group_elems(int n_models)
+{
+    return 4u * static_cast<uint32_t>(n_models) + ((n_models & 1) ? 0u : 4u);
 }
 
 // Starts the copies of one stack for this thread's block position; returns nothing.
@@ -65,9 +76,17 @@ __device__ __forceinline__ void async_fetch(uint32_t image, void *base, const Po
             for (int j = 0; j < n_models; ++j, src += row_bytes, dst += T_ * kVec) cp_async<kVec>(dst, src);
         }
     } else {
-        const uint32_t vecs = groups_in_block * n_models;
+        // vector k is vector j = k % N of group k / N; the pair is advanced without dividing again
+        const uint32_t vecs = groups_in_block * n_models, N_ = static_cast<uint32_t>(n_models);
+        const uint32_t stride = pn_group_elems(n_models) / 4u, dq = T_ / N_, dr = T_ - dq * N_;
         const char *src = static_cast<const char *>(base) + 4ll * static_cast<long long>(g_block) * n_models * T::kBytes;
-        for (uint32_t k = t; k < vecs; k += T_) cp_async<kVec>(image + k * kVec, src + static_cast<size_t>(k) * kVec);
+        uint32_t group = t / N_, j = t - group * N_;
+        for (uint32_t k = t; k < vecs; k += T_) {
+            cp_async<kVec>(image + (group * stride + j) * kVec, src + static_cast<size_t>(k) * kVec);
+            group += dq;
+            j += dr;
+            if (j >= N_) { j -= N_; ++group; }
+        }
     }
 }
 
@@ -77,9 +96,90 @@ __device__ __forceinline__ uint32_t image_value(const unsigned char *image, int 
 {
     const uint32_t T_ = blockDim.x;
     const uint32_t elem = LAYOUT == kLayoutNP ? (static_cast<uint32_t>(n) * T_ + t) * 4u + c
-                                              : (4u * t + c) * n_models + n;
+                                              : t * pn_group_elems(n_models) + static_cast<uint32_t>(c * n_models + n);
     if (T::kBytes == 4) return reinterpret_cast<const uint32_t *>(image)[elem];
     return reinterpret_cast<const uint16_t *>(image)[elem];
+}
+
+// Dense selection: every lane serves its own group.  It draws the permutations of its selected
+// coordinates (identity for the others) and writes the group back as whole vectors -- model n's
+// vector takes coordinate c from model pi_c(n) -- instead of one 4-byte store per moved value:
+// no list, no dealing, a quarter of the store instructions, and full 16-byte pieces of a sector.
+// An unselected coordinate of such a group is rewritten with the bits it already has.  PERM is
+// uint32_t (N <= 8) or uint64_t (N <= 16); the caller has checked that the group is whole.
+template <class TA, class TB, int LAYOUT, class PERM>
+__device__ __forceinline__ void serve_group_dense(const ShuffleArgs &a, const unsigned char *image_a, const unsigned char *image_b,
+                                                  uint64_t g_block, uint32_t sel, const GroupInfo &gi, uint32_t &selected, uint32_t &moved)
+{
+    constexpr bool kHasB = TB::kCode != kDtypeNone;
+    constexpr PERM kIdentity = static_cast<PERM>(0xFEDCBA9876543210ull), kOnes = static_cast<PERM>(0x1111111111111111ull);
+    const int n_models = a.pop.N;
+    const uint32_t T_ = blockDim.x, t = threadIdx.x;
+    PERM perm[4];
+#pragma unroll
+    for (int c = 0; c < 4; ++c) {
+        perm[c] = kIdentity;
+        if ((sel >> c) & 1u) {
+            if (sizeof(PERM) == 4) perm[c] = static_cast<PERM>(draw_permutation_packed32(n_models, 4u * gi.cgroup + c, gi.tensor_id, a.step_lo, a.step_hi8, a.keys));
+            else perm[c] = static_cast<PERM>(draw_permutation_packed(n_models, 4u * gi.cgroup + c, gi.tensor_id, a.step_lo, a.step_hi8, a.keys));
+            // values that leave their model: the nibbles of pi that differ from the identity's
+            PERM x = perm[c] ^ kIdentity;
+            x = (x | (x >> 1) | (x >> 2) | (x >> 3)) & kOnes;
+            moved += sizeof(PERM) == 4 ? __popc(static_cast<uint32_t>(x)) : __popcll(static_cast<uint64_t>(x));
+            ++selected;
+        }
+    }
+    auto value_a = [&](uint32_t from) -> uint32_t {
+        return TA::kBytes == 4 ? reinterpret_cast<const uint32_t *>(image_a)[from] : reinterpret_cast<const uint16_t *>(image_a)[from];
+    };
+    auto value_b = [&](uint32_t from) -> uint32_t {
+        return TB::kBytes == 4 ? reinterpret_cast<const uint32_t *>(image_b)[from] : reinterpret_cast<const uint16_t *>(image_b)[from];
+    };
+    if (LAYOUT == kLayoutNP) {
+        // model n's vector of the group: one row further in the stack per n
+        char *out_a = group_vec_ptr<TA, LAYOUT>(a.a, a.pop, g_block + t, 0);
+        char *out_b = kHasB ? group_vec_ptr<TB, LAYOUT>(a.b, a.pop, g_block + t, 0) : nullptr;
+        const size_t row_a = static_cast<size_t>(a.pop.padded_P) * TA::kBytes, row_b = static_cast<size_t>(a.pop.padded_P) * TB::kBytes;
+        const uint32_t img_step = T_ * 4u, img0 = t * 4u;
+        for (int n = 0; n < n_models; ++n, out_a += row_a, out_b += row_b) {
+            uint32_t wa[4], wb[4];
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+                const uint32_t from = (static_cast<uint32_t>(perm[c]) & 15u) * img_step + img0 + c;
+                perm[c] >>= 4;
+                wa[c] = value_a(from);
+                if constexpr (kHasB) wb[c] = value_b(from);
+            }
+            TA::store_group(out_a, TA::pack(wa[0], wa[1], wa[2], wa[3]));
+            if constexpr (kHasB) TB::store_group(out_b, TB::pack(wb[0], wb[1], wb[2], wb[3]));
+        }
+    } else {
+        // the group's 4N elements are contiguous: element c*N + n is (coordinate c, model n)
+        char *out_a = group_vec_ptr<TA, LAYOUT>(a.a, a.pop, g_block + t, 0);
+        char *out_b = kHasB ? group_vec_ptr<TB, LAYOUT>(a.b, a.pop, g_block + t, 0) : nullptr;
+        const uint32_t img0 = t * pn_group_elems(n_models);
+        PERM rest = perm[0];
+        uint32_t base = img0;   // image element of (coordinate c, model 0)
+        int n = 0, c = 0;
+        for (int j = 0; j < n_models; ++j) {
+            uint32_t wa[4], wb[4];
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                const uint32_t from = base + (static_cast<uint32_t>(rest) & 15u);
+                rest >>= 4;
+                wa[q] = value_a(from);
+                if constexpr (kHasB) wb[q] = value_b(from);
+                if (++n == n_models) {
+                    n = 0;
+                    ++c;
+                    base += static_cast<uint32_t>(n_models);
+                    rest = c == 1 ? perm[1] : (c == 2 ? perm[2] : perm[3]);
+                }
+            }
+            TA::store_group(out_a + static_cast<size_t>(j) * (TA::kBytes * 4), TA::pack(wa[0], wa[1], wa[2], wa[3]));
+            if constexpr (kHasB) TB::store_group(out_b + static_cast<size_t>(j) * (TB::kBytes * 4), TB::pack(wb[0], wb[1], wb[2], wb[3]));
+        }
+    }
 }
 
 // Serves the selected coordinates of one tile of T groups (one group per thread): the warp's
@@ -97,6 +197,18 @@ __device__ __forceinline__ void serve_tile(const ShuffleArgs &a, const unsigned 
     const uint32_t lane = threadIdx.x & 31u, warp_base = threadIdx.x & ~31u;
     if (!__any_sync(0xFFFFFFFFu, sel != 0)) return;   // most warps have nothing selected at small p
     const uint32_t mine = __popc(sel);
+    // Half of the warp's coordinates or more selected: dealing them out would take two rounds or
+    // more, in each of which a lane draws one permutation and stores 4-byte values; every lane
+    // serving its own group costs less from there on (measured crossover near 64 of 128).
+    if (n_models <= 16 && __reduce_add_sync(0xFFFFFFFFu, mine) >= kDenseMinSelected &&
+        __all_sync(0xFFFFFFFFu, sel == 0 || gi.valid == 4)) {
+        if (sel) {
+            const uint64_t g_tile = g_block;
+            if (n_models <= 8) serve_group_dense<TA, TB, LAYOUT, uint32_t>(a, image_a, image_b, g_tile, sel, gi, selected, moved);
+            else serve_group_dense<TA, TB, LAYOUT, uint64_t>(a, image_a, image_b, g_tile, sel, gi, selected, moved);
+        }
+        return;
+    }
     uint32_t upto = mine;   // inclusive prefix sum over the lanes
 #pragma unroll
     for (int d = 1; d < 32; d <<= 1) {
@@ -127,7 +239,7 @@ __device__ __forceinline__ void serve_tile(const ShuffleArgs &a, const unsigned 
         const long long out_step = LAYOUT == kLayoutNP ? a.pop.padded_P : 1;
         const long long out0 = LAYOUT == kLayoutNP ? e : e * n_models;
         const uint32_t img_step = LAYOUT == kLayoutNP ? T_ * 4u : 1u;
-        const uint32_t img0 = LAYOUT == kLayoutNP ? t_owner * 4u + c : (4u * t_owner + c) * n_models;
+        const uint32_t img0 = LAYOUT == kLayoutNP ? t_owner * 4u + c : t_owner * pn_group_elems(n_models) + c * n_models;
         long long out = out0;
         uint64_t rest = perm;   // nibble n on top of the low end when model n's turn comes
         for (int n = 0; n < n_models; ++n, out += out_step, rest >>= 4) {
@@ -244,8 +356,9 @@ __global__ void __launch_bounds__(256, 5) shuffle_async_kernel(const __grid_cons
     const int n_models = a.pop.N;
     const uint32_t T_ = blockDim.x;
     // G pairs of images of the two stacks, then the warps' lists, then the permutation columns
-    const size_t a_bytes = static_cast<size_t>(n_models) * T_ * TA::kBytes * 4;
-    const size_t b_bytes = kHasB ? static_cast<size_t>(n_models) * T_ * TB::kBytes * 4 : 0;
+    const size_t group_elems = LAYOUT == kLayoutPN ? pn_group_elems(n_models) : 4u * static_cast<size_t>(n_models);
+    const size_t a_bytes = group_elems * T_ * TA::kBytes;
+    const size_t b_bytes = kHasB ? group_elems * T_ * TB::kBytes : 0;
     uint8_t *s_list = smem_raw + G * (a_bytes + b_bytes);   // 128 bytes per warp
     uint8_t *s_perm = s_list + 4 * T_ + threadIdx.x;        // column [n][T], used when N > 16
 
@@ -271,15 +384,14 @@ __global__ void __launch_bounds__(256, 5) shuffle_async_kernel(const __grid_cons
         if (threadIdx.x < in_tile[i]) {
             gi[i] = find_group(a.pop, static_cast<uint32_t>(g_first + static_cast<uint64_t>(i) * T_ + threadIdx.x), a.status);
             if (gi[i].thr != 0 && gi[i].valid != 0) {
-                const Philox4 w = philox4x32_10(gi[i].cgroup, gi[i].tensor_id, a.step_lo, a.step_hi8, a.keys);
-                // word < thr with thr in [0, 2^32]: a 32-bit compare, or always when thr is 2^32
-                const uint32_t thr_lo = static_cast<uint32_t>(gi[i].thr);
-                const bool always = (gi[i].thr >> 32) != 0;
-                uint32_t m = 0;
-                m |= (w.x < thr_lo || always) ? 1u : 0u;
-                m |= (w.y < thr_lo || always) ? 2u : 0u;
-                m |= (w.z < thr_lo || always) ? 4u : 0u;
-                m |= (w.w < thr_lo || always) ? 8u : 0u;
+                // word < thr with thr in [0, 2^32]: a 32-bit compare; a threshold of 2^32 selects
+                // whatever the word is, so the block is not drawn at all
+                uint32_t m = 0xFu;
+                if ((gi[i].thr >> 32) == 0) {
+                    const Philox4 w = philox4x32_10(gi[i].cgroup, gi[i].tensor_id, a.step_lo, a.step_hi8, a.keys);
+                    const uint32_t thr_lo = static_cast<uint32_t>(gi[i].thr);
+                    m = (w.x < thr_lo ? 1u : 0u) | (w.y < thr_lo ? 2u : 0u) | (w.z < thr_lo ? 4u : 0u) | (w.w < thr_lo ? 8u : 0u);
+                }
                 sel[i] = m & ((1u << gi[i].valid) - 1u);   // coordinates beyond the tensor's end do not exist
             }
         }
@@ -312,7 +424,9 @@ cudaError_t launch_shuffle_async_tiles(const ShuffleArgs &args, const LaunchShap
 {
     constexpr bool kHasB = TB::kCode != kDtypeNone;
     // G images of both stacks, 4 bytes of the warp's list, a byte per model for the permutation
-    const size_t image = static_cast<size_t>(args.pop.N) * (TA::kBytes * 4 + (kHasB ? TB::kBytes * 4 : 0));
+    // a group's values in both images ([P][N] with an even N: one vector of padding per group and stack)
+    const size_t group_elems = 4 * static_cast<size_t>(args.pop.N) + ((args.pop.layout == kLayoutPN && !(args.pop.N & 1)) ? 4 : 0);
+    const size_t image = group_elems * (TA::kBytes + (kHasB ? TB::kBytes : 0));
     const size_t per_thread = image * G + args.pop.N + 4;
     // block size: as many threads as keep a block's image near 44 KiB, so that five blocks
     // (about 200 KiB in flight) share an SM

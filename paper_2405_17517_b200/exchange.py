@@ -114,12 +114,14 @@ class ExchangeWorker:
             raise ValueError("staging capacity must be positive")
         for stack, r in self.rows.items():
             ops.bind(self.ctx, self.rank, stack, r)
+        self.handles = {}    # (stack, parity) -> the N workers' buffer handles, as exchanged
         for stack in self.rows:
             for parity in (0, 1):
                 mine = ops.staging_create(self.ctx, stack, parity, self.capacity)
                 handles = [None] * self.N
                 dist.all_gather_object(handles, mine, group=group)
                 ops.staging_open(self.ctx, stack, parity, handles)
+                self.handles[(stack, parity)] = handles
         self._token = ops.barrier_token(group)
         dist.barrier(group=group)   # every rank has mapped every buffer
 

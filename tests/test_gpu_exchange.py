@@ -238,9 +238,15 @@ def _process_worker(rank, world, port, out_dir):
         opt = to_device(mom.reshape(world, P)[rank])
         stats = torch.zeros(2, dtype=torch.int64, device="cuda")
         worker = ExchangeWorker(numel, row, opt, capacity=P // 2)
+        # a set of peers' buffers is mapped once: a second open is refused and changes nothing
+        refused = False
+        try:
+            B.wash_exchange_staging_open(worker.ctx, 0, 0, worker.handles[(0, 0)])
+        except B.WashError as err:
+            refused = err.code == B.WASH_ERR_STATE
         pop = oracle.Population(world, numel, off, P, 0)
         pl = [0.05, 1.0, 0.2]
-        ok = True
+        ok = refused
         for step in range(3):
             worker.step(step, 0.0, pl, seed=17, stats=stats)
             torch.cuda.synchronize()
@@ -266,3 +272,28 @@ def test_workers_in_two_processes_exchange_through_mapped_buffers(tmp_path):
         port = s.getsockname()[1]
     mp.spawn(_process_worker, args=(2, port, str(tmp_path)), nprocs=2, join=True)
     assert (tmp_path / "result.txt").read_text() == "ok"
+
+
+def test_bench_arm_with_two_ranks_on_one_device():
+    """bench.py --exchange-ranks under torchrun with two ranks that share the one GPU (gloo,
+    barrier on the host): the step runs through ExchangeWorker and the plan's slot counts
+    equal the oracle's."""
+    import json
+    import os
+    import socket
+    import subprocess
+    import sys
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        port = s.getsockname()[1]
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", "--nproc-per-node", "2", "--master-addr", "127.0.0.1",
+           "--master-port", str(port), os.path.join(root, "bench.py"), "--gpus", "2", "--exchange-ranks", "--workload",
+           "cfg2_resnet18_n5", "--steps", "4", "--warmup", "3"]
+    res = subprocess.run(cmd, capture_output=True, text=True, cwd=root, timeout=600)
+    assert res.returncode == 0, res.stderr[-2000:]
+    line = [json.loads(ln) for ln in res.stdout.splitlines() if ln.startswith("{")][-1]
+    assert line["arm"] == "exchange-ranks" and line["ranks"] == 2
+    assert line["counts_match_oracle"] is True
+    expect = line["expected_values_per_rank_per_step"]
+    assert abs(line["values_received_per_rank_per_step"] - expect) < 6 * expect ** 0.5
