@@ -262,9 +262,14 @@ def measure_philox_rate(B, torch, stream) -> float:
     return 5 * n_blocks / (e0.elapsed_time(e1) * 1e-3)
 
 
-def time_launches(torch, stream, launch, first_step: int, min_s: float = 0.06, blocks: int = 3, max_n: int = 2000):
+B2B_MIN_S = 0.06           # GPU time of a back-to-back series (set to 0 together with --min-timed-s 0)
+
+
+def time_launches(torch, stream, launch, first_step: int, min_s: float = None, blocks: int = 3, max_n: int = 2000):
     """Median and minimum per-launch time (ms) of `launch(step)` issued back to back, two events
     around each block of launches; the block length is chosen so that a block lasts min_s / blocks."""
+    if min_s is None:
+        min_s = B2B_MIN_S
     for k in range(3):
         launch(first_step + k)
     torch.cuda.synchronize()
@@ -493,7 +498,7 @@ def run_ours(args, rank: int, world: int, local_rank: int) -> None:
         block_ms.append(total)
         kernel_ms.append(per_kernel)
         if len(block_ms) == 1:       # the same count on every rank: derived from the all-reduced first block
-            repeats_wanted = int(min(MAX_REPEATS, max(1, np.ceil(MIN_TIMED_S * 1e3 / max(total, 1e-3)))))
+            repeats_wanted = int(min(MAX_REPEATS, max(1, np.ceil(args.min_timed_s * 1e3 / max(total, 1e-3)))))
     clocks = sampler.stop()
     launches = B.wash_launch_count() - launches0
     B.wash_check(pop.ctx)
@@ -888,6 +893,8 @@ def main() -> None:
     ap.add_argument("--threads", type=int, default=0)
     ap.add_argument("--blocks-per-sm", type=int, default=0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--min-timed-s", type=float, default=MIN_TIMED_S,
+                    help="repeat the timed block of --steps steps until this much GPU time has been measured (0: one block; for profiler runs)")
     ap.add_argument("--no-configs", action="store_true", help="skip the record of the other configurations (configs 1-4, cells of config 5)")
     ap.add_argument("--sweep", action="store_true", help="config-5 sweep of the shuffle kernel (many JSON lines)")
     ap.add_argument("--sweep-modes", default="stream,sparse")
@@ -903,6 +910,9 @@ def main() -> None:
     args.workload_given = any(a == "--workload" or a.startswith("--workload=") for a in sys.argv[1:])
     if args.warmup < 3 and args.impl == "ours":
         args.warmup = 3
+    if args.min_timed_s <= 0:
+        global B2B_MIN_S
+        B2B_MIN_S = 0.0
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))

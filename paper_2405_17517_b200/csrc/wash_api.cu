@@ -40,7 +40,7 @@ int cuda_fail(cudaError_t err, const char *what)
 }
 
 constexpr int kSlots = 4;   // pinned staging slots for table uploads
-constexpr int kPipeChunks = 8;   // wash_step_host cuts a large population into this many coordinate ranges
+constexpr int kPipeChunks = 32;   // wash_step_host cuts a large population into at most this many coordinate ranges
 
 // makes `device` current for the lifetime of the guard
 struct DeviceGuard {
@@ -266,6 +266,13 @@ int shuffle_impl(wash_ctx *ctx, int which, uint64_t step, double p, const double
             // and stack in [N][P], one or two for all N models in [P][N]
             const double share = ctx->layout == WASH_LAYOUT_PN ? 0.10 : 0.03;
             mode = ctx->expected_selected < share * coordinates ? WASH_MODE_SPARSE : WASH_MODE_STREAM;
+        }
+        // [P][N], even N: the streaming kernel pads its shared-memory image against bank conflicts
+        // once a fifth of the coordinates is expected to be served from it
+        if (ctx->layout == WASH_LAYOUT_PN && !(ctx->N & 1)) {
+            double coordinates = 0.0;
+            for (int s = 0; s < ctx->n_seg; ++s) coordinates += static_cast<double>(ctx->seg_host[s].numel);
+            args.pn_pad = ctx->expected_selected >= 0.2 * coordinates ? 4u : 0u;
         }
         if (sq) {   // the statistic is gathered by the streaming kernel only
             mode = WASH_MODE_STREAM;
@@ -607,7 +614,12 @@ int wash_step_host(wash_ctx *ctx, int32_t ops, void *host_params, void *host_opt
             if ((err = cudaEventRecord(ev_start, stream)) != cudaSuccess ||
                 (err = cudaStreamWaitEvent(ctx->copy_in, ev_start, 0)) != cudaSuccess ||
                 (err = cudaStreamWaitEvent(ctx->copy_out, ev_start, 0)) != cudaSuccess) return cuda_fail(err, "pipeline set-up");
-            const uint32_t per = ((ctx->n_groups + kPipeChunks - 1) / kPipeChunks + 255u) & ~255u;   // groups per range
+            // ranges of about 32 MiB of stack (8 at least, kPipeChunks at most): the first range's copy in and
+            // the last range's copy out are the part of the transfers that nothing overlaps
+            const size_t stack_bytes = p_bytes + o_bytes;
+            int chunks = static_cast<int>(stack_bytes >> 25);
+            chunks = chunks < 8 ? 8 : (chunks > kPipeChunks ? kPipeChunks : chunks);
+            const uint32_t per = ((ctx->n_groups + chunks - 1) / chunks + 255u) & ~255u;   // groups per range
             // moves the elements [e0, e0 + count) of every model between a host and the device stack
             auto copy_range = [&](void *dst, const void *src, int dtype, size_t e0, size_t count, cudaMemcpyKind kind, cudaStream_t s) {
                 const size_t eb = elem_bytes(dtype);

@@ -82,6 +82,7 @@ struct ShuffleArgs {
     StatSlot *stat_slots;         // device, kStatSlots zeroed entries (left zeroed by every launch), or nullptr
     uint32_t *status;             // device status word
     SqArgs sq;                    // consensus distance of the first stack (streaming kernel only)
+    uint32_t pn_pad = 0;          // streaming kernel, [P][N]: elements of padding after a group in the shared-memory image (0 or 4)
 };
 
 struct ReduceArgs {

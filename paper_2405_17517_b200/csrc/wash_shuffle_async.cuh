@@ -15,10 +15,11 @@
 //           are copied by their own thread, bf16 rows cooperatively in 16-byte pieces
 //   [P][N]: the block's T*4N elements are contiguous in global memory and are copied
 //           vector by vector, vector k*T + t by thread t; a group's 4N elements stay together
-//           and, when N is even, are followed by one vector of padding, so that a group spans
-//           an odd number of vectors and the lanes of a warp (one group each) fall into
-//           different shared-memory banks: thread t's coordinate c of model n is element
-//           t*pn_group_elems(N) + c*N + n of that image.
+//           and, when N is even and the launch expects to serve many coordinates, are followed
+//           by one vector of padding, so that a group spans an odd number of vectors and the
+//           lanes of a warp (one group each) fall into different shared-memory banks (at small
+//           p the image is hardly read and the padding would only cost bytes in flight):
+//           thread t's coordinate c of model n is element t*pn_group_elems + c*N + n.
 #pragma once
 #include "wash_device.cuh"
 #include "wash_launch.cuh"
@@ -41,16 +42,16 @@ __device__ __forceinline__ void cp_async_wait_all()
     asm volatile("cp.async.wait_all;" ::: "memory");
 }
 
-// elements a group takes in the [P][N] image: its 4N values, plus one vector of padding when N is even
-__device__ __forceinline__ uint32_t pn_group_elems(int n_models)
+// elements a group takes in the [P][N] image: its 4N values plus the launch's padding (0 or one vector)
+__device__ __forceinline__ uint32_t pn_group_elems(int n_models, uint32_t pad)
 {
-    return 4u * static_cast<uint32_t>(n_models) + ((n_models & 1) ? 0u : 4u);
+    return 4u * static_cast<uint32_t>(n_models) + pad;
 }
 
 // Starts the copies of one stack for this thread's block position; returns nothing.
 template <class T, int LAYOUT>
 __device__ __forceinline__ void async_fetch(uint32_t image, void *base, const PopView &pop, uint64_t g_block,
-                                            uint32_t groups_in_block, int n_models)
+                                            uint32_t groups_in_block, int n_models, uint32_t pn_pad)
 {
     constexpr int kVec = T::kBytes * 4;
     const uint32_t t = threadIdx.x, T_ = blockDim.x;
@@ -76,9 +77,14 @@ __device__ __forceinline__ void async_fetch(uint32_t image, void *base, const Po
             for (int j = 0; j < n_models; ++j, src += row_bytes, dst += T_ * kVec) cp_async<kVec>(dst, src);
         }
     } else {
-        // vector k is vector j = k % N of group k / N; the pair is advanced without dividing again
         const uint32_t vecs = groups_in_block * n_models, N_ = static_cast<uint32_t>(n_models);
-        const uint32_t stride = pn_group_elems(n_models) / 4u, dq = T_ / N_, dr = T_ - dq * N_;
+        if (pn_pad == 0) {   // the image is the block's bytes as they lie
+            const char *src = static_cast<const char *>(base) + 4ll * static_cast<long long>(g_block) * n_models * T::kBytes;
+            for (uint32_t k = t; k < vecs; k += T_) cp_async<kVec>(image + k * kVec, src + static_cast<size_t>(k) * kVec);
+            return;
+        }
+        // vector k is vector j = k % N of group k / N; the pair is advanced without dividing again
+        const uint32_t stride = pn_group_elems(n_models, pn_pad) / 4u, dq = T_ / N_, dr = T_ - dq * N_;
         const char *src = static_cast<const char *>(base) + 4ll * static_cast<long long>(g_block) * n_models * T::kBytes;
         uint32_t group = t / N_, j = t - group * N_;
         for (uint32_t k = t; k < vecs; k += T_) {
@@ -92,11 +98,11 @@ __device__ __forceinline__ void async_fetch(uint32_t image, void *base, const Po
 
 // raw bits of (model n, coordinate c) of the group of block thread t, out of the block image
 template <class T, int LAYOUT>
-__device__ __forceinline__ uint32_t image_value(const unsigned char *image, int n_models, uint32_t t, int n, int c)
+__device__ __forceinline__ uint32_t image_value(const unsigned char *image, int n_models, uint32_t pn_pad, uint32_t t, int n, int c)
 {
     const uint32_t T_ = blockDim.x;
     const uint32_t elem = LAYOUT == kLayoutNP ? (static_cast<uint32_t>(n) * T_ + t) * 4u + c
-                                              : t * pn_group_elems(n_models) + static_cast<uint32_t>(c * n_models + n);
+                                              : t * pn_group_elems(n_models, pn_pad) + static_cast<uint32_t>(c * n_models + n);
     if (T::kBytes == 4) return reinterpret_cast<const uint32_t *>(image)[elem];
     return reinterpret_cast<const uint16_t *>(image)[elem];
 }
@@ -157,7 +163,7 @@ __device__ __forceinline__ void serve_group_dense(const ShuffleArgs &a, const un
         // the group's 4N elements are contiguous: element c*N + n is (coordinate c, model n)
         char *out_a = group_vec_ptr<TA, LAYOUT>(a.a, a.pop, g_block + t, 0);
         char *out_b = kHasB ? group_vec_ptr<TB, LAYOUT>(a.b, a.pop, g_block + t, 0) : nullptr;
-        const uint32_t img0 = t * pn_group_elems(n_models);
+        const uint32_t img0 = t * pn_group_elems(n_models, a.pn_pad);
         PERM rest = perm[0];
         uint32_t base = img0;   // image element of (coordinate c, model 0)
         int n = 0, c = 0;
@@ -239,7 +245,7 @@ __device__ __forceinline__ void serve_tile(const ShuffleArgs &a, const unsigned 
         const long long out_step = LAYOUT == kLayoutNP ? a.pop.padded_P : 1;
         const long long out0 = LAYOUT == kLayoutNP ? e : e * n_models;
         const uint32_t img_step = LAYOUT == kLayoutNP ? T_ * 4u : 1u;
-        const uint32_t img0 = LAYOUT == kLayoutNP ? t_owner * 4u + c : t_owner * pn_group_elems(n_models) + c * n_models;
+        const uint32_t img0 = LAYOUT == kLayoutNP ? t_owner * 4u + c : t_owner * pn_group_elems(n_models, a.pn_pad) + c * n_models;
         long long out = out0;
         uint64_t rest = perm;   // nibble n on top of the low end when model n's turn comes
         for (int n = 0; n < n_models; ++n, out += out_step, rest >>= 4) {
@@ -260,7 +266,7 @@ __device__ __forceinline__ void serve_tile(const ShuffleArgs &a, const unsigned 
 
 // the four values of model n in the group of block thread t, widened to binary32
 template <class T, int LAYOUT>
-__device__ __forceinline__ void image_group(const unsigned char *image, int n_models, uint32_t t, int n, float (&x)[4])
+__device__ __forceinline__ void image_group(const unsigned char *image, int n_models, uint32_t pn_pad, uint32_t t, int n, float (&x)[4])
 {
     if (LAYOUT == kLayoutNP) {
         const typename T::vec v = reinterpret_cast<const typename T::vec *>(image)[static_cast<uint32_t>(n) * blockDim.x + t];
@@ -268,7 +274,7 @@ __device__ __forceinline__ void image_group(const unsigned char *image, int n_mo
         for (int c = 0; c < 4; ++c) x[c] = T::to_float(T::get(v, c));
     } else {
 #pragma unroll
-        for (int c = 0; c < 4; ++c) x[c] = T::to_float(image_value<T, LAYOUT>(image, n_models, t, n, c));
+        for (int c = 0; c < 4; ++c) x[c] = T::to_float(image_value<T, LAYOUT>(image, n_models, pn_pad, t, n, c));
     }
 }
 
@@ -290,7 +296,7 @@ __device__ __forceinline__ void consensus_warp(const ShuffleArgs &a, const unsig
     if (WHOLE || r1) {
         float x[4];
         for (int n = 0; n < n_models; ++n) {
-            image_group<T, LAYOUT>(image, n_models, threadIdx.x, n, x);
+            image_group<T, LAYOUT>(image, n_models, a.pn_pad, threadIdx.x, n, x);
 #pragma unroll
             for (int c = 0; c < 4; ++c) mean[c] += static_cast<double>(x[c]);
         }
@@ -309,7 +315,7 @@ __device__ __forceinline__ void consensus_warp(const ShuffleArgs &a, const unsig
             double s = 0.0;
             if (WHOLE || r1 == r) {
                 float x[4];
-                image_group<T, LAYOUT>(image, n_models, threadIdx.x, n, x);
+                image_group<T, LAYOUT>(image, n_models, a.pn_pad, threadIdx.x, n, x);
 #pragma unroll
                 for (int c = 0; c < 4; ++c)
                     if (WHOLE || c < valid) {   // padding beyond the tensor's end holds no coordinate
@@ -356,7 +362,7 @@ __global__ void __launch_bounds__(256, 5) shuffle_async_kernel(const __grid_cons
     const int n_models = a.pop.N;
     const uint32_t T_ = blockDim.x;
     // G pairs of images of the two stacks, then the warps' lists, then the permutation columns
-    const size_t group_elems = LAYOUT == kLayoutPN ? pn_group_elems(n_models) : 4u * static_cast<size_t>(n_models);
+    const size_t group_elems = LAYOUT == kLayoutPN ? pn_group_elems(n_models, a.pn_pad) : 4u * static_cast<size_t>(n_models);
     const size_t a_bytes = group_elems * T_ * TA::kBytes;
     const size_t b_bytes = kHasB ? group_elems * T_ * TB::kBytes : 0;
     uint8_t *s_list = smem_raw + G * (a_bytes + b_bytes);   // 128 bytes per warp
@@ -370,8 +376,8 @@ __global__ void __launch_bounds__(256, 5) shuffle_async_kernel(const __grid_cons
         in_tile[i] = g_block < a.group_hi ? static_cast<uint32_t>(min(static_cast<uint64_t>(T_), a.group_hi - g_block)) : 0u;
         if (in_tile[i] == 0) continue;
         unsigned char *image_a = smem_raw + i * (a_bytes + b_bytes);
-        async_fetch<TA, LAYOUT>(smem_addr(image_a), a.a, a.pop, g_block, in_tile[i], n_models);
-        if constexpr (kHasB) async_fetch<TB, LAYOUT>(smem_addr(image_a + a_bytes), a.b, a.pop, g_block, in_tile[i], n_models);
+        async_fetch<TA, LAYOUT>(smem_addr(image_a), a.a, a.pop, g_block, in_tile[i], n_models, a.pn_pad);
+        if constexpr (kHasB) async_fetch<TB, LAYOUT>(smem_addr(image_a + a_bytes), a.b, a.pop, g_block, in_tile[i], n_models, a.pn_pad);
     }
 
     uint32_t selected = 0, moved = 0;
@@ -424,8 +430,8 @@ cudaError_t launch_shuffle_async_tiles(const ShuffleArgs &args, const LaunchShap
 {
     constexpr bool kHasB = TB::kCode != kDtypeNone;
     // G images of both stacks, 4 bytes of the warp's list, a byte per model for the permutation
-    // a group's values in both images ([P][N] with an even N: one vector of padding per group and stack)
-    const size_t group_elems = 4 * static_cast<size_t>(args.pop.N) + ((args.pop.layout == kLayoutPN && !(args.pop.N & 1)) ? 4 : 0);
+    // a group's values in both images (with the launch's padding per group and stack in [P][N])
+    const size_t group_elems = 4 * static_cast<size_t>(args.pop.N) + (args.pop.layout == kLayoutPN ? args.pn_pad : 0);
     const size_t image = group_elems * (TA::kBytes + (kHasB ? TB::kBytes : 0));
     const size_t per_thread = image * G + args.pop.N + 4;
     // block size: as many threads as keep a block's image near 44 KiB, so that five blocks
