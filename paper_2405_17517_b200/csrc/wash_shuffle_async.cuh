@@ -12,7 +12,7 @@
 // One group per thread, one trip per thread (the block scheduler refills the SM as
 // blocks retire).  Block image in shared memory:
 //   [N][P]: vector j of thread t at (j*T + t) * vec      (T = threads per block); fp32 vectors
-//           are copied by their own thread, bf16 rows cooperatively in 16-byte pieces
+//           are copied by their own thread, bf16 vectors in 16-byte pairs by the two lanes that own them
 //   [P][N]: the block's T*4N elements are contiguous in global memory and are copied
 //           vector by vector, vector k*T + t by thread t; a group's 4N elements stay together
 //           and, when N is even and the launch expects to serve many coordinates, are followed
@@ -56,15 +56,16 @@ __device__ __forceinline__ void async_fetch(uint32_t image, void *base, const Po
     constexpr int kVec = T::kBytes * 4;
     const uint32_t t = threadIdx.x, T_ = blockDim.x;
     if (LAYOUT == kLayoutNP && kVec == 8) {
-        // bf16: a row of the image (T groups of 8 bytes) is contiguous in global memory too;
-        // copy it in 16-byte pieces, thread t taking pieces t, t + T, ... of the N rows (the
-        // number of groups in a block is even, so a row is a whole number of pieces)
-        const uint32_t per_row = groups_in_block / 2, pieces = per_row * n_models;
-        const char *row0 = group_vec_ptr<T, LAYOUT>(base, pop, g_block, 0);
-        const size_t row_bytes = static_cast<size_t>(pop.padded_P) * T::kBytes;
-        for (uint32_t k = t; k < pieces; k += T_) {
-            const uint32_t j = k / per_row, piece = k - j * per_row;
-            cp_async<16>(image + j * T_ * kVec + piece * 16, row0 + j * row_bytes + piece * 16);
+        // bf16: two neighbouring groups of a row are 16 contiguous bytes in global memory and in the
+        // image.  The two lanes that own them share the work: lane 2k takes the even rows of the
+        // pair's piece, lane 2k+1 the odd rows, each copy 16 bytes (the number of groups in a block
+        // is even).  A warp's groups are thus copied by that warp's lanes alone.
+        const uint32_t piece = t >> 1;
+        if (2u * piece < groups_in_block) {
+            const size_t row_bytes = static_cast<size_t>(pop.padded_P) * T::kBytes;
+            const char *src = group_vec_ptr<T, LAYOUT>(base, pop, g_block, 0) + (t & 1u) * row_bytes + piece * 16;
+            uint32_t dst = image + (t & 1u) * T_ * kVec + piece * 16;
+            for (uint32_t j = t & 1u; j < static_cast<uint32_t>(n_models); j += 2, src += 2 * row_bytes, dst += 2 * T_ * kVec) cp_async<16>(dst, src);
         }
     } else if (LAYOUT == kLayoutNP) {
         if (t < groups_in_block) {
@@ -405,10 +406,9 @@ __global__ void __launch_bounds__(256, 5) shuffle_async_kernel(const __grid_cons
     // Every thread waits for its own copies (none may be in flight when the block ends).
     // A selected coordinate is served by whichever lane of the warp gets it, so the warp
     // must see each other's copies; in the [P][N] image a group's values were copied by
-    // threads of other warps, so a block with a selected coordinate needs a block-wide
-    // barrier instead.
+    // threads of other warps, so there a block-wide barrier is needed instead.
     cp_async_wait_all();
-    constexpr bool kSharedCopies = LAYOUT == kLayoutPN || TA::kBytes == 2 || (kHasB && TB::kBytes == 2);   // a group's bytes were copied by other threads
+    constexpr bool kSharedCopies = LAYOUT == kLayoutPN;   // a group's bytes were copied by threads of other warps
     if (kSharedCopies) __syncthreads();
     else __syncwarp();
     if constexpr (STAT) {
