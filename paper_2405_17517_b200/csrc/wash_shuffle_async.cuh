@@ -189,6 +189,85 @@ __device__ __forceinline__ void serve_group_dense(const ShuffleArgs &a, const un
     }
 }
 
+// The same for N > 16, where a permutation does not fit a register: the four coordinates'
+// permutations are four columns of bytes in shared memory (column c of the thread at
+// s_perm + c*N*T, entry n at [n*T]) and their Fisher-Yates chains run side by side, so that the
+// four Philox draws of a step overlap and a swap's shared-memory round trip hides behind the
+// other three chains.
+template <class TA, class TB, int LAYOUT>
+__device__ __forceinline__ void serve_group_dense_bytes(const ShuffleArgs &a, const unsigned char *image_a, const unsigned char *image_b,
+                                                        uint8_t *s_perm, uint64_t g_block, uint32_t sel, const GroupInfo &gi,
+                                                        uint32_t &selected, uint32_t &moved)
+{
+    constexpr bool kHasB = TB::kCode != kDtypeNone;
+    const int n_models = a.pop.N;
+    const uint32_t T_ = blockDim.x, t = threadIdx.x;
+    const uint32_t col = static_cast<uint32_t>(n_models) * T_;   // bytes from one coordinate's column to the next
+    for (int n = 0; n < n_models; ++n) {
+#pragma unroll
+        for (int c = 0; c < 4; ++c) s_perm[c * col + n * T_] = static_cast<uint8_t>(n);
+    }
+    Philox4 w[4];
+    for (int k = n_models - 1, m = 0; k >= 1; --k, ++m) {
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+            if (!((sel >> c) & 1u)) continue;
+            if ((m & 3) == 0) w[c] = philox4x32_10(4u * gi.cgroup + c, gi.tensor_id, a.step_lo, a.step_hi8 | (1u + (static_cast<uint32_t>(m) >> 2)), a.keys);
+            const uint32_t r = w[c].x;
+            w[c].x = w[c].y; w[c].y = w[c].z; w[c].z = w[c].w;
+            const uint32_t j = __umulhi(r, static_cast<uint32_t>(k + 1));
+            uint8_t *column = s_perm + c * col;
+            const uint8_t pk = column[k * T_], pj = column[j * T_];
+            column[k * T_] = pj;
+            column[j * T_] = pk;
+        }
+    }
+    selected += __popc(sel);
+    auto value_a = [&](uint32_t from) -> uint32_t {
+        return TA::kBytes == 4 ? reinterpret_cast<const uint32_t *>(image_a)[from] : reinterpret_cast<const uint16_t *>(image_a)[from];
+    };
+    auto value_b = [&](uint32_t from) -> uint32_t {
+        return TB::kBytes == 4 ? reinterpret_cast<const uint32_t *>(image_b)[from] : reinterpret_cast<const uint16_t *>(image_b)[from];
+    };
+    char *out_a = group_vec_ptr<TA, LAYOUT>(a.a, a.pop, g_block + t, 0);
+    char *out_b = kHasB ? group_vec_ptr<TB, LAYOUT>(a.b, a.pop, g_block + t, 0) : nullptr;
+    if (LAYOUT == kLayoutNP) {
+        const size_t row_a = static_cast<size_t>(a.pop.padded_P) * TA::kBytes, row_b = static_cast<size_t>(a.pop.padded_P) * TB::kBytes;
+        const uint32_t img_step = T_ * 4u, img0 = t * 4u;
+        for (int n = 0; n < n_models; ++n, out_a += row_a, out_b += row_b) {
+            uint32_t wa[4], wb[4];
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+                const uint32_t src = s_perm[c * col + n * T_];
+                moved += src != static_cast<uint32_t>(n) ? 1u : 0u;
+                const uint32_t from = src * img_step + img0 + c;
+                wa[c] = value_a(from);
+                if constexpr (kHasB) wb[c] = value_b(from);
+            }
+            TA::store_group(out_a, TA::pack(wa[0], wa[1], wa[2], wa[3]));
+            if constexpr (kHasB) TB::store_group(out_b, TB::pack(wb[0], wb[1], wb[2], wb[3]));
+        }
+    } else {
+        // the group's 4N elements are contiguous: element c*N + n is (coordinate c, model n)
+        const uint32_t img0 = t * pn_group_elems(n_models, a.pn_pad);
+        int n = 0, c = 0;
+        for (int j = 0; j < n_models; ++j) {
+            uint32_t wa[4], wb[4];
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                const uint32_t src = s_perm[c * col + n * T_];
+                moved += src != static_cast<uint32_t>(n) ? 1u : 0u;
+                const uint32_t from = img0 + static_cast<uint32_t>(c * n_models) + src;
+                wa[q] = value_a(from);
+                if constexpr (kHasB) wb[q] = value_b(from);
+                if (++n == n_models) { n = 0; ++c; }
+            }
+            TA::store_group(out_a + static_cast<size_t>(j) * (TA::kBytes * 4), TA::pack(wa[0], wa[1], wa[2], wa[3]));
+            if constexpr (kHasB) TB::store_group(out_b + static_cast<size_t>(j) * (TB::kBytes * 4), TB::pack(wb[0], wb[1], wb[2], wb[3]));
+        }
+    }
+}
+
 // Serves the selected coordinates of one tile of T groups (one group per thread): the warp's
 // selected coordinates are listed in shared memory and dealt out to the lanes 32 at a time:
 // with a few selected coordinates per warp (p around 0.01-0.1) one round serves them all,
@@ -207,12 +286,13 @@ __device__ __forceinline__ void serve_tile(const ShuffleArgs &a, const unsigned 
     // Half of the warp's coordinates or more selected: dealing them out would take two rounds or
     // more, in each of which a lane draws one permutation and stores 4-byte values; every lane
     // serving its own group costs less from there on (measured crossover near 64 of 128).
-    if (n_models <= 16 && __reduce_add_sync(0xFFFFFFFFu, mine) >= kDenseMinSelected &&
-        __all_sync(0xFFFFFFFFu, sel == 0 || gi.valid == 4)) {
+    // (In the moved-values count of the byte version an unselected coordinate adds nothing: its
+    // column stays the identity.)
+    if (__reduce_add_sync(0xFFFFFFFFu, mine) >= kDenseMinSelected && __all_sync(0xFFFFFFFFu, sel == 0 || gi.valid == 4)) {
         if (sel) {
-            const uint64_t g_tile = g_block;
-            if (n_models <= 8) serve_group_dense<TA, TB, LAYOUT, uint32_t>(a, image_a, image_b, g_tile, sel, gi, selected, moved);
-            else serve_group_dense<TA, TB, LAYOUT, uint64_t>(a, image_a, image_b, g_tile, sel, gi, selected, moved);
+            if (n_models <= 8) serve_group_dense<TA, TB, LAYOUT, uint32_t>(a, image_a, image_b, g_block, sel, gi, selected, moved);
+            else if (n_models <= 16) serve_group_dense<TA, TB, LAYOUT, uint64_t>(a, image_a, image_b, g_block, sel, gi, selected, moved);
+            else serve_group_dense_bytes<TA, TB, LAYOUT>(a, image_a, image_b, s_perm, g_block, sel, gi, selected, moved);
         }
         return;
     }
@@ -367,7 +447,7 @@ __global__ void __launch_bounds__(256, 5) shuffle_async_kernel(const __grid_cons
     const size_t a_bytes = group_elems * T_ * TA::kBytes;
     const size_t b_bytes = kHasB ? group_elems * T_ * TB::kBytes : 0;
     uint8_t *s_list = smem_raw + G * (a_bytes + b_bytes);   // 128 bytes per warp
-    uint8_t *s_perm = s_list + 4 * T_ + threadIdx.x;        // column [n][T], used when N > 16
+    uint8_t *s_perm = s_list + 4 * T_ + threadIdx.x;        // four columns [c][n][T] of bytes, used when N > 16
 
     const uint64_t g_first = a.group_lo + static_cast<uint64_t>(blockIdx.x) * (T_ * G);
     uint32_t in_tile[G];   // groups of tile i that exist
@@ -429,11 +509,10 @@ template <class TA, class TB, int G>
 cudaError_t launch_shuffle_async_tiles(const ShuffleArgs &args, const LaunchShape &shape, cudaStream_t stream)
 {
     constexpr bool kHasB = TB::kCode != kDtypeNone;
-    // G images of both stacks, 4 bytes of the warp's list, a byte per model for the permutation
     // a group's values in both images (with the launch's padding per group and stack in [P][N])
     const size_t group_elems = 4 * static_cast<size_t>(args.pop.N) + (args.pop.layout == kLayoutPN ? args.pn_pad : 0);
     const size_t image = group_elems * (TA::kBytes + (kHasB ? TB::kBytes : 0));
-    const size_t per_thread = image * G + args.pop.N + 4;
+    const size_t per_thread = image * G + (args.pop.N > 16 ? 4 * args.pop.N : 0) + 4;   // images, the permutation columns (N > 16), the warp's list
     // block size: as many threads as keep a block's image near 44 KiB, so that five blocks
     // (about 200 KiB in flight) share an SM
     int threads = shape.threads > 0 ? shape.threads : 64;   // measured: 64 beats 128 and 256 (a block holds its shared memory until its slowest thread is done)
