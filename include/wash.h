@@ -125,7 +125,10 @@ int wash_set_mode(wash_ctx *ctx, int32_t mode);
  * > 0 a persistent grid of SM count x min(blocks_per_sm, resident blocks per SM) blocks
  * that stride over the groups, < 0 one group of 4 coordinates per thread.  For
  * WASH_MODE_STREAM blocks_per_sm = 1 or 2 fixes the number of groups a thread takes
- * (default: 2 when a group of all models is at most 64 bytes, else 1). */
+ * (default: 2 when a group of all models is at most 64 bytes, else 1); blocks_per_sm = -2 / -3
+ * forces the streaming kernel's lean / early flavour (early draws the permutations while the
+ * stack's copies are in flight and serves populations of more than 16 models densely; by
+ * default it is launched for N > 16 when the call's probabilities select 30 % or more). */
 int wash_set_launch(wash_ctx *ctx, int32_t threads, int32_t blocks_per_sm);
 
 /* ---- the shuffling step ----------------------------------------------------------- */

@@ -40,6 +40,7 @@ int cuda_fail(cudaError_t err, const char *what)
 }
 
 constexpr int kSlots = 4;   // pinned staging slots for table uploads
+constexpr double kEarlyShare = 0.3;   // expected share of selected coordinates from which the streaming kernel's early flavour is launched (N > 16)
 constexpr int kPipeChunks = 32;   // wash_step_host cuts a large population into at most this many coordinate ranges
 
 // makes `device` current for the lifetime of the guard
@@ -267,13 +268,18 @@ int shuffle_impl(wash_ctx *ctx, int which, uint64_t step, double p, const double
             const double share = ctx->layout == WASH_LAYOUT_PN ? 0.10 : 0.03;
             mode = ctx->expected_selected < share * coordinates ? WASH_MODE_SPARSE : WASH_MODE_STREAM;
         }
+        double coordinates = 0.0;
+        for (int s = 0; s < ctx->n_seg; ++s) coordinates += static_cast<double>(ctx->seg_host[s].numel);
         // [P][N], even N: the streaming kernel pads its shared-memory image against bank conflicts
         // once a fifth of the coordinates is expected to be served from it
-        if (ctx->layout == WASH_LAYOUT_PN && !(ctx->N & 1)) {
-            double coordinates = 0.0;
-            for (int s = 0; s < ctx->n_seg; ++s) coordinates += static_cast<double>(ctx->seg_host[s].numel);
-            args.pn_pad = ctx->expected_selected >= 0.2 * coordinates ? 4u : 0u;
-        }
+        if (ctx->layout == WASH_LAYOUT_PN && !(ctx->N & 1)) args.pn_pad = ctx->expected_selected >= 0.2 * coordinates ? 4u : 0u;
+        // The streaming kernel's early flavour (permutations drawn while the copies are in flight, dense
+        // serving for N > 16) costs registers and, for N > 16, three more permutation columns of shared
+        // memory per thread: measured, it pays only for large populations of which most coordinates are
+        // served (N = 32, p = 1: 15.7 -> 10.4 ms, [P][N] 29.8 -> 13.3 ms; slower by 0-15 % everywhere else).
+        args.early = ctx->N > 16 && ctx->expected_selected >= kEarlyShare * coordinates;
+        if (ctx->shape.blocks_per_sm == -2) args.early = false;   // tuning override (wash_set_launch)
+        if (ctx->shape.blocks_per_sm == -3) args.early = true;
         if (sq) {   // the statistic is gathered by the streaming kernel only
             mode = WASH_MODE_STREAM;
             args.stat_slots = ctx->stat_slots_dev;

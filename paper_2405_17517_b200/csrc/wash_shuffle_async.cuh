@@ -114,15 +114,14 @@ __device__ __forceinline__ uint32_t image_value(const unsigned char *image, int 
 // no list, no dealing, a quarter of the store instructions, and full 16-byte pieces of a sector.
 // An unselected coordinate of such a group is rewritten with the bits it already has.  PERM is
 // uint32_t (N <= 8) or uint64_t (N <= 16); the caller has checked that the group is whole.
-template <class TA, class TB, int LAYOUT, class PERM>
-__device__ __forceinline__ void serve_group_dense(const ShuffleArgs &a, const unsigned char *image_a, const unsigned char *image_b,
-                                                  uint64_t g_block, uint32_t sel, const GroupInfo &gi, uint32_t &selected, uint32_t &moved)
+// The draw needs no data, the write needs the image: two halves, so that a kernel can draw while
+// its copies are still in flight.
+template <class PERM>
+__device__ __forceinline__ void dense_draw(const ShuffleArgs &a, uint32_t sel, const GroupInfo &gi, PERM (&perm)[4],
+                                           uint32_t &selected, uint32_t &moved)
 {
-    constexpr bool kHasB = TB::kCode != kDtypeNone;
     constexpr PERM kIdentity = static_cast<PERM>(0xFEDCBA9876543210ull), kOnes = static_cast<PERM>(0x1111111111111111ull);
     const int n_models = a.pop.N;
-    const uint32_t T_ = blockDim.x, t = threadIdx.x;
-    PERM perm[4];
 #pragma unroll
     for (int c = 0; c < 4; ++c) {
         perm[c] = kIdentity;
@@ -136,6 +135,15 @@ __device__ __forceinline__ void serve_group_dense(const ShuffleArgs &a, const un
             ++selected;
         }
     }
+}
+
+template <class TA, class TB, int LAYOUT, class PERM>
+__device__ __forceinline__ void dense_write(const ShuffleArgs &a, const unsigned char *image_a, const unsigned char *image_b,
+                                            uint64_t g_block, PERM (&perm)[4])
+{
+    constexpr bool kHasB = TB::kCode != kDtypeNone;
+    const int n_models = a.pop.N;
+    const uint32_t T_ = blockDim.x, t = threadIdx.x;
     auto value_a = [&](uint32_t from) -> uint32_t {
         return TA::kBytes == 4 ? reinterpret_cast<const uint32_t *>(image_a)[from] : reinterpret_cast<const uint16_t *>(image_a)[from];
     };
@@ -194,14 +202,10 @@ __device__ __forceinline__ void serve_group_dense(const ShuffleArgs &a, const un
 // s_perm + c*N*T, entry n at [n*T]) and their Fisher-Yates chains run side by side, so that the
 // four Philox draws of a step overlap and a swap's shared-memory round trip hides behind the
 // other three chains.
-template <class TA, class TB, int LAYOUT>
-__device__ __forceinline__ void serve_group_dense_bytes(const ShuffleArgs &a, const unsigned char *image_a, const unsigned char *image_b,
-                                                        uint8_t *s_perm, uint64_t g_block, uint32_t sel, const GroupInfo &gi,
-                                                        uint32_t &selected, uint32_t &moved)
+__device__ __forceinline__ void dense_bytes_draw(const ShuffleArgs &a, uint8_t *s_perm, uint32_t sel, uint32_t cgroup, uint32_t tensor_id)
 {
-    constexpr bool kHasB = TB::kCode != kDtypeNone;
     const int n_models = a.pop.N;
-    const uint32_t T_ = blockDim.x, t = threadIdx.x;
+    const uint32_t T_ = blockDim.x;
     const uint32_t col = static_cast<uint32_t>(n_models) * T_;   // bytes from one coordinate's column to the next
     for (int n = 0; n < n_models; ++n) {
 #pragma unroll
@@ -212,7 +216,7 @@ __device__ __forceinline__ void serve_group_dense_bytes(const ShuffleArgs &a, co
 #pragma unroll
         for (int c = 0; c < 4; ++c) {
             if (!((sel >> c) & 1u)) continue;
-            if ((m & 3) == 0) w[c] = philox4x32_10(4u * gi.cgroup + c, gi.tensor_id, a.step_lo, a.step_hi8 | (1u + (static_cast<uint32_t>(m) >> 2)), a.keys);
+            if ((m & 3) == 0) w[c] = philox4x32_10(4u * cgroup + c, tensor_id, a.step_lo, a.step_hi8 | (1u + (static_cast<uint32_t>(m) >> 2)), a.keys);
             const uint32_t r = w[c].x;
             w[c].x = w[c].y; w[c].y = w[c].z; w[c].z = w[c].w;
             const uint32_t j = __umulhi(r, static_cast<uint32_t>(k + 1));
@@ -222,7 +226,19 @@ __device__ __forceinline__ void serve_group_dense_bytes(const ShuffleArgs &a, co
             column[j * T_] = pk;
         }
     }
-    selected += __popc(sel);
+}
+
+// (an unselected coordinate adds nothing to the moved-values count: its column is the identity)
+// Returns the number of values that moved.
+template <class TA, class TB, int LAYOUT>
+__device__ __forceinline__ uint32_t dense_bytes_write(const ShuffleArgs &a, const unsigned char *image_a, const unsigned char *image_b,
+                                                          const uint8_t *s_perm, uint64_t g_block)
+{
+    constexpr bool kHasB = TB::kCode != kDtypeNone;
+    uint32_t moved = 0;
+    const int n_models = a.pop.N;
+    const uint32_t T_ = blockDim.x, t = threadIdx.x;
+    const uint32_t col = static_cast<uint32_t>(n_models) * T_;
     auto value_a = [&](uint32_t from) -> uint32_t {
         return TA::kBytes == 4 ? reinterpret_cast<const uint32_t *>(image_a)[from] : reinterpret_cast<const uint16_t *>(image_a)[from];
     };
@@ -266,33 +282,169 @@ __device__ __forceinline__ void serve_group_dense_bytes(const ShuffleArgs &a, co
             if constexpr (kHasB) TB::store_group(out_b + static_cast<size_t>(j) * (TB::kBytes * 4), TB::pack(wb[0], wb[1], wb[2], wb[3]));
         }
     }
+    return moved;
 }
 
-// Serves the selected coordinates of one tile of T groups (one group per thread): the warp's
-// selected coordinates are listed in shared memory and dealt out to the lanes 32 at a time:
-// with a few selected coordinates per warp (p around 0.01-0.1) one round serves them all,
-// instead of one divergent pass per coordinate slot.  Called by all threads of the block.
+// The moves of one selected coordinate (coordinate c of the group of block thread t_owner): model n
+// takes the value of model pi(n), nibble n of `perm` (N <= 16) or byte n of the column s_perm.
+template <class TA, class TB, int LAYOUT>
+__device__ __forceinline__ void move_coordinate(const ShuffleArgs &a, const unsigned char *image_a, const unsigned char *image_b,
+                                                const uint8_t *s_perm, uint64_t perm, uint32_t t_owner, uint32_t c, uint64_t g_block,
+                                                uint32_t &moved)
+{
+    constexpr bool kHasB = TB::kCode != kDtypeNone;
+    const int n_models = a.pop.N;
+    const uint32_t T_ = blockDim.x;
+    const long long e = 4ll * static_cast<long long>(g_block + t_owner) + c;
+    // model n's value of this coordinate sits at out0 + n*out_step in the stack and at
+    // element img0 + n*img_step of the image: no multiplication left inside the loop
+    const long long out_step = LAYOUT == kLayoutNP ? a.pop.padded_P : 1;
+    const long long out0 = LAYOUT == kLayoutNP ? e : e * n_models;
+    const uint32_t img_step = LAYOUT == kLayoutNP ? T_ * 4u : 1u;
+    const uint32_t img0 = LAYOUT == kLayoutNP ? t_owner * 4u + c : t_owner * pn_group_elems(n_models, a.pn_pad) + c * n_models;
+    long long out = out0;
+    uint64_t rest = perm;   // nibble n on top of the low end when model n's turn comes
+    for (int n = 0; n < n_models; ++n, out += out_step, rest >>= 4) {
+        const uint32_t src = n_models <= 16 ? static_cast<uint32_t>(rest) & 15u : static_cast<uint32_t>(s_perm[n * T_]);
+        if (src == static_cast<uint32_t>(n)) continue;
+        const uint32_t from = img0 + src * img_step;
+        TA::store_elem(a.a, out, TA::kBytes == 4 ? reinterpret_cast<const uint32_t *>(image_a)[from]
+                                                 : reinterpret_cast<const uint16_t *>(image_a)[from]);
+        if constexpr (kHasB)
+            TB::store_elem(a.b, out, TB::kBytes == 4 ? reinterpret_cast<const uint32_t *>(image_b)[from]
+                                                     : reinterpret_cast<const uint16_t *>(image_b)[from]);
+        ++moved;
+    }
+}
+
+// Serving one tile of T groups (one group per thread), in two halves.  `plan_tile` needs no data:
+// it decides how the warp serves the tile and draws permutations; `apply_tile` moves the values
+// once the image has landed.  A kernel may run the first while its copies are still in flight.
+//   dealt  the warp's selected coordinates are listed in shared memory and dealt out to the lanes
+//          32 at a time: with a few selected coordinates per warp (p around 0.01-0.1) one round
+//          serves them all, instead of one divergent pass per coordinate slot; the plan draws the
+//          first round's permutations, later rounds draw theirs when they are served;
+//   dense  half of the warp's coordinates or more selected (and every such group whole): dealing
+//          would take two rounds or more, in each of which a lane draws one permutation and stores
+//          4-byte values; every lane serving its own group costs less from there on.
+// Both are called by all threads of the block.
+struct TilePlan {
+    uint32_t mode;      // kServeNothing / kServeDealt / kServeDense: the same on every lane of a warp
+    uint32_t total;     // dealt: selected coordinates of the warp
+    uint32_t entry;     // dealt: the lane's coordinate of the first round, owner lane * 4 + coordinate slot
+    uint64_t perm[4];   // dense: the permutations of the lane's four coordinates; dealt: [0] is the entry's (N <= 16)
+};
+constexpr uint32_t kServeNothing = 0, kServeDealt = 1, kServeDense = 2;
+
+__device__ __forceinline__ void plan_tile(const ShuffleArgs &a, uint8_t *s_list, uint8_t *s_perm, uint32_t sel, const GroupInfo &gi,
+                                          TilePlan &pl, uint32_t &selected, uint32_t &moved)
+{
+    const int n_models = a.pop.N;
+    const uint32_t T_ = blockDim.x;
+    const uint32_t lane = threadIdx.x & 31u;
+    pl.mode = kServeNothing;
+    if (!__any_sync(0xFFFFFFFFu, sel != 0)) return;   // most warps have nothing selected at small p
+    const uint32_t mine = __popc(sel);
+    const uint32_t total = __reduce_add_sync(0xFFFFFFFFu, mine);
+    if (total >= kDenseMinSelected && __all_sync(0xFFFFFFFFu, sel == 0 || gi.valid == 4)) {
+        pl.mode = kServeDense;
+        if (sel) {
+            if (n_models <= 16) dense_draw<uint64_t>(a, sel, gi, pl.perm, selected, moved);
+            else {
+                dense_bytes_draw(a, s_perm, sel, gi.cgroup, gi.tensor_id);
+                selected += __popc(sel);
+            }
+        }
+        return;
+    }
+    pl.mode = kServeDealt;
+    pl.total = total;
+    uint32_t upto = mine;   // inclusive prefix sum over the lanes
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+        const uint32_t v = __shfl_up_sync(0xFFFFFFFFu, upto, d);
+        if (lane >= static_cast<uint32_t>(d)) upto += v;
+    }
+    uint8_t *list = s_list + (threadIdx.x >> 5) * 128;   // entry = owner lane * 4 + coordinate slot
+    uint32_t pos = upto - mine;
+#pragma unroll
+    for (int c = 0; c < 4; ++c)
+        if ((sel >> c) & 1u) list[pos++] = static_cast<uint8_t>(lane * 4 + c);
+    __syncwarp();
+    const bool active = lane < total;
+    pl.entry = active ? list[lane] : 0u;
+    const uint32_t owner = pl.entry >> 2, c = pl.entry & 3u;
+    const uint32_t cgroup = __shfl_sync(0xFFFFFFFFu, gi.cgroup, owner);
+    const uint32_t tensor = __shfl_sync(0xFFFFFFFFu, gi.tensor_id, owner);
+    if (active) {
+        if (n_models <= 16) pl.perm[0] = draw_permutation_packed(n_models, 4u * cgroup + c, tensor, a.step_lo, a.step_hi8, a.keys);
+        else draw_permutation_u8(s_perm, T_, n_models, 4u * cgroup + c, tensor, a.step_lo, a.step_hi8, a.keys);
+        ++selected;
+    }
+}
+
+template <class TA, class TB, int LAYOUT>
+__device__ __forceinline__ void apply_tile(const ShuffleArgs &a, const unsigned char *image_a, const unsigned char *image_b,
+                                           uint8_t *s_list, uint8_t *s_perm, uint64_t g_block, uint32_t sel, const GroupInfo &gi,
+                                           TilePlan &pl, uint32_t &selected, uint32_t &moved)
+{
+    const int n_models = a.pop.N;
+    const uint32_t T_ = blockDim.x;
+    const uint32_t lane = threadIdx.x & 31u, warp_base = threadIdx.x & ~31u;
+    if (pl.mode == kServeNothing) return;
+    if (pl.mode == kServeDense) {
+        if (sel) {
+            if (n_models <= 16) dense_write<TA, TB, LAYOUT, uint64_t>(a, image_a, image_b, g_block, pl.perm);
+            else moved += dense_bytes_write<TA, TB, LAYOUT>(a, image_a, image_b, s_perm, g_block);
+        }
+        return;
+    }
+    if (lane < pl.total) move_coordinate<TA, TB, LAYOUT>(a, image_a, image_b, s_perm, pl.perm[0], warp_base + (pl.entry >> 2), pl.entry & 3u, g_block, moved);
+    const uint8_t *list = s_list + (threadIdx.x >> 5) * 128;
+    for (uint32_t first = 32; first < pl.total; first += 32) {   // further rounds: draw and move
+        const bool active = first + lane < pl.total;
+        const uint32_t entry = active ? list[first + lane] : 0u;
+        const uint32_t owner = entry >> 2, c = entry & 3u;
+        const uint32_t cgroup = __shfl_sync(0xFFFFFFFFu, gi.cgroup, owner);
+        const uint32_t tensor = __shfl_sync(0xFFFFFFFFu, gi.tensor_id, owner);
+        if (!active) continue;
+        uint64_t perm = 0;
+        if (n_models <= 16) perm = draw_permutation_packed(n_models, 4u * cgroup + c, tensor, a.step_lo, a.step_hi8, a.keys);
+        else draw_permutation_u8(s_perm, T_, n_models, 4u * cgroup + c, tensor, a.step_lo, a.step_hi8, a.keys);
+        move_coordinate<TA, TB, LAYOUT>(a, image_a, image_b, s_perm, perm, warp_base + owner, c, g_block, moved);
+        ++selected;
+    }
+    __syncwarp();   // the warp's list is rewritten by the next tile
+}
+
+// ---- the lean flavour's serving: everything after the wait, in one piece --------------------
+// (The early flavour splits the same work in two halves around the wait, see plan_tile.  The lean
+// one is compiled for 48 registers so that as many blocks stay resident as the shared memory
+// allows; it keeps a permutation in a 32-bit register where it can and serves N > 16 by dealing.)
+template <class TA, class TB, int LAYOUT, class PERM>
+__device__ __forceinline__ void serve_group_dense(const ShuffleArgs &a, const unsigned char *image_a, const unsigned char *image_b,
+                                                  uint64_t g_block, uint32_t sel, const GroupInfo &gi, uint32_t &selected, uint32_t &moved)
+{
+    PERM perm[4];
+    dense_draw<PERM>(a, sel, gi, perm, selected, moved);
+    dense_write<TA, TB, LAYOUT, PERM>(a, image_a, image_b, g_block, perm);
+}
+
 template <class TA, class TB, int LAYOUT>
 __device__ __forceinline__ void serve_tile(const ShuffleArgs &a, const unsigned char *image_a, const unsigned char *image_b,
                                            uint8_t *s_list, uint8_t *s_perm, uint64_t g_block,
                                            uint32_t sel, const GroupInfo &gi, uint32_t &selected, uint32_t &moved)
 {
-    constexpr bool kHasB = TB::kCode != kDtypeNone;
     const int n_models = a.pop.N;
     const uint32_t T_ = blockDim.x;
     const uint32_t lane = threadIdx.x & 31u, warp_base = threadIdx.x & ~31u;
     if (!__any_sync(0xFFFFFFFFu, sel != 0)) return;   // most warps have nothing selected at small p
     const uint32_t mine = __popc(sel);
-    // Half of the warp's coordinates or more selected: dealing them out would take two rounds or
-    // more, in each of which a lane draws one permutation and stores 4-byte values; every lane
-    // serving its own group costs less from there on (measured crossover near 64 of 128).
-    // (In the moved-values count of the byte version an unselected coordinate adds nothing: its
-    // column stays the identity.)
-    if (__reduce_add_sync(0xFFFFFFFFu, mine) >= kDenseMinSelected && __all_sync(0xFFFFFFFFu, sel == 0 || gi.valid == 4)) {
+    if (n_models <= 16 && __reduce_add_sync(0xFFFFFFFFu, mine) >= kDenseMinSelected &&
+        __all_sync(0xFFFFFFFFu, sel == 0 || gi.valid == 4)) {
         if (sel) {
             if (n_models <= 8) serve_group_dense<TA, TB, LAYOUT, uint32_t>(a, image_a, image_b, g_block, sel, gi, selected, moved);
-            else if (n_models <= 16) serve_group_dense<TA, TB, LAYOUT, uint64_t>(a, image_a, image_b, g_block, sel, gi, selected, moved);
-            else serve_group_dense_bytes<TA, TB, LAYOUT>(a, image_a, image_b, s_perm, g_block, sel, gi, selected, moved);
+            else serve_group_dense<TA, TB, LAYOUT, uint64_t>(a, image_a, image_b, g_block, sel, gi, selected, moved);
         }
         return;
     }
@@ -316,30 +468,10 @@ __device__ __forceinline__ void serve_tile(const ShuffleArgs &a, const unsigned 
         const uint32_t cgroup = __shfl_sync(0xFFFFFFFFu, gi.cgroup, owner);
         const uint32_t tensor = __shfl_sync(0xFFFFFFFFu, gi.tensor_id, owner);
         if (!active) continue;
-        const uint32_t t_owner = warp_base + owner;
-        const long long e = 4ll * static_cast<long long>(g_block + t_owner) + c;
         uint64_t perm = 0;
         if (n_models <= 16) perm = draw_permutation_packed(n_models, 4u * cgroup + c, tensor, a.step_lo, a.step_hi8, a.keys);
         else draw_permutation_u8(s_perm, T_, n_models, 4u * cgroup + c, tensor, a.step_lo, a.step_hi8, a.keys);
-        // model n's value of this coordinate sits at out0 + n*out_step in the stack and at
-        // element img0 + n*img_step of the image: no multiplication left inside the loop
-        const long long out_step = LAYOUT == kLayoutNP ? a.pop.padded_P : 1;
-        const long long out0 = LAYOUT == kLayoutNP ? e : e * n_models;
-        const uint32_t img_step = LAYOUT == kLayoutNP ? T_ * 4u : 1u;
-        const uint32_t img0 = LAYOUT == kLayoutNP ? t_owner * 4u + c : t_owner * pn_group_elems(n_models, a.pn_pad) + c * n_models;
-        long long out = out0;
-        uint64_t rest = perm;   // nibble n on top of the low end when model n's turn comes
-        for (int n = 0; n < n_models; ++n, out += out_step, rest >>= 4) {
-            const uint32_t src = n_models <= 16 ? static_cast<uint32_t>(rest) & 15u : static_cast<uint32_t>(s_perm[n * T_]);
-            if (src == static_cast<uint32_t>(n)) continue;
-            const uint32_t from = img0 + src * img_step;
-            TA::store_elem(a.a, out, TA::kBytes == 4 ? reinterpret_cast<const uint32_t *>(image_a)[from]
-                                                     : reinterpret_cast<const uint16_t *>(image_a)[from]);
-            if constexpr (kHasB)
-                TB::store_elem(a.b, out, TB::kBytes == 4 ? reinterpret_cast<const uint32_t *>(image_b)[from]
-                                                         : reinterpret_cast<const uint16_t *>(image_b)[from]);
-            ++moved;
-        }
+        move_coordinate<TA, TB, LAYOUT>(a, image_a, image_b, s_perm, perm, warp_base + owner, c, g_block, moved);
         ++selected;
     }
     __syncwarp();   // the warp's list is rewritten by the next tile
@@ -435,8 +567,12 @@ __device__ __forceinline__ void consensus_tile(const ShuffleArgs &a, const unsig
 // G = tiles per block (one group per thread and tile).  Small populations move few bytes per
 // group (N * 16 for fp32), so a thread takes G = 2 groups, T apart, to keep more bytes in
 // flight per SM; the two Philox draws overlap as well.
-template <class TA, class TB, int LAYOUT, int G, bool STAT>
-__global__ void __launch_bounds__(256, 5) shuffle_async_kernel(const __grid_constant__ ShuffleArgs a)
+// EARLY: the tile's serving is planned (permutations drawn) before the wait for the copies, so that
+// the integer work of a launch that selects much hides behind the copies' flight instead of holding
+// the block's shared memory after them; it keeps a plan in registers across the wait, which the
+// lean flavour (48 registers, as many resident blocks as the shared memory allows) cannot afford.
+template <class TA, class TB, int LAYOUT, int G, bool STAT, bool EARLY>
+__global__ void __launch_bounds__(256, EARLY ? 3 : 5) shuffle_async_kernel(const __grid_constant__ ShuffleArgs a)
 {
     extern __shared__ __align__(128) unsigned char smem_raw[];
     constexpr bool kHasB = TB::kCode != kDtypeNone;
@@ -446,8 +582,8 @@ __global__ void __launch_bounds__(256, 5) shuffle_async_kernel(const __grid_cons
     const size_t group_elems = LAYOUT == kLayoutPN ? pn_group_elems(n_models, a.pn_pad) : 4u * static_cast<size_t>(n_models);
     const size_t a_bytes = group_elems * T_ * TA::kBytes;
     const size_t b_bytes = kHasB ? group_elems * T_ * TB::kBytes : 0;
-    uint8_t *s_list = smem_raw + G * (a_bytes + b_bytes);   // 128 bytes per warp
-    uint8_t *s_perm = s_list + 4 * T_ + threadIdx.x;        // four columns [c][n][T] of bytes, used when N > 16
+    uint8_t *s_list = smem_raw + G * (a_bytes + b_bytes);   // 128 bytes per warp and tile
+    uint8_t *s_perm = s_list + G * 4 * T_ + threadIdx.x;    // four columns [c][n][T] of bytes, used when N > 16
 
     const uint64_t g_first = a.group_lo + static_cast<uint64_t>(blockIdx.x) * (T_ * G);
     uint32_t in_tile[G];   // groups of tile i that exist
@@ -487,20 +623,35 @@ __global__ void __launch_bounds__(256, 5) shuffle_async_kernel(const __grid_cons
     // A selected coordinate is served by whichever lane of the warp gets it, so the warp
     // must see each other's copies; in the [P][N] image a group's values were copied by
     // threads of other warps, so there a block-wide barrier is needed instead.
-    cp_async_wait_all();
     constexpr bool kSharedCopies = LAYOUT == kLayoutPN;   // a group's bytes were copied by threads of other warps
-    if (kSharedCopies) __syncthreads();
-    else __syncwarp();
-    if constexpr (STAT) {
+    if constexpr (EARLY) {
+        TilePlan plan[G];
 #pragma unroll
-        for (int i = 0; i < G; ++i)
-            consensus_tile<TA, LAYOUT>(a, smem_raw + i * (a_bytes + b_bytes), gi[i], threadIdx.x < in_tile[i]);
-    }
+        for (int i = 0; i < G; ++i) plan_tile(a, s_list + i * 4 * T_, s_perm, sel[i], gi[i], plan[i], selected, moved);
+        cp_async_wait_all();
+        if (kSharedCopies) __syncthreads();
+        else __syncwarp();
 #pragma unroll
-    for (int i = 0; i < G; ++i) {
-        const unsigned char *image_a = smem_raw + i * (a_bytes + b_bytes);
-        serve_tile<TA, TB, LAYOUT>(a, image_a, image_a + a_bytes, s_list, s_perm,
-                                   g_first + static_cast<uint64_t>(i) * T_, sel[i], gi[i], selected, moved);
+        for (int i = 0; i < G; ++i) {
+            const unsigned char *image_a = smem_raw + i * (a_bytes + b_bytes);
+            apply_tile<TA, TB, LAYOUT>(a, image_a, image_a + a_bytes, s_list + i * 4 * T_, s_perm,
+                                       g_first + static_cast<uint64_t>(i) * T_, sel[i], gi[i], plan[i], selected, moved);
+        }
+    } else {
+        cp_async_wait_all();
+        if (kSharedCopies) __syncthreads();
+        else __syncwarp();
+        if constexpr (STAT) {
+#pragma unroll
+            for (int i = 0; i < G; ++i)
+                consensus_tile<TA, LAYOUT>(a, smem_raw + i * (a_bytes + b_bytes), gi[i], threadIdx.x < in_tile[i]);
+        }
+#pragma unroll
+        for (int i = 0; i < G; ++i) {
+            const unsigned char *image_a = smem_raw + i * (a_bytes + b_bytes);
+            serve_tile<TA, TB, LAYOUT>(a, image_a, image_a + a_bytes, s_list, s_perm,
+                                       g_first + static_cast<uint64_t>(i) * T_, sel[i], gi[i], selected, moved);
+        }
     }
     publish_block_stats(a.stats, a.stat_slots, selected, moved);
 }
@@ -512,7 +663,8 @@ cudaError_t launch_shuffle_async_tiles(const ShuffleArgs &args, const LaunchShap
     // a group's values in both images (with the launch's padding per group and stack in [P][N])
     const size_t group_elems = 4 * static_cast<size_t>(args.pop.N) + (args.pop.layout == kLayoutPN ? args.pn_pad : 0);
     const size_t image = group_elems * (TA::kBytes + (kHasB ? TB::kBytes : 0));
-    const size_t per_thread = image * G + (args.pop.N > 16 ? 4 * args.pop.N : 0) + 4;   // images, the permutation columns (N > 16), the warp's list
+    // images, the permutation columns of bytes (N > 16: one, four in the early flavour), the warps' lists
+    const size_t per_thread = image * G + (args.pop.N > 16 ? (args.early ? 4 : 1) * args.pop.N : 0) + 4 * G;
     // block size: as many threads as keep a block's image near 44 KiB, so that five blocks
     // (about 200 KiB in flight) share an SM
     int threads = shape.threads > 0 ? shape.threads : 64;   // measured: 64 beats 128 and 256 (a block holds its shared memory until its slowest thread is done)
@@ -521,8 +673,10 @@ cudaError_t launch_shuffle_async_tiles(const ShuffleArgs &args, const LaunchShap
         while (threads > 32 && per_thread * threads > 44 * 1024) threads >>= 1;
     const size_t smem = (per_thread * threads + 15) & ~static_cast<size_t>(15);
     const bool np = args.pop.layout == kLayoutNP;
-    auto kernel = args.sq.slots ? (np ? shuffle_async_kernel<TA, TB, kLayoutNP, G, true> : shuffle_async_kernel<TA, TB, kLayoutPN, G, true>)
-                                : (np ? shuffle_async_kernel<TA, TB, kLayoutNP, G, false> : shuffle_async_kernel<TA, TB, kLayoutPN, G, false>);
+    constexpr bool kEarlyBuilt = G == 1;   // the early flavour exists for one group per thread (what large populations get)
+    auto kernel = np ? shuffle_async_kernel<TA, TB, kLayoutNP, G, false, false> : shuffle_async_kernel<TA, TB, kLayoutPN, G, false, false>;
+    if (args.sq.slots) kernel = np ? shuffle_async_kernel<TA, TB, kLayoutNP, G, true, false> : shuffle_async_kernel<TA, TB, kLayoutPN, G, true, false>;
+    else if (args.early && kEarlyBuilt) kernel = np ? shuffle_async_kernel<TA, TB, kLayoutNP, 1, false, true> : shuffle_async_kernel<TA, TB, kLayoutPN, 1, false, true>;
     KernelFit fit;
     cudaError_t err = kernel_fit(reinterpret_cast<const void *>(kernel), threads, smem, &fit);
     if (err != cudaSuccess) return err;

@@ -71,6 +71,30 @@ def test_shuffle_both_stacks_and_dtypes(dtype, opt_dtype, layout, mode):
     c.close()
 
 
+@pytest.mark.parametrize("flavour", [-2, -3], ids=["lean", "early"])
+@pytest.mark.parametrize("layout", [0, 1])
+@pytest.mark.parametrize("N,dtype,opt_dtype", [(5, "f32", "f32"), (16, "f32", None), (17, "f32", "f32"), (33, "bf16", "f32"), (64, "f32", None)])
+def test_streaming_flavours_on_dense_and_mixed_selection(N, dtype, opt_dtype, layout, flavour):
+    """The streaming kernel's two flavours (permutations drawn after or before the wait for the
+    copies; the early one serves N > 16 densely from byte columns) on tensors that are selected
+    in full, mostly, half, rarely and not at all, with ragged ends."""
+    numel = [9000, 33, 4100, 7, 2600, 1, 5003]
+    p_layer = [1.0, 1.0, 0.9, 0.5, 0.45, 1.0, 0.02]
+    c = Case(N, numel, layout, dtype, opt_dtype, seed=40 + N)
+    B.wash_set_launch(c.gpu.ctx, 0, flavour)
+    tot = [0, 0]
+    for step in (0, 1, (3 << 32) | 9):
+        if opt_dtype is None:
+            B.wash_shuffle(c.gpu.ctx, step, 0.0, p_layer, seed=123, stats=c.stats_dev)
+        else:
+            B.wash_shuffle_both(c.gpu.ctx, step, 0.0, p_layer, seed=123, stats=c.stats_dev)
+        s = oracle.shuffle(c.ora, c.host, p_layer, seed=123, step=step, stack2=c.host_opt)
+        tot[0] += s[0]; tot[1] += s[1]
+        c.assert_equal("N=%d layout=%d step=%d" % (N, layout, step))
+    assert c.gpu_stats() == tuple(tot)
+    c.close()
+
+
 @pytest.mark.parametrize("layout", [0, 1])
 def test_separate_calls_equal_the_fused_call(layout):
     N = 8
@@ -93,7 +117,7 @@ def test_sparse_mode_and_launch_shapes_give_the_same_bits(N):
     ref = Case(N, RAGGED, 0, seed=8)
     oracle.shuffle(ref.ora, ref.host, 0.1, seed=2, step=3)
     for mode in (B.WASH_MODE_STREAM, B.WASH_MODE_SPARSE, B.WASH_MODE_AUTO):
-        for threads, bps in ((0, 0), (64, 1), (128, 2), (256, -1), (96, 0), (32, 4), (256, 2), (128, 1)):
+        for threads, bps in ((0, 0), (64, 1), (128, 2), (256, -1), (96, 0), (32, 4), (256, 2), (128, 1), (0, -2), (0, -3), (128, -3)):
             c = Case(N, RAGGED, 0, seed=8)
             B.wash_set_mode(c.gpu.ctx, mode)
             B.wash_set_launch(c.gpu.ctx, threads, bps)
