@@ -385,7 +385,8 @@ const char *wash_last_error(void);
  * wash_shuffle for tensor 0 at step 0 with key = seed) and folds them into one word,
  * which it adds to *dev_checksum (DEVICE, uint32, caller-zeroed; may be NULL).  Timing it
  * gives the rate at which masks can be drawn when memory costs nothing, i.e. the bound
- * that takes over from HBM for small N.  No stack is touched.  Diagnostic only. */
+ * that takes over from HBM for small N.  A thread draws four blocks (four independent
+ * chains, the form that measured fastest).  No stack is touched.  Diagnostic only. */
 int wash_philox_probe(uint64_t n_blocks, uint64_t seed, uint32_t *dev_checksum, int32_t device, void *stream);
 
 /* Number of kernels this library has launched in this process. */

@@ -73,14 +73,19 @@ cudaError_t launch_sq_flush(const SqArgs &sq, int N, double *out, cudaStream_t s
     return cudaGetLastError();
 }
 
-// Nothing but the mask's Philox blocks: one block of four words per thread, folded by XOR.
+// Nothing but the mask's Philox blocks: four blocks per thread (four independent chains, as in the
+// kernels that draw masks without touching memory), folded by XOR.  With one block per thread the
+// same kernel measures a quarter less (3.17 against 4.2e11 blocks/s): the chains' latency shows.
 __global__ void __launch_bounds__(256) philox_probe_kernel(unsigned long long n_blocks, const __grid_constant__ PhiloxKeys keys, uint32_t *checksum)
 {
-    const unsigned long long i = static_cast<unsigned long long>(blockIdx.x) * blockDim.x + threadIdx.x;
+    const unsigned long long i = (static_cast<unsigned long long>(blockIdx.x) * blockDim.x + threadIdx.x) * 4ull;
     uint32_t fold = 0;
-    if (i < n_blocks) {
-        const Philox4 w = philox4x32_10(static_cast<uint32_t>(i), 0u, 0u, static_cast<uint32_t>(i >> 32) << 8, keys);
-        fold = w.x ^ w.y ^ w.z ^ w.w;
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+        if (i + q < n_blocks) {
+            const Philox4 w = philox4x32_10(static_cast<uint32_t>(i + q), 0u, 0u, static_cast<uint32_t>((i + q) >> 32) << 8, keys);
+            fold ^= w.x ^ w.y ^ w.z ^ w.w;
+        }
     }
     fold = __reduce_xor_sync(0xFFFFFFFFu, fold);
     if (checksum && (threadIdx.x & 31) == 0 && fold == 0x9E3779B9u) atomicAdd(checksum, 1u);   // keeps the work alive; rarely true
@@ -89,7 +94,7 @@ __global__ void __launch_bounds__(256) philox_probe_kernel(unsigned long long n_
 cudaError_t launch_philox_probe(unsigned long long n_blocks, uint64_t seed, uint32_t *checksum, cudaStream_t stream)
 {
     if (n_blocks == 0) return cudaSuccess;
-    const unsigned long long grid = (n_blocks + 255) / 256;
+    const unsigned long long grid = ((n_blocks + 3) / 4 + 255) / 256;
     if (grid > 0x7FFFFFFFull) return cudaErrorInvalidConfiguration;
     philox_probe_kernel<<<static_cast<unsigned>(grid), 256, 0, stream>>>(n_blocks, philox_keys(seed), checksum);
     count_launch();
