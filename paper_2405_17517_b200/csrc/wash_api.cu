@@ -272,6 +272,7 @@ int shuffle_impl(wash_ctx *ctx, int which, uint64_t step, double p, const double
         for (int s = 0; s < ctx->n_seg; ++s) coordinates += static_cast<double>(ctx->seg_host[s].numel);
         // [P][N], even N: the streaming kernel pads its shared-memory image against bank conflicts
         // once a fifth of the coordinates is expected to be served from it
+        args.expected_share = coordinates > 0.0 ? static_cast<float>(ctx->expected_selected / coordinates) : 0.f;
         if (ctx->layout == WASH_LAYOUT_PN && !(ctx->N & 1)) args.pn_pad = ctx->expected_selected >= 0.2 * coordinates ? 4u : 0u;
         // The streaming kernel's early flavour (permutations drawn while the copies are in flight, dense
         // serving for N > 16) costs registers and, for N > 16, three more permutation columns of shared

@@ -84,6 +84,7 @@ struct ShuffleArgs {
     SqArgs sq;                    // consensus distance of the first stack (streaming kernel only)
     uint32_t pn_pad = 0;          // streaming kernel, [P][N]: elements of padding after a group in the shared-memory image (0 or 4)
     bool early = false;           // streaming kernel: the flavour that draws permutations while the copies are in flight
+    float expected_share = 0.f;   // share of the coordinates the call's probabilities select, in expectation (sizes the sparse kernel's grid)
 };
 
 struct ReduceArgs {

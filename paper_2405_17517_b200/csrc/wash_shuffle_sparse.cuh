@@ -117,7 +117,19 @@ cudaError_t launch_shuffle_sparse_typed(const ShuffleArgs &args, const LaunchSha
     // one resident wave of blocks, fewer for short rows; the warps share the tiles evenly
     const uint32_t resident = static_cast<uint32_t>(shape.sm_count > 0 ? shape.sm_count : 148) * static_cast<uint32_t>(fit.occupancy);
     const uint32_t want = (p.n_wtiles + kSparseWarps - 1) / kSparseWarps;
-    p.n_blocks = want < resident ? want : resident;
+    // Grid: one resident wave when a warp expects few selected coordinates; up to four waves when it
+    // expects many.  A warp serves its queue in full rounds and once at the end of its range, so with
+    // one wave every warp reaches its (latency-bound) last round at the same time, after the
+    // (multiply-bound) mask; with shorter ranges in several waves the block scheduler overlaps one
+    // wave's serving with the next one's mask and evens out ranges that select unequally (per-layer p).
+    // Measured (1 / 2 / 4 waves): cfg2 21.3 / 26.6 / 35.7 us at 2.4 coordinates a warp, cfg3 77.3 / 71.0 /
+    // 75.6 us at 11, cfg4 104.1 / 94.4 / 89.4 us at 27.  A warp keeps at least two tiles.
+    const double per_warp = static_cast<double>(args.expected_share) * 4.0 * static_cast<double>(args.group_hi - args.group_lo) /
+                            (static_cast<double>(resident) * kSparseWarps);
+    uint32_t waves = per_warp <= 8.0 ? 1u : (per_warp <= 20.0 ? 2u : 4u);
+    while (waves > 1 && p.n_wtiles < 2ull * waves * resident * kSparseWarps) waves >>= 1;
+    const uint32_t cap = resident * waves;
+    p.n_blocks = want < cap ? want : cap;
     kernel<<<p.n_blocks, kSparseThreads, smem, stream>>>(p);
     count_launch();
     return cudaGetLastError();
