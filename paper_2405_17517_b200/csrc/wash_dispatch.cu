@@ -80,9 +80,14 @@ __global__ void __launch_bounds__(256) philox_probe_kernel(unsigned long long n_
 {
     const unsigned long long i = (static_cast<unsigned long long>(blockIdx.x) * blockDim.x + threadIdx.x) * 4ull;
     uint32_t fold = 0;
+    if (i + 3 < n_blocks) {   // the four chains under one condition, so that they interleave
 #pragma unroll
-    for (int q = 0; q < 4; ++q) {
-        if (i + q < n_blocks) {
+        for (int q = 0; q < 4; ++q) {
+            const Philox4 w = philox4x32_10(static_cast<uint32_t>(i + q), 0u, 0u, static_cast<uint32_t>((i + q) >> 32) << 8, keys);
+            fold ^= w.x ^ w.y ^ w.z ^ w.w;
+        }
+    } else {
+        for (int q = 0; q < 4 && i + q < n_blocks; ++q) {
             const Philox4 w = philox4x32_10(static_cast<uint32_t>(i + q), 0u, 0u, static_cast<uint32_t>((i + q) >> 32) << 8, keys);
             fold ^= w.x ^ w.y ^ w.z ^ w.w;
         }
