@@ -63,7 +63,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
     os.makedirs(BUILD, exist_ok=True)
     jobs = [(os.path.join(CSRC, "wash_api.cu"), os.path.join(BUILD, "wash_api.o"), [], verbose),
             (os.path.join(CSRC, "wash_dispatch.cu"), os.path.join(BUILD, "wash_dispatch.o"), [], verbose)]
-    for name in ("wash_noalloc", "wash_shuffle", "wash_exchange"):
+    for name in ("wash_noalloc", "wash_shuffle", "wash_shuffle_loop", "wash_exchange"):
         jobs.append((os.path.join(CSRC, name + ".cu"), os.path.join(BUILD, name + ".o"), [], verbose))
     for n in [0] + population_sizes():
         jobs.append((os.path.join(CSRC, "wash_inst.cu"), os.path.join(BUILD, "wash_inst_n%d.o" % n), ["-DWASH_N=%d" % n], verbose))

@@ -11,6 +11,7 @@ WASH_N_LIST(WASH_DECL)
 #undef WASH_DECL
 cudaError_t launch_shuffle_sparse(const ShuffleArgs &, int, int, const LaunchShape &, cudaStream_t, bool *);
 cudaError_t launch_shuffle_stream(const ShuffleArgs &, int, int, const LaunchShape &, cudaStream_t, bool *);
+cudaError_t launch_shuffle_stream_loop(const ShuffleArgs &, int, int, const LaunchShape &, cudaStream_t, bool *);
 cudaError_t launch_reduce_n0(const ReduceArgs &, int, int, int, const LaunchShape &, cudaStream_t, bool *);
 
 static std::atomic<uint64_t> g_launches{0};
@@ -110,6 +111,17 @@ static cudaError_t launch_shuffle_kernel(const ShuffleArgs &args, int a_dtype, i
                                          const LaunchShape &shape, cudaStream_t stream, bool *supported)
 {
     if (mode == kModeSparse) return launch_shuffle_sparse(args, a_dtype, b_dtype, shape, stream, supported);
+    // Two streaming kernels.  A group of all models (both stacks) of at most kLoopMaxGroupBytes goes to the
+    // resident-warp kernel, whose instruction count per group is a fraction of the one-trip kernel's, unless
+    // most coordinates are expected to be served (there the one-trip kernel measured 6 % faster); larger
+    // groups, the consensus statistic and the early flavour stay with the one-trip kernel.
+    // blocks_per_sm of wash_set_launch: -4 forces the resident-warp kernel, -5 the one-trip kernel.
+    const size_t elem_a = a_dtype == kDtypeF32 ? 4 : a_dtype == kDtypeBF16 ? 2 : 0, elem_b = b_dtype == kDtypeF32 ? 4 : b_dtype == kDtypeBF16 ? 2 : 0;
+    const size_t per_group = static_cast<size_t>(args.pop.N) * 4 * (elem_a + elem_b);
+    bool loop = per_group <= kLoopMaxGroupBytes && args.expected_share <= kLoopMaxShare;
+    if (shape.blocks_per_sm == -4) loop = true;
+    if (shape.blocks_per_sm == -5 || args.sq.slots || args.early) loop = false;
+    if (loop) return launch_shuffle_stream_loop(args, a_dtype, b_dtype, shape, stream, supported);
     return launch_shuffle_stream(args, a_dtype, b_dtype, shape, stream, supported);
 }
 

@@ -129,6 +129,12 @@ cudaError_t launch_exchange_receive(const ExchangeArgs &args, cudaStream_t strea
 
 enum ReduceOp { kOpEma = 0, kOpAverage = 1, kOpPapaAll = 2, kOpConsensus = 3 };
 
+// The resident-warp streaming kernel takes groups (all models, both stacks) of up to 48 bytes -- fp32 N = 2, 3;
+// bf16 N <= 6 -- when at most 30 % of the coordinates are expected to be selected.  Measured on 2^27 coordinates
+// against the one-trip kernel: 32 bytes 0.73-0.93 of its time, 48 bytes 0.89-0.98, 64 bytes 0.97-1.12.
+constexpr size_t kLoopMaxGroupBytes = 48;
+constexpr float kLoopMaxShare = 0.3f;
+
 struct LaunchShape {
     int threads;         // 0 = default
     int blocks_per_sm;   // <= 0: one group per thread; > 0: persistent grid, that many blocks per SM

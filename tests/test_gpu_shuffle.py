@@ -95,6 +95,32 @@ def test_streaming_flavours_on_dense_and_mixed_selection(N, dtype, opt_dtype, la
     c.close()
 
 
+@pytest.mark.parametrize("code", [-4, -5, 0], ids=["resident", "one-trip", "default"])
+@pytest.mark.parametrize("layout", [0, 1])
+@pytest.mark.parametrize("N,dtype,opt_dtype", [(2, "f32", None), (2, "bf16", "f32"), (3, "f32", "f32"), (4, "bf16", None), (8, "f32", None), (17, "bf16", "bf16")])
+def test_resident_warp_streaming_kernel(N, dtype, opt_dtype, layout, code):
+    """The streaming kernel for small groups (a resident grid of warps walking tiles with two
+    shared-memory stages), forced, excluded and as the library chooses, against the oracle: enough
+    coordinates for several trips per warp, tensors selected in full, half, rarely and not at
+    all, ragged ends, a tensor boundary inside a tile."""
+    numel = [2_600_003 if N <= 4 else 200_003, 33, 4100, 7, 260_000, 1, 5003, 90_001]
+    p_layer = [0.004, 1.0, 0.9, 0.5, 0.3, 1.0, 0.0, 1.0]
+    c = Case(N, numel, layout, dtype, opt_dtype, seed=70 + N)
+    B.wash_set_launch(c.gpu.ctx, 0, code)
+    tot = [0, 0]
+    for step in (0, 1, (5 << 32) | 2):
+        if opt_dtype is None:
+            B.wash_shuffle(c.gpu.ctx, step, 0.0, p_layer, seed=77, stats=c.stats_dev)
+        else:
+            B.wash_shuffle_both(c.gpu.ctx, step, 0.0, p_layer, seed=77, stats=c.stats_dev)
+        s = oracle.shuffle(c.ora, c.host, p_layer, seed=77, step=step, stack2=c.host_opt)
+        tot[0] += s[0]; tot[1] += s[1]
+        c.assert_equal("N=%d layout=%d step=%d" % (N, layout, step))
+    assert c.gpu_stats() == tuple(tot)
+    B.wash_check(c.gpu.ctx)
+    c.close()
+
+
 @pytest.mark.parametrize("layout", [0, 1])
 def test_separate_calls_equal_the_fused_call(layout):
     N = 8
@@ -117,7 +143,7 @@ def test_sparse_mode_and_launch_shapes_give_the_same_bits(N):
     ref = Case(N, RAGGED, 0, seed=8)
     oracle.shuffle(ref.ora, ref.host, 0.1, seed=2, step=3)
     for mode in (B.WASH_MODE_STREAM, B.WASH_MODE_SPARSE, B.WASH_MODE_AUTO):
-        for threads, bps in ((0, 0), (64, 1), (128, 2), (256, -1), (96, 0), (32, 4), (256, 2), (128, 1), (0, -2), (0, -3), (128, -3)):
+        for threads, bps in ((0, 0), (64, 1), (128, 2), (256, -1), (96, 0), (32, 4), (256, 2), (128, 1), (0, -2), (0, -3), (128, -3), (0, -4), (0, -5)):
             c = Case(N, RAGGED, 0, seed=8)
             B.wash_set_mode(c.gpu.ctx, mode)
             B.wash_set_launch(c.gpu.ctx, threads, bps)
