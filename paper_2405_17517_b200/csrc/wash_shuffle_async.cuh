@@ -430,6 +430,34 @@ __device__ __forceinline__ void serve_group_dense(const ShuffleArgs &a, const un
     dense_write<TA, TB, LAYOUT, PERM>(a, image_a, image_b, g_block, perm);
 }
 
+// A warp with one selected coordinate in its tile (the usual case from p = 1e-3 to 1e-2): no list and
+// no dealing.  Every lane draws the coordinate's permutation (the same instructions for all, so
+// nothing diverges) and lane n moves model n's value: one load and one store per lane instead of N
+// of each on a single lane.  N <= 16.  (Serving two to four coordinates this way, one after the
+// other, measured 1-30 % slower than dealing them.)
+template <class TA, class TB, int LAYOUT>
+__device__ __forceinline__ void serve_single(const ShuffleArgs &a, const unsigned char *image_a, const unsigned char *image_b,
+                                             uint64_t g_block, uint32_t sel, const GroupInfo &gi, uint32_t &selected, uint32_t &moved)
+{
+    constexpr bool kHasB = TB::kCode != kDtypeNone;
+    const int n_models = a.pop.N;
+    const uint32_t lane = threadIdx.x & 31u, warp_base = threadIdx.x & ~31u;
+    const uint32_t owner = __ffs(__ballot_sync(0xFFFFFFFFu, sel != 0)) - 1;
+    const uint32_t c = __ffs(__shfl_sync(0xFFFFFFFFu, sel, owner)) - 1;
+    const uint32_t cgroup = __shfl_sync(0xFFFFFFFFu, gi.cgroup, owner);
+    const uint32_t tensor = __shfl_sync(0xFFFFFFFFu, gi.tensor_id, owner);
+    const uint64_t perm = draw_permutation_packed(n_models, 4u * cgroup + c, tensor, a.step_lo, a.step_hi8, a.keys);
+    if (lane == 0) ++selected;
+    const uint32_t src = static_cast<uint32_t>(perm >> (4u * (lane & 15u))) & 15u;
+    if (lane >= static_cast<uint32_t>(n_models) || src == lane) return;
+    const uint32_t t_owner = warp_base + owner;
+    const long long e = 4ll * static_cast<long long>(g_block + t_owner) + c;
+    const long long out = elem_index<LAYOUT>(a.pop, static_cast<int>(lane), e);
+    TA::store_elem(a.a, out, image_value<TA, LAYOUT>(image_a, n_models, a.pn_pad, t_owner, static_cast<int>(src), static_cast<int>(c)));
+    if constexpr (kHasB) TB::store_elem(a.b, out, image_value<TB, LAYOUT>(image_b, n_models, a.pn_pad, t_owner, static_cast<int>(src), static_cast<int>(c)));
+    ++moved;
+}
+
 template <class TA, class TB, int LAYOUT>
 __device__ __forceinline__ void serve_tile(const ShuffleArgs &a, const unsigned char *image_a, const unsigned char *image_b,
                                            uint8_t *s_list, uint8_t *s_perm, uint64_t g_block,
@@ -440,8 +468,12 @@ __device__ __forceinline__ void serve_tile(const ShuffleArgs &a, const unsigned 
     const uint32_t lane = threadIdx.x & 31u, warp_base = threadIdx.x & ~31u;
     if (!__any_sync(0xFFFFFFFFu, sel != 0)) return;   // most warps have nothing selected at small p
     const uint32_t mine = __popc(sel);
-    if (n_models <= 16 && __reduce_add_sync(0xFFFFFFFFu, mine) >= kDenseMinSelected &&
-        __all_sync(0xFFFFFFFFu, sel == 0 || gi.valid == 4)) {
+    const uint32_t total = __reduce_add_sync(0xFFFFFFFFu, mine);
+    if (n_models <= 16 && total == 1) {
+        serve_single<TA, TB, LAYOUT>(a, image_a, image_b, g_block, sel, gi, selected, moved);
+        return;
+    }
+    if (n_models <= 16 && total >= kDenseMinSelected && __all_sync(0xFFFFFFFFu, sel == 0 || gi.valid == 4)) {
         if (sel) {
             if (n_models <= 8) serve_group_dense<TA, TB, LAYOUT, uint32_t>(a, image_a, image_b, g_block, sel, gi, selected, moved);
             else serve_group_dense<TA, TB, LAYOUT, uint64_t>(a, image_a, image_b, g_block, sel, gi, selected, moved);
@@ -454,7 +486,6 @@ __device__ __forceinline__ void serve_tile(const ShuffleArgs &a, const unsigned 
         const uint32_t v = __shfl_up_sync(0xFFFFFFFFu, upto, d);
         if (lane >= static_cast<uint32_t>(d)) upto += v;
     }
-    const uint32_t total = __shfl_sync(0xFFFFFFFFu, upto, 31);
     uint8_t *list = s_list + (threadIdx.x >> 5) * 128;   // entry = owner lane * 4 + coordinate slot
     uint32_t pos = upto - mine;
 #pragma unroll

@@ -29,7 +29,7 @@ struct SparseArgs {
 template <class TA, class TB, int LAYOUT>
 __global__ void __launch_bounds__(kSparseThreads, 4) shuffle_sparse_kernel(const __grid_constant__ SparseArgs p)
 {
-    extern __shared__ __align__(16) unsigned char smem_raw[];
+    extern __shared__ __align__(128) unsigned char smem_raw[];
     constexpr bool kHasB = TB::kCode != kDtypeNone;
     const ShuffleArgs &a = p.s;
     const int n_models = a.pop.N;
