@@ -430,32 +430,70 @@ __device__ __forceinline__ void serve_group_dense(const ShuffleArgs &a, const un
     dense_write<TA, TB, LAYOUT, PERM>(a, image_a, image_b, g_block, perm);
 }
 
-// A warp with one selected coordinate in its tile (the usual case from p = 1e-3 to 1e-2): no list and
-// no dealing.  Every lane draws the coordinate's permutation (the same instructions for all, so
-// nothing diverges) and lane n moves model n's value: one load and one store per lane instead of N
-// of each on a single lane.  N <= 16.  (Serving two to four coordinates this way, one after the
-// other, measured 1-30 % slower than dealing them.)
+// One selected coordinate served by the whole warp: the permutation is drawn so that lane n ends up
+// with pi(n), and lane n moves model n's value -- one load and one store per lane instead of N of
+// each on a single lane.  N <= 32.  Called by all lanes with the same arguments.
+//   N <= 8: every lane draws the packed permutation (one or two Philox blocks, the same instructions
+//           on all lanes) and takes its nibble;
+//   N > 8:  lane b draws block b of the coordinate's permutation stream (up to eight blocks side by
+//           side instead of one after the other); the Fisher-Yates steps run on a permutation held
+//           one entry per lane: step k hands lane k's and lane j's entries to each other.
 template <class TA, class TB, int LAYOUT>
-__device__ __forceinline__ void serve_single(const ShuffleArgs &a, const unsigned char *image_a, const unsigned char *image_b,
-                                             uint64_t g_block, uint32_t sel, const GroupInfo &gi, uint32_t &selected, uint32_t &moved)
+__device__ __forceinline__ void serve_coordinate_by_warp(const ShuffleArgs &a, const unsigned char *image_a, const unsigned char *image_b,
+                                                         uint64_t g_block, uint32_t t_owner, uint32_t c, uint32_t cgroup, uint32_t tensor,
+                                                         uint32_t &selected, uint32_t &moved)
 {
     constexpr bool kHasB = TB::kCode != kDtypeNone;
     const int n_models = a.pop.N;
-    const uint32_t lane = threadIdx.x & 31u, warp_base = threadIdx.x & ~31u;
-    const uint32_t owner = __ffs(__ballot_sync(0xFFFFFFFFu, sel != 0)) - 1;
-    const uint32_t c = __ffs(__shfl_sync(0xFFFFFFFFu, sel, owner)) - 1;
-    const uint32_t cgroup = __shfl_sync(0xFFFFFFFFu, gi.cgroup, owner);
-    const uint32_t tensor = __shfl_sync(0xFFFFFFFFu, gi.tensor_id, owner);
-    const uint64_t perm = draw_permutation_packed(n_models, 4u * cgroup + c, tensor, a.step_lo, a.step_hi8, a.keys);
+    const uint32_t lane = threadIdx.x & 31u;
+    uint32_t src;
+    if (n_models <= 8) {
+        const uint32_t perm = draw_permutation_packed32(n_models, 4u * cgroup + c, tensor, a.step_lo, a.step_hi8, a.keys);
+        src = (perm >> (4u * (lane & 7u))) & 15u;
+    } else {
+        const Philox4 w = philox4x32_10(4u * cgroup + c, tensor, a.step_lo, a.step_hi8 | (1u + lane), a.keys);
+        src = lane;
+        int k = n_models - 1;
+        for (uint32_t b = 0; k >= 1; ++b) {
+            const uint32_t r[4] = {__shfl_sync(0xFFFFFFFFu, w.x, b), __shfl_sync(0xFFFFFFFFu, w.y, b),
+                                   __shfl_sync(0xFFFFFFFFu, w.z, b), __shfl_sync(0xFFFFFFFFu, w.w, b)};
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                if (k < 1) break;
+                const uint32_t j = __umulhi(r[q], static_cast<uint32_t>(k + 1));
+                const uint32_t at_k = __shfl_sync(0xFFFFFFFFu, src, k), at_j = __shfl_sync(0xFFFFFFFFu, src, j);
+                src = lane == static_cast<uint32_t>(k) ? at_j : (lane == j ? at_k : src);
+                --k;
+            }
+        }
+    }
     if (lane == 0) ++selected;
-    const uint32_t src = static_cast<uint32_t>(perm >> (4u * (lane & 15u))) & 15u;
     if (lane >= static_cast<uint32_t>(n_models) || src == lane) return;
-    const uint32_t t_owner = warp_base + owner;
     const long long e = 4ll * static_cast<long long>(g_block + t_owner) + c;
     const long long out = elem_index<LAYOUT>(a.pop, static_cast<int>(lane), e);
     TA::store_elem(a.a, out, image_value<TA, LAYOUT>(image_a, n_models, a.pn_pad, t_owner, static_cast<int>(src), static_cast<int>(c)));
     if constexpr (kHasB) TB::store_elem(a.b, out, image_value<TB, LAYOUT>(image_b, n_models, a.pn_pad, t_owner, static_cast<int>(src), static_cast<int>(c)));
     ++moved;
+}
+
+// A warp tile with very few selected coordinates (the usual case from p = 1e-3 to 1e-2): no list and
+// no dealing, the warp serves them one after the other.  `few`: 1 for N <= 16 (two to four
+// coordinates served this way measured 1-30 % slower than dealing them), more for larger
+// populations, where a dealt coordinate costs a lane up to eight Philox blocks in a row, a
+// permutation kept as bytes in shared memory and N loads and stores.
+constexpr uint32_t kFewWide = 3;   // N = 32, 2^25 coordinates, p = 0.01: 0.877 ms with 1, 0.818 with 3, 0.820 with 5; p = 0.03: 1.19, 1.17, 1.22
+template <class TA, class TB, int LAYOUT>
+__device__ __forceinline__ void serve_few(const ShuffleArgs &a, const unsigned char *image_a, const unsigned char *image_b,
+                                          uint64_t g_block, uint32_t sel, const GroupInfo &gi, uint32_t &selected, uint32_t &moved)
+{
+    const uint32_t warp_base = threadIdx.x & ~31u;
+    for (uint32_t owners = __ballot_sync(0xFFFFFFFFu, sel != 0); owners; owners &= owners - 1u) {
+        const uint32_t owner = __ffs(owners) - 1;
+        const uint32_t cgroup = __shfl_sync(0xFFFFFFFFu, gi.cgroup, owner);
+        const uint32_t tensor = __shfl_sync(0xFFFFFFFFu, gi.tensor_id, owner);
+        for (uint32_t bits = __shfl_sync(0xFFFFFFFFu, sel, owner); bits; bits &= bits - 1u)
+            serve_coordinate_by_warp<TA, TB, LAYOUT>(a, image_a, image_b, g_block, warp_base + owner, __ffs(bits) - 1, cgroup, tensor, selected, moved);
+    }
 }
 
 template <class TA, class TB, int LAYOUT>
@@ -469,8 +507,8 @@ __device__ __forceinline__ void serve_tile(const ShuffleArgs &a, const unsigned 
     if (!__any_sync(0xFFFFFFFFu, sel != 0)) return;   // most warps have nothing selected at small p
     const uint32_t mine = __popc(sel);
     const uint32_t total = __reduce_add_sync(0xFFFFFFFFu, mine);
-    if (n_models <= 16 && total == 1) {
-        serve_single<TA, TB, LAYOUT>(a, image_a, image_b, g_block, sel, gi, selected, moved);
+    if (n_models <= 32 && total <= (n_models <= 16 ? 1u : kFewWide)) {
+        serve_few<TA, TB, LAYOUT>(a, image_a, image_b, g_block, sel, gi, selected, moved);
         return;
     }
     if (n_models <= 16 && total >= kDenseMinSelected && __all_sync(0xFFFFFFFFu, sel == 0 || gi.valid == 4)) {
