@@ -128,7 +128,12 @@ int wash_set_mode(wash_ctx *ctx, int32_t mode);
  * (default: 2 when a group of all models is at most 64 bytes, else 1); blocks_per_sm = -2 / -3
  * forces the streaming kernel's lean / early flavour (early draws the permutations while the
  * stack's copies are in flight and serves populations of more than 16 models densely; by
- * default it is launched for N > 16 when the call's probabilities select 30 % or more). */
+ * default it is launched for N > 16 when the call's probabilities select 30 % or more);
+ * blocks_per_sm = -4 / -5 forces / excludes the streaming kernel for small groups (a
+ * resident grid of warps walking tiles through two shared-memory stages; by default
+ * it is launched when a group of all models of both stacks is at most 48 bytes and the
+ * call's probabilities select at most 30 %; it ignores `threads`).  Results do not
+ * depend on any of this. */
 int wash_set_launch(wash_ctx *ctx, int32_t threads, int32_t blocks_per_sm);
 
 /* ---- the shuffling step ----------------------------------------------------------- */
