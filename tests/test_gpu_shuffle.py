@@ -190,9 +190,11 @@ def test_last_layer_untouched_and_schedules_agree_with_oracle():
     c.close()
 
 
-def test_shards_reproduce_the_unsharded_shuffle():
-    """Coordinate shards keyed by the global (tensor, coordinate) need no communication."""
-    N, numel = 4, [4000, 1000, 36]
+@pytest.mark.parametrize("N", [2, 4])
+def test_shards_reproduce_the_unsharded_shuffle(N):
+    """Coordinate shards keyed by the global (tensor, coordinate) need no communication
+    (N = 2 goes through the streaming kernel for small groups, N = 4 through the one-trip kernel)."""
+    numel = [4000, 1000, 36]
     full = Case(N, numel, 0, seed=6)
     dense = W.from_stack(full.host, N, numel, full.off, full.P)
     oracle.shuffle(full.ora, full.host, 0.3, seed=77, step=5)
