@@ -633,6 +633,7 @@ __device__ __forceinline__ void consensus_tile(const ShuffleArgs &a, const unsig
     else consensus_warp<T, LAYOUT, false>(a, image, exists ? gi.valid : 0, r1, r_lo, r_hi);
 }
 
+#ifndef WASH_SERVING_ONLY   // a translation unit that only wants the copy and serving helpers above
 // G = tiles per block (one group per thread and tile).  Small populations move few bytes per
 // group (N * 16 for fp32), so a thread takes G = 2 groups, T apart, to keep more bytes in
 // flight per SM; the two Philox draws overlap as well.
@@ -787,5 +788,7 @@ inline cudaError_t launch_shuffle_async(const ShuffleArgs &args, int a_dtype, in
     *supported = false;
     return cudaSuccess;
 }
+
+#endif  // WASH_SERVING_ONLY
 
 }  // namespace wash

@@ -15,6 +15,7 @@
 // The image of a stage is the one-trip kernel's block image with T = 32 (the block is one warp,
 // so every helper of that kernel -- copies, serving, padding rule -- is used as it is).
 #pragma once
+#define WASH_SERVING_ONLY
 #include "wash_shuffle_async.cuh"
 
 namespace wash {
