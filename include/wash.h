@@ -61,10 +61,12 @@ enum wash_mode {
                              per-thread asynchronous copies (cp.async).  Default.            */
     WASH_MODE_SPARSE = 1, /* draws the mask first; touches only selected coordinates          */
     WASH_MODE_AUTO = 2             /* SPARSE when the call's probabilities select, in expectation,
-                                      fewer than 3 % of the coordinates of an [N][padded_P] stack
-                                      or 10 % of a [padded_P][N] stack, else STREAM (the measured
+                                      less than a share of the coordinates that depends on layout
+                                      and N, else STREAM.  [N][padded_P]: max(3 %, 35 % / N);
+                                      [padded_P][N]: 30 % up to N = 8, 10 % above (the measured
                                       crossovers on B200: in the second layout the N values of a
-                                      coordinate share a DRAM access)                            */
+                                      coordinate share a DRAM access; a small population leaves
+                                      the streaming kernel bound by issue slots)                 */
 };
 
 #define WASH_MAX_N 64            /* largest population                                     */

@@ -263,9 +263,11 @@ int shuffle_impl(wash_ctx *ctx, int which, uint64_t step, double p, const double
         if (ctx->mode == WASH_MODE_AUTO) {
             double coordinates = 0.0;
             for (int s = 0; s < ctx->n_seg; ++s) coordinates += static_cast<double>(ctx->seg_host[s].numel);
-            // measured crossover of the two kernels: serving a coordinate costs a 128-byte DRAM access per model
-            // and stack in [N][P], one or two for all N models in [P][N]
-            const double share = ctx->layout == WASH_LAYOUT_PN ? 0.10 : 0.03;
+            // measured crossovers of the two kernels (fp32, 2^25-2^26 coordinates): serving a coordinate costs a
+            // 128-byte DRAM access per model and stack in [N][P], one or two for all N models in [P][N]; and a
+            // small population leaves the streaming kernel bound by issue slots, not by the stack's bytes.
+            // [N][P]: N = 2 17 %, 4 10 %, 8 4 %, 16 2.5 %, 32 3-5 %; [P][N]: N <= 8 above 30 %, 16 10 %, 32 12 %
+            const double share = ctx->layout == WASH_LAYOUT_PN ? (ctx->N <= 8 ? 0.30 : 0.10) : std::fmax(0.03, 0.35 / ctx->N);
             mode = ctx->expected_selected < share * coordinates ? WASH_MODE_SPARSE : WASH_MODE_STREAM;
         }
         double coordinates = 0.0;

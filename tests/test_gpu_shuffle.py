@@ -311,8 +311,8 @@ def test_resume_from_a_host_copy_continues_bit_identically():
 
 
 def test_auto_mode_takes_either_kernel_and_keeps_the_bits():
-    """WASH_MODE_AUTO picks the sparse kernel below 3 % expected selection ([N][P]; 10 % in [P][N])
-    and the streaming one above; a per-layer vector is judged by its expectation over the whole model."""
+    """WASH_MODE_AUTO picks the sparse kernel below a share of expected selection (N = 6 in [N][P]:
+    5.8 %) and the streaming one above; a per-layer vector is judged by its expectation over the whole model."""
     N = 6
     numel = [70000, 9, 3000]
     c = Case(N, numel, 0, "f32", "f32", seed=21)
