@@ -190,6 +190,24 @@ def test_last_layer_untouched_and_schedules_agree_with_oracle():
     c.close()
 
 
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("N", [2, 4])
+def test_resident_warp_kernel_with_a_padded_coordinate_major_image(N, dtype):
+    """[P][N] with an even N and a quarter of the coordinates selected: the shared-memory image is
+    padded against bank conflicts while the small-group streaming kernel is still the one launched
+    (forced here for N = 4 in fp32, whose groups it does not take by default)."""
+    c = Case(N, [300_007, 12, 40_000], 1, dtype, None, seed=90 + N)
+    B.wash_set_launch(c.gpu.ctx, 0, -4)
+    tot = [0, 0]
+    for step in (0, 1):
+        B.wash_shuffle(c.gpu.ctx, step, 0.25, None, seed=5, stats=c.stats_dev)
+        s = oracle.shuffle(c.ora, c.host, 0.25, seed=5, step=step)
+        tot[0] += s[0]; tot[1] += s[1]
+        c.assert_equal("N=%d %s step=%d" % (N, dtype, step))
+    assert c.gpu_stats() == tuple(tot)
+    c.close()
+
+
 @pytest.mark.parametrize("N", [2, 4])
 def test_shards_reproduce_the_unsharded_shuffle(N):
     """Coordinate shards keyed by the global (tensor, coordinate) need no communication
