@@ -134,7 +134,8 @@ int wash_set_mode(wash_ctx *ctx, int32_t mode);
  * blocks_per_sm = -4 / -5 forces / excludes the streaming kernel for small groups (a
  * resident grid of warps walking tiles through two shared-memory stages; by default
  * it is launched when a group of all models of both stacks is at most 48 bytes and the
- * call's probabilities select at most 30 %; it ignores `threads`).  Results do not
+ * call's probabilities select at most 30 %, and for groups of up to 64 bytes when they
+ * select between 0.7 % and 5 %; it ignores `threads`).  Results do not
  * depend on any of this. */
 int wash_set_launch(wash_ctx *ctx, int32_t threads, int32_t blocks_per_sm);
 

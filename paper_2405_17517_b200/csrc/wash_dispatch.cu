@@ -119,6 +119,8 @@ static cudaError_t launch_shuffle_kernel(const ShuffleArgs &args, int a_dtype, i
     const size_t elem_a = a_dtype == kDtypeF32 ? 4 : a_dtype == kDtypeBF16 ? 2 : 0, elem_b = b_dtype == kDtypeF32 ? 4 : b_dtype == kDtypeBF16 ? 2 : 0;
     const size_t per_group = static_cast<size_t>(args.pop.N) * 4 * (elem_a + elem_b);
     bool loop = per_group <= kLoopMaxGroupBytes && args.expected_share <= kLoopMaxShare;
+    // 64-byte groups (fp32 N = 4, two fp32 stacks of N = 2, bf16 N = 8): only where serving weighs most
+    if (per_group > kLoopMaxGroupBytes && per_group <= kLoopWideGroupBytes) loop = args.expected_share >= kLoopWideShareLo && args.expected_share <= kLoopWideShareHi;
     if (shape.blocks_per_sm == -4) loop = true;
     if (shape.blocks_per_sm == -5 || args.sq.slots || args.early) loop = false;
     if (loop) return launch_shuffle_stream_loop(args, a_dtype, b_dtype, shape, stream, supported);

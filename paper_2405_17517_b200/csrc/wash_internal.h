@@ -134,6 +134,10 @@ enum ReduceOp { kOpEma = 0, kOpAverage = 1, kOpPapaAll = 2, kOpConsensus = 3 };
 // against the one-trip kernel: 32 bytes 0.73-0.93 of its time, 48 bytes 0.89-0.98, 64 bytes 0.97-1.12.
 constexpr size_t kLoopMaxGroupBytes = 48;
 constexpr float kLoopMaxShare = 0.3f;
+// Groups of 49 to 64 bytes go to it only for an expected selection between 0.7 % and 5 %: measured at 1 % and 3 %
+// it takes 0.89-0.97 of the one-trip kernel's time (both layouts), at 0.3 % 1.01-1.03, at 10 % 0.93 in [P][N] but 1.20 in [N][P].
+constexpr size_t kLoopWideGroupBytes = 64;
+constexpr float kLoopWideShareLo = 0.007f, kLoopWideShareHi = 0.05f;
 
 struct LaunchShape {
     int threads;         // 0 = default

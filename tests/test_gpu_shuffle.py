@@ -97,7 +97,7 @@ def test_streaming_flavours_on_dense_and_mixed_selection(N, dtype, opt_dtype, la
 
 @pytest.mark.parametrize("code", [-4, -5, 0], ids=["resident", "one-trip", "default"])
 @pytest.mark.parametrize("layout", [0, 1])
-@pytest.mark.parametrize("N,dtype,opt_dtype", [(2, "f32", None), (2, "bf16", "f32"), (3, "f32", "f32"), (4, "bf16", None), (8, "f32", None), (17, "bf16", "bf16")])
+@pytest.mark.parametrize("N,dtype,opt_dtype", [(2, "f32", None), (2, "bf16", "f32"), (3, "f32", "f32"), (4, "bf16", None), (4, "f32", None), (8, "f32", None), (17, "bf16", "bf16")])
 def test_resident_warp_streaming_kernel(N, dtype, opt_dtype, layout, code):
     """The streaming kernel for small groups (a resident grid of warps walking tiles with two
     shared-memory stages), forced, excluded and as the library chooses, against the oracle: enough
