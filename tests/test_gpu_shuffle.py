@@ -340,3 +340,42 @@ def test_auto_mode_takes_either_kernel_and_keeps_the_bits():
         oracle.shuffle(c.ora, c.host, p if pl is None else pl, seed=77, step=step, stack2=c.host_opt)
         c.assert_equal("step %d" % step)
     c.close()
+
+
+@pytest.mark.parametrize("seed", [11, 12, 13])
+def test_random_configurations_match_oracle(seed):
+    """Seeded random draws of population size, layout, dtypes, tensor table, probabilities (uniform
+    or per layer), kernel family and forced streaming flavour: stacks, padding and counters equal
+    the oracle's after two steps each."""
+    import random
+    rng = random.Random(seed)
+    for it in range(40):
+        N = rng.choice([2, 2, 3, 3, 4, 4, 5, 6, 8, 9, 12, 16, 17, 24, 32, 33])
+        layout = rng.randint(0, 1)
+        dtype = rng.choice(["f32", "bf16"])
+        opt = rng.choice([None, None, "f32", "bf16"])
+        T = rng.randint(1, 6)
+        big = rng.choice([20000, 200000, 700000 if N <= 8 else 60000])
+        numel = [rng.choice([1, 3, 4, 5, 8, 31, 33, 260, 4099, rng.randint(1, big)]) for _ in range(T)]
+        numel[rng.randrange(T)] = rng.randint(big // 2, big)
+        mode = rng.choice([B.WASH_MODE_STREAM, B.WASH_MODE_STREAM, B.WASH_MODE_SPARSE, B.WASH_MODE_AUTO])
+        code = rng.choice([0, 0, -4, -5, -2, -3])
+        uniform = rng.random() < 0.5
+        p = rng.choice([0.0005, 0.003, 0.01, 0.03, 0.1, 0.25, 0.6, 1.0]) if uniform else 0.0
+        pl = None if uniform else [rng.choice([0.0, 0.002, 0.01, 0.05, 0.3, 1.0]) for _ in range(T)]
+        what = "seed %d case %d: N=%d layout=%d %s/%s numel=%s mode=%d code=%d p=%s" % (seed, it, N, layout, dtype, opt, numel, mode, code, p if uniform else pl)
+        c = Case(N, numel, layout, dtype, opt, seed=1000 * seed + it)
+        B.wash_set_mode(c.gpu.ctx, mode)
+        B.wash_set_launch(c.gpu.ctx, 0, code)
+        tot = [0, 0]
+        for step in (it, (it << 33) | 7):
+            if opt is None:
+                B.wash_shuffle(c.gpu.ctx, step, p, pl, seed=it * 77 + 1, stats=c.stats_dev)
+            else:
+                B.wash_shuffle_both(c.gpu.ctx, step, p, pl, seed=it * 77 + 1, stats=c.stats_dev)
+            s = oracle.shuffle(c.ora, c.host, p if uniform else pl, seed=it * 77 + 1, step=step, stack2=c.host_opt)
+            tot[0] += s[0]; tot[1] += s[1]
+            c.assert_equal(what)
+        assert c.gpu_stats() == tuple(tot), what
+        B.wash_check(c.gpu.ctx)
+        c.close()
