@@ -51,6 +51,9 @@ def test_two_calls_in_a_row_match_the_context_based_shuffle():
         dict(N=8, numel=[64, 40000, 9], layout=1, bf16=True, step=(2 << 32) | 7, p=0.0, p_layer=[1.0, 0.01, 0.5], seed=12),
         # and the first shape again, next step
         dict(N=5, numel=[1000, 33, 7, 1, 4, 8, 5003, 2048], layout=0, bf16=False, step=4, p=0.25, p_layer=None, seed=11),
+        # small groups: the entry point launches the streaming kernel for them (several trips per warp here)
+        dict(N=2, numel=[700001, 5, 4099], layout=0, bf16=False, step=9, p=0.02, p_layer=None, seed=13),
+        dict(N=3, numel=[33, 90000, 7], layout=1, bf16=False, step=10, p=0.0, p_layer=[1.0, 0.3, 0.0], seed=14),
     ]
     for c in calls:
         stack, P, host, off = _make(c["N"], c["numel"], c["layout"], c["bf16"], seed=c["seed"])
